@@ -1,0 +1,174 @@
+"""Seeded synthetic inputs for the BlockFFN chunk-verify FFN path.
+
+This module holds data generation only: random draws, the bf16 storage format
+and the workload shapes. None of the method's arithmetic (router, union, expert
+FFN) lives here, so the CUDA path and the CPU checker can both be fed from it
+without sharing any computation.
+
+Random numbers come from numpy's counter-based Philox generator, keyed by
+(seed, stream id), so every tensor of every layer and chunk has its own
+reproducible stream regardless of generation order.
+
+The workloads stand in for the paper's trained checkpoints and decoding traces,
+which are not available: the shapes follow the paper's model table (hidden size,
+expert width, expert count), and the score generator reproduces the operating
+point the paper reports (about 80 % token-level sparsity with about 30 % of the
+experts in the union of an 8-token chunk).
+"""
+from __future__ import annotations
+
+from dataclasses import dataclass
+
+import numpy as np
+
+BASE_SEED = 0xB10CFF
+
+
+# ----------------------------------------------------------------------------
+# bf16 storage (bit patterns in uint16)
+# ----------------------------------------------------------------------------
+def f32_to_bf16_bits(a: np.ndarray) -> np.ndarray:
+    """float32 -> bf16 bit patterns, round to nearest even (NaN kept quiet)."""
+    a = np.ascontiguousarray(a, dtype=np.float32)
+    w = a.view(np.uint32)
+    lsb = (w >> np.uint32(16)) & np.uint32(1)
+    r = ((w + np.uint32(0x7FFF) + lsb) >> np.uint32(16)).astype(np.uint16)
+    nan = (w & np.uint32(0x7FFFFFFF)) > np.uint32(0x7F800000)
+    if nan.any():
+        r = np.where(nan, ((w >> np.uint32(16)) | np.uint32(0x40)).astype(np.uint16), r)
+    return r
+
+
+def bf16_bits_to_f32(b: np.ndarray) -> np.ndarray:
+    """bf16 bit patterns -> float32 (exact)."""
+    b = np.ascontiguousarray(b, dtype=np.uint16)
+    return (b.astype(np.uint32) << np.uint32(16)).view(np.float32)
+
+
+# ----------------------------------------------------------------------------
+# shapes
+# ----------------------------------------------------------------------------
+@dataclass(frozen=True)
+class Shape:
+    """One FFN layer shape. d = hidden size, E = experts, d_e = expert width."""
+    name: str
+    d: int
+    E: int
+    d_e: int
+    L: int              # default chunk length
+    union_frac: float   # fraction of experts in the chunk union (scores-in workloads)
+
+    @property
+    def u(self) -> int:
+        return int(round(self.union_frac * self.E))
+
+    @property
+    def expert_bytes(self) -> int:
+        """bf16 bytes of one expert (up and down blocks)."""
+        return 2 * self.d_e * self.d * 2
+
+    def active_bytes(self, u: int | None = None) -> int:
+        return (self.u if u is None else u) * self.expert_bytes
+
+
+# index = position in the benchmark's configuration list
+SHAPES = {
+    0: Shape("tiny", d=256, E=16, d_e=64, L=4, union_frac=1.0),
+    1: Shape("scores_in_0p8b", d=1536, E=48, d_e=128, L=8, union_frac=0.3),
+    2: Shape("l_sweep", d=2048, E=64, d_e=128, L=8, union_frac=0.3),
+    3: Shape("full_layer", d=2048, E=64, d_e=128, L=8, union_frac=0.3),
+    4: Shape("stack24", d=2048, E=64, d_e=128, L=8, union_frac=0.3),
+}
+STACK_LAYERS = 24
+STACK_CHUNKS = 256
+L_SWEEP = (1, 2, 4, 8, 16, 32)
+ROUTER_BIAS_SHIFT = -0.8     # in units of the logit's standard deviation (= 1 here)
+
+# stream ids (second half of the Philox key)
+_T_X, _T_WR, _T_GAIN, _T_U, _T_D, _T_SCORES, _T_MISC = range(7)
+
+
+def stream(seed: int, tensor: int, layer: int = 0, chunk: int = 0) -> np.random.Generator:
+    """Independent generator for (seed, tensor kind, layer, chunk)."""
+    sid = (tensor & 0xFF) | ((layer & 0xFFFF) << 8) | ((chunk & 0xFFFFFFFF) << 24)
+    return np.random.Generator(np.random.Philox(key=[seed & (2**64 - 1), sid]))
+
+
+def config_seed(index: int) -> int:
+    return BASE_SEED + index
+
+
+# ----------------------------------------------------------------------------
+# tensors
+# ----------------------------------------------------------------------------
+def _normal_bf16(g: np.random.Generator, shape, std: float) -> np.ndarray:
+    a = g.standard_normal(size=shape, dtype=np.float32)
+    a *= np.float32(std)
+    return f32_to_bf16_bits(a)
+
+
+def make_x(d: int, L: int, seed: int, layer: int = 0, chunk: int = 0) -> np.ndarray:
+    """Hidden states x ~ N(0, 1), bf16 bits [L][d]."""
+    return _normal_bf16(stream(seed, _T_X, layer, chunk), (L, d), 1.0)
+
+
+def make_correlated_x(d: int, L: int, rho: float, seed: int, chunk: int = 0) -> np.ndarray:
+    """x_t = sqrt(rho) * c + sqrt(1 - rho) * z_t with c, z_t ~ N(0, 1): neighbouring
+    tokens share a common component, as trained activation locality would give."""
+    g = stream(seed, _T_X, 0xC0, chunk)
+    c = g.standard_normal(size=(1, d), dtype=np.float32)
+    z = g.standard_normal(size=(L, d), dtype=np.float32)
+    return f32_to_bf16_bits(np.float32(np.sqrt(rho)) * c + np.float32(np.sqrt(1.0 - rho)) * z)
+
+
+def make_router(d: int, E: int, seed: int, layer: int = 0, bias_shift: float | None = None):
+    """Router parameters: W_r ~ N(0, std 1/sqrt(d)) bf16 [E][d]; gain ~ U(0.5, 1.5) f32 [E];
+    bias = a constant shift (f32 [E]) or None."""
+    W_r = _normal_bf16(stream(seed, _T_WR, layer), (E, d), 1.0 / np.sqrt(d))
+    gain = stream(seed, _T_GAIN, layer).uniform(0.5, 1.5, size=E).astype(np.float32)
+    bias = None if bias_shift is None else np.full(E, bias_shift, np.float32)
+    return W_r, gain, bias
+
+
+def make_experts(d: int, E: int, d_e: int, seed: int, layer: int = 0):
+    """Expert weights, bf16 bits: U [E][d_e][d] ~ N(0, std 1/sqrt(d)); D [E][d][d_e] ~ N(0, std 1/sqrt(d_e))."""
+    U = _normal_bf16(stream(seed, _T_U, layer), (E, d_e, d), 1.0 / np.sqrt(d))
+    D = _normal_bf16(stream(seed, _T_D, layer), (E, d, d_e), 1.0 / np.sqrt(d_e))
+    return U, D
+
+
+def make_scores(E: int, L: int, u: int, seed: int, layer: int = 0, chunk: int = 0,
+                tls_target: float = 0.8) -> np.ndarray:
+    """Router scores for one chunk, float32 [L][E], with a prescribed union.
+
+    A union of u experts is drawn uniformly without replacement. Each (token,
+    union expert) pair is active with probability p = (1 - tls_target) * E / u
+    (capped at 1); a union expert no token hit gets one token chosen uniformly,
+    so the union has exactly u members. Active scores are |N(0,1)| + 0.05, all
+    others exactly 0.0.
+    """
+    g = stream(seed, _T_SCORES, layer, chunk)
+    s = np.zeros((L, E), np.float32)
+    if u <= 0:
+        return s
+    members = np.sort(g.choice(E, size=u, replace=False))
+    p = min(1.0, (1.0 - tls_target) * E / u)
+    hit = g.random(size=(L, u)) < p
+    fix_tok = g.integers(0, L, size=u)
+    for q in range(u):
+        if not hit[:, q].any():
+            hit[fix_tok[q], q] = True
+    vals = np.abs(g.standard_normal(size=(L, u), dtype=np.float32)) + np.float32(0.05)
+    s[:, members] = np.where(hit, vals, np.float32(0.0))
+    return s
+
+
+def make_layer(shape: Shape, seed: int, layer: int = 0, with_router: bool = True,
+               bias_shift: float | None = None) -> dict:
+    """All parameters of one layer as a dict of numpy arrays."""
+    U, D = make_experts(shape.d, shape.E, shape.d_e, seed, layer)
+    out = {"U": U, "D": D}
+    if with_router:
+        W_r, gain, bias = make_router(shape.d, shape.E, seed, layer, bias_shift)
+        out.update({"W_r": W_r, "gain": gain, "bias": bias})
+    return out
