@@ -1,0 +1,461 @@
+#!/usr/bin/env python
+"""Benchmark of the BlockFFN chunk-verify FFN forward on B200.
+
+One step = one pass of the whole hot path (chunk union + expert FFN over the union
+experts, scores-in) over one batch of CHUNKS successive L-token chunks, each chunk
+reading a different copy of the layer's weights so that no weight byte is served
+from L2. The batch is captured once in a CUDA graph and replayed per step.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config 1|2|3|4] [--L 8]
+    python bench.py --impl reference      # the CPU oracle on the host cores
+
+Prints one JSON line (rank 0). `value` is active-expert-weight bytes per second.
+"""
+import argparse
+import json
+import math
+import os
+import subprocess
+import sys
+import tempfile
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2507_08771_b200 import inputs as I  # noqa: E402
+
+METRIC = "chunk-verify FFN active-weight HBM GB/s (latency us per chunk alongside)"
+L2_BYTES = 126e6
+NOMINAL_HBM_GBS = 8000.0
+FALLBACK_HBM_GBS = 6650.0
+
+
+def parse():
+    p = argparse.ArgumentParser()
+    p.add_argument("--gpus", type=int, default=1)
+    p.add_argument("--steps", type=int, default=20)
+    p.add_argument("--warmup", type=int, default=5)
+    p.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    p.add_argument("--config", type=int, default=1, choices=[1, 2, 3, 4])
+    p.add_argument("--L", type=int, default=None, help="chunk length (default: the config's)")
+    p.add_argument("--chunks", type=int, default=256, help="chunks per step")
+    p.add_argument("--variant", type=int, default=0, help="0 auto, 1 CUDA-core, 2 tensor-core")
+    p.add_argument("--no-cpu-baseline", action="store_true")
+    p.add_argument("--sweep", action="store_true", help="also report every L of the sweep (config 2)")
+    return p.parse_args()
+
+
+def measured_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+def copies_needed(active_bytes):
+    """Enough weight copies that twice the L2 is streamed between two uses of one copy."""
+    return max(8, int(math.ceil(2 * L2_BYTES / active_bytes)) + 1)
+
+
+class ClockSampler:
+    """nvidia-smi clock / throttle-reason samples while the timed region runs."""
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+         "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index):
+        self.gpu = gpu_index
+        self.proc = None
+        self.path = None
+
+    def start(self):
+        try:
+            fd, self.path = tempfile.mkstemp(suffix=".csv")
+            os.close(fd)
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.gpu), f"--query-gpu={self.Q}",
+                 "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return out
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        try:
+            for line in open(self.path):
+                f = [v.strip() for v in line.split(",")]
+                if len(f) < 9:
+                    continue
+                try:
+                    sm.append(float(f[1])); mx.append(float(f[2]))
+                except ValueError:
+                    continue
+                for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown",
+                                    "sw_power_cap"), f[5:9]):
+                    if v.lower().startswith("active"):
+                        reasons.add(name)
+            os.unlink(self.path)
+        except Exception:
+            pass
+        if sm:
+            out.update(sm_mhz=float(np.median(sm)), sm_max_mhz=float(max(mx)), samples=len(sm),
+                       reasons=sorted(reasons))
+        return out
+
+
+# ----------------------------------------------------------------------------
+# workload
+# ----------------------------------------------------------------------------
+class Workload:
+    """Device-resident synthetic inputs for one benchmark configuration."""
+
+    def __init__(self, cfg_index, L, chunks, variant, device):
+        import torch
+        from paper_2507_08771_b200 import binding as B
+        self.torch, self.B = torch, B
+        self.idx, self.chunks, self.device = cfg_index, chunks, device
+        self.sh = sh = I.SHAPES[cfg_index]
+        self.L = L or sh.L
+        seed = I.config_seed(cfg_index)
+        self.u = sh.u
+        self.active_bytes = sh.active_bytes()
+        self.layer = B.Layer(sh.d, sh.E, sh.d_e, L_max=max(self.L, 8), variant=variant, device=device)
+        if cfg_index == 4:
+            self.n_copies = I.STACK_LAYERS          # 24 distinct layers, 1.6 GB >> L2
+            host = [I.make_experts(sh.d, sh.E, sh.d_e, seed, layer=l) for l in range(self.n_copies)]
+        else:
+            self.n_copies = copies_needed(self.active_bytes)
+            one = I.make_experts(sh.d, sh.E, sh.d_e, seed)
+            host = [one] * self.n_copies             # same values, distinct device addresses
+        self.dws = []
+        for U, D in host:
+            tU, tD = B.to_device_bf16(U, device), B.to_device_bf16(D, device)
+            self.dws.append(B.DeviceWeights(B.make_weights(U=tU, D=tD), {"U": tU, "D": tD}))
+        self.host_weights = host
+        # per-chunk inputs, on the host (pinned) and on the device
+        n = chunks
+        if cfg_index == 4:
+            # chunk c runs through all 24 layers; scores differ per (layer, chunk)
+            self.calls_per_chunk = self.n_copies
+            sc = np.stack([np.stack([I.make_scores(sh.E, self.L, sh.u, seed, layer=l, chunk=c)
+                                     for l in range(self.n_copies)]) for c in range(n)])
+        else:
+            self.calls_per_chunk = 1
+            sc = np.stack([I.make_scores(sh.E, self.L, sh.u, seed, chunk=c) for c in range(n)])[:, None]
+        xs = np.stack([I.make_x(sh.d, self.L, seed, chunk=c) for c in range(n)])
+        self.scores_host = torch.from_numpy(sc).pin_memory()
+        self.x_host = torch.from_numpy(xs.view(np.int16)).pin_memory()
+        self.scores = self.scores_host.to(device)
+        self.x = self.x_host.to(device).view(torch.bfloat16)
+        self.out = torch.zeros(n, self.L, sh.d, dtype=torch.float32, device=device)
+        self.out_host = torch.empty(n, self.L, sh.d, dtype=torch.float32).pin_memory()
+        self.x_pp = torch.zeros(2, self.L, sh.d, dtype=torch.bfloat16, device=device)
+        self.ids = torch.zeros(n, self.calls_per_chunk, sh.E, dtype=torch.int32, device=device)
+        self.nu = torch.zeros(n, self.calls_per_chunk, dtype=torch.int32, device=device)
+        self.calls_per_step = n * self.calls_per_chunk
+        self.h2d_bytes = self.x_host.numel() * 2 + self.scores_host.numel() * 4
+        self.d2h_bytes = self.out_host.numel() * 4
+
+    # -- the hot path: union + expert FFN per chunk (and per layer for the stack) --
+    def enqueue_step(self, stream):
+        B, lay = self.B, self.layer
+        if self.idx == 4:
+            for c in range(self.chunks):
+                # residual stream: out[c] starts as h0 = f32(x[c]); x ping-pongs in bf16
+                self.out[c].copy_(self.x[c])
+                self.x_pp[0].copy_(self.x[c])
+                for l in range(self.n_copies):
+                    B.blockffn_layer_forward_scores(
+                        lay.h, self.dws[l].struct, self.x_pp[l % 2], self.scores[c, l], self.L,
+                        self.out[c], self.x_pp[(l + 1) % 2], lay.stats,
+                        B.CALL_ACCUMULATE | B.CALL_INDEPENDENT, stream)
+        else:
+            for c in range(self.chunks):
+                B.blockffn_layer_forward_scores(
+                    lay.h, self.dws[c % self.n_copies].struct, self.x[c], self.scores[c, 0], self.L,
+                    self.out[c], None, lay.stats, B.CALL_INDEPENDENT, stream)
+
+    # -- expert stage alone (the dominant kernels), unions precomputed --
+    def enqueue_unions(self, stream):
+        B, lay = self.B, self.layer
+        for c in range(self.chunks):
+            for l in range(self.calls_per_chunk):
+                B.blockffn_chunk_union(lay.h, self.scores[c, l], self.L, None, self.ids[c, l],
+                                       self.nu[c, l:l + 1], None, stream)
+
+    def enqueue_expert_only(self, stream):
+        B, lay = self.B, self.layer
+        for c in range(self.chunks):
+            for l in range(self.calls_per_chunk):
+                k = l if self.idx == 4 else c % self.n_copies
+                B.blockffn_expert_ffn(lay.h, self.dws[k].struct, self.x[c], self.scores[c, l], self.L,
+                                      self.ids[c, l], self.nu[c, l:l + 1], self.out[c], None,
+                                      B.CALL_INDEPENDENT, stream)
+
+
+def capture(torch, stream, fn):
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(stream):
+        fn(stream)                      # eager once: warms up, surfaces errors
+        stream.synchronize()
+        with torch.cuda.graph(g, stream=stream):
+            fn(stream)
+    return g
+
+
+def time_replays(torch, stream, graph, steps, warmup, pre=None, post=None):
+    with torch.cuda.stream(stream):
+        for _ in range(warmup):
+            if pre:
+                pre()
+            graph.replay()
+            if post:
+                post()
+        stream.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(steps):
+            if pre:
+                pre()
+            graph.replay()
+            if post:
+                post()
+        e1.record(stream)
+        stream.synchronize()
+    return e0.elapsed_time(e1) / steps      # ms per step
+
+
+# ----------------------------------------------------------------------------
+# CPU oracle legs
+# ----------------------------------------------------------------------------
+def oracle_sample(cfg_index, L, budget_s, max_chunks):
+    """Times the CPU oracle (as it stands, one thread) on successive chunks of the
+    workload until the time budget is used. Returns (GB/s of active weights, us/chunk, n)."""
+    import oracle
+    sh = I.SHAPES[cfg_index]
+    L = L or sh.L
+    seed = I.config_seed(cfg_index)
+    U, D = I.make_experts(sh.d, sh.E, sh.d_e, seed)
+    oracle.build()
+    t_total, n = 0.0, 0
+    while n < max_chunks and (t_total < budget_s or n == 0):
+        x = I.make_x(sh.d, L, seed, chunk=n)
+        s = I.make_scores(sh.E, L, sh.u, seed, chunk=n)
+        t0 = time.perf_counter()
+        oracle.layer_forward_scores(x, s, U, D, union_only=True)
+        t_total += time.perf_counter() - t0
+        n += 1
+    per = t_total / n
+    return sh.active_bytes() / per / 1e9, per * 1e6, n
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    sh = I.SHAPES[args.config]
+    L = args.L or sh.L
+    per_step_chunks = 2
+    import oracle
+    oracle.build()
+    seed = I.config_seed(args.config)
+    U, D = I.make_experts(sh.d, sh.E, sh.d_e, seed)
+
+    def step(k):
+        for c in range(per_step_chunks):
+            x = I.make_x(sh.d, L, seed, chunk=k * per_step_chunks + c)
+            s = I.make_scores(sh.E, L, sh.u, seed, chunk=k * per_step_chunks + c)
+            oracle.layer_forward_scores(x, s, U, D, union_only=True)
+
+    for k in range(args.warmup):
+        step(k)
+    t0 = time.perf_counter()
+    for k in range(args.steps):
+        step(k)
+    dt = (time.perf_counter() - t0) / args.steps
+    gbs = per_step_chunks * sh.active_bytes() / dt / 1e9
+    sample = (f"{per_step_chunks} chunks per step of config {args.config} "
+              f"(d={sh.d}, E={sh.E}, d_e={sh.d_e}, L={L}, union {sh.u}), union-restricted sum, float64")
+    line = {
+        "impl": "reference", "metric": METRIC, "value": gbs, "unit": "GB/s", "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt * 1e3,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+        "data": "synthetic", "latency_us_per_chunk": dt / per_step_chunks * 1e6,
+        "config": {"workload": f"config {args.config}: {sh.name}", "d": sh.d, "E": sh.E,
+                   "d_e": sh.d_e, "L": L, "union": sh.u, "chunks_per_step": per_step_chunks},
+        "cpu_baseline": {"value": gbs, "unit": "GB/s", "cores": 1, "kind": "oracle", "sample": sample},
+        "e2e": {"value": gbs, "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+# ----------------------------------------------------------------------------
+# main
+# ----------------------------------------------------------------------------
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+    from paper_2507_08771_b200 import binding as B
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback); "
+                         "use --impl reference for the CPU oracle")
+    torch.cuda.set_device(local)
+    device = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=device)
+    B.load()
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    wl = Workload(args.config, args.L, args.chunks, args.variant, device)
+    sh = wl.sh
+    stream = torch.cuda.Stream(device)
+    lay = wl.layer
+
+    n0 = lay.launch_count()
+    g_step = capture(torch, stream, wl.enqueue_step)
+    launches_per_step = (lay.launch_count() - n0) // 2       # fn ran twice (eager + capture)
+    with torch.cuda.stream(stream):
+        wl.enqueue_unions(stream)
+        stream.synchronize()
+    n0 = lay.launch_count()
+    g_expert = capture(torch, stream, wl.enqueue_expert_only)
+    expert_launches = (lay.launch_count() - n0) // 2
+
+    sampler = ClockSampler(local)
+    barrier()
+    if rank == 0:
+        sampler.start()
+    ms_step = time_replays(torch, stream, g_step, args.steps, args.warmup)
+    barrier()
+    clocks = sampler.stop() if rank == 0 else {}
+
+    # end to end: host buffers in, host buffers out, copies inside the timed region
+    def pre():
+        wl.x.view(torch.int16).copy_(wl.x_host, non_blocking=True)
+        wl.scores.copy_(wl.scores_host, non_blocking=True)
+
+    def post():
+        wl.out_host.copy_(wl.out, non_blocking=True)
+
+    barrier()
+    ms_e2e = time_replays(torch, stream, g_step, max(3, args.steps // 2), 3, pre, post)
+    barrier()
+    ms_expert = time_replays(torch, stream, g_expert, args.steps, args.warmup)
+    barrier()
+    status = lay.last_status()
+    assert status == 0, f"device status word {status}"
+    assert torch.isfinite(wl.out).all()
+
+    t = torch.tensor([ms_step, ms_e2e, ms_expert], dtype=torch.float64, device=device)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    ms_step, ms_e2e, ms_expert = (float(v) for v in t.cpu())
+
+    calls = wl.calls_per_step
+    bytes_step = calls * wl.active_bytes
+    value = world * bytes_step / (ms_step * 1e-3) / 1e9
+    e2e = world * bytes_step / (ms_e2e * 1e-3) / 1e9
+    peak, peak_kind = measured_peak()
+    # algorithmic bytes of one expert-stage call: weights + x + out + scores
+    alg_bytes = wl.active_bytes + 2 * wl.L * sh.d + 4 * wl.L * sh.d + 4 * wl.L * sh.E
+    us_expert = ms_expert * 1e3 / calls
+    achieved = alg_bytes / (us_expert * 1e-6) / 1e9
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    line = {
+        "metric": METRIC, "value": value, "unit": "GB/s", "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "bf16 weights, f32 accumulate",
+        "data": "synthetic",
+        "latency_us_per_chunk": ms_step * 1e3 / wl.chunks,
+        "latency_us_per_layer_call": ms_step * 1e3 / calls,
+        "pct_of_nominal_8TBs": 100.0 * value / world / NOMINAL_HBM_GBS,
+        "config": {
+            "workload": f"config {args.config}: {sh.name} (scores-in: chunk union + expert FFN)",
+            "d": sh.d, "E": sh.E, "d_e": sh.d_e, "L": wl.L, "union": wl.u,
+            "chunks_per_step": wl.chunks, "layer_calls_per_step": calls,
+            "active_bytes_per_call": wl.active_bytes, "weight_copies": wl.n_copies,
+            "l2": f"inputs larger than L2: {wl.n_copies} weight copies rotated, "
+                  f"{wl.n_copies * wl.active_bytes / 1e6:.0f} MB streamed between reuses",
+            "replicas": "independent replicas per GPU, no collective" if world > 1 else "single GPU",
+            "variant": args.variant,
+        },
+        "clocks": clocks,
+        "e2e": {"value": e2e, "unit": "GB/s", "h2d_bytes_per_step": wl.h2d_bytes,
+                "d2h_bytes_per_step": wl.d2h_bytes, "ms_per_step": ms_e2e},
+        "gpu_launches": launches_per_step * args.steps,
+        "gpu_launches_per_step": launches_per_step,
+        "roofline": {
+            "bound": "hbm", "kernel": "expert stage (up + down projection kernels of one call)",
+            "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+            "peak_kind": f"of {peak_kind}", "us_per_launch": us_expert,
+            "algorithmic_bytes_per_launch": alg_bytes, "launches_per_call": expert_launches // calls,
+            "traffic": None,
+        },
+    }
+    if not args.no_cpu_baseline and world == 1:
+        gbs, us, n = oracle_sample(args.config, wl.L, budget_s=12.0, max_chunks=64)
+        line["cpu_baseline"] = {
+            "value": gbs, "unit": "GB/s", "cores": 1, "kind": "oracle", "us_per_chunk": us,
+            "sample": f"{n} chunks of the same workload (one layer call each), union-restricted "
+                      f"sum, float64, single thread"}
+    if args.sweep and args.config == 2:
+        line["sweep"] = sweep(args, torch, device)
+    print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def sweep(args, torch, device):
+    rows = []
+    for L in I.L_SWEEP:
+        for variant in (1, 2):
+            try:
+                wl = Workload(2, L, args.chunks, variant, device)
+            except Exception as e:  # a variant that does not support the shape
+                rows.append({"L": L, "variant": variant, "error": str(e)})
+                continue
+            stream = torch.cuda.Stream(device)
+            g = capture(torch, stream, wl.enqueue_step)
+            ms = time_replays(torch, stream, g, args.steps, args.warmup)
+            us = ms * 1e3 / wl.chunks
+            rows.append({"L": L, "variant": variant, "us_per_chunk": us,
+                         "GBps": wl.active_bytes / (us * 1e-6) / 1e9})
+            del wl, g
+            torch.cuda.empty_cache()
+    return rows
+
+
+if __name__ == "__main__":
+    a = parse()
+    if a.impl == "reference":
+        run_reference(a)
+    else:
+        run_ours(a)

@@ -1,0 +1,181 @@
+/*
+ * blockffn.h - C ABI of the BlockFFN chunk-verify FFN forward for NVIDIA B200 (sm_100a).
+ *
+ * One call evaluates one BlockFFN layer for a chunk of L draft tokens that a
+ * speculative-decoding step verifies in parallel (Sec. 3.3 of the BlockFFN paper):
+ *   1. router       A(x) = RMSNorm(ReLU(W_router^T x))                       (Eq. 3)
+ *   2. chunk union  Union(x) = experts activated by any of the L tokens      (Sec. 3.3)
+ *   3. expert FFN   FFN(x_t) = sum_{i in Union} A_i(x_t) W_down^(i)T Swish(W_up^(i)T x_t)
+ *                                                                            (Eq. 1, Eq. 2)
+ * Only the union experts' weights are read from device memory.
+ *
+ * Conventions (all entry points)
+ *   - Every data pointer is a DEVICE pointer owned by the caller, 16-byte aligned,
+ *     valid until the work enqueued by the call has finished. The library owns only
+ *     the workspace inside its handle.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).
+ *     Calls only enqueue work: no allocation, no host synchronisation, no copy to
+ *     the host. Two calls on one handle must not run concurrently on the device
+ *     (they share the handle's workspace); use one handle per stream.
+ *   - Row-major layouts. bf16 = the upper 16 bits of an IEEE float32.
+ *       x       bf16 [L][d]           hidden states of the chunk
+ *       scores  f32  [L][E]           A(x); expert i is active for token t iff
+ *                                     scores[t][i] != 0.0f by value (-0.0f is zero,
+ *                                     NaN counts as active and propagates)
+ *       out     f32  [L][d]
+ *   - The return value reports what the host can detect (bad arguments, launch
+ *     failures). Problems found on the device (a union id out of range, a count
+ *     larger than E) set bits in a sticky status word, skip the offending work and
+ *     never fault; read it with blockffn_last_status().
+ *   - Limits: 1 <= L <= L_max <= 32 per call; d % 8 == 0; d_e % 8 == 0;
+ *     1 <= E <= 1024.
+ */
+#ifndef BLOCKFFN_H_
+#define BLOCKFFN_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#if defined(_WIN32)
+#define BLOCKFFN_API
+#else
+#define BLOCKFFN_API __attribute__((visibility("default")))
+#endif
+
+typedef enum {
+  BLOCKFFN_OK = 0,
+  BLOCKFFN_ERR_INVALID_ARG = 1, /* NULL / misaligned pointer, size out of range   */
+  BLOCKFFN_ERR_UNSUPPORTED = 2, /* shape outside the limits above                 */
+  BLOCKFFN_ERR_WORKSPACE = 3,   /* workspace allocation failed in blockffn_create */
+  BLOCKFFN_ERR_CUDA = 4,        /* a CUDA runtime call or launch failed           */
+  BLOCKFFN_ERR_DEVICE = 5       /* the device status word is nonzero              */
+} blockffn_status;
+
+/* Bits of the device status word (blockffn_last_status). */
+#define BLOCKFFN_DEV_BAD_UNION_ID 1u    /* a union id was < 0 or >= E: that entry was skipped   */
+#define BLOCKFFN_DEV_BAD_UNION_COUNT 2u /* n_union was < 0 or > E: it was clamped               */
+#define BLOCKFFN_DEV_WAIT_EXPIRED 4u    /* a bounded on-chip wait ran out: the call's out is invalid */
+
+/* Kernel family used by the expert stage. AUTO picks by L and shape. */
+#define BLOCKFFN_VARIANT_AUTO 0
+#define BLOCKFFN_VARIANT_SIMT 1   /* CUDA-core dot products, fp32 intermediate             */
+#define BLOCKFFN_VARIANT_MMA 2    /* bulk-copy staged, tensor-core tiles, bf16 intermediate */
+
+typedef struct {
+  int32_t d;       /* hidden size d_h                                          */
+  int32_t E;       /* number of experts N_e                                    */
+  int32_t d_e;     /* expert width                                             */
+  int32_t L_max;   /* largest chunk length a call may pass (<= 32)             */
+  float rms_eps;   /* RMSNorm epsilon, added to the mean square (Eq. 3); 1e-6  */
+  int32_t variant; /* BLOCKFFN_VARIANT_*                                       */
+  int32_t flags;   /* reserved, 0                                              */
+} blockffn_config;
+
+/* Layer parameters: device pointers, caller-owned, read-only to the library. */
+typedef struct {
+  const void* W_r;   /* bf16 [E][d]: row i = column i of W_router (Eq. 3). May be NULL for
+                        scores-in calls.                                                   */
+  const float* gain; /* f32 [E]: RMSNorm gain (Eq. 3). May be NULL for scores-in calls.    */
+  const float* bias; /* f32 [E] added to the router logits, or NULL (NULL = Eq. 3 as
+                        printed; a synthetic router uses it to set its sparsity).          */
+  const void* U;     /* bf16 [E][d_e][d]: U[i][j][k] = W_up^(i)[k][j]   (Eq. 2)            */
+  const void* D;     /* bf16 [E][d][d_e]: D[i][c][j] = W_down^(i)[j][c] (Eq. 2)            */
+} blockffn_weights;
+
+/* Counters behind TLS and CLS_L (Sec. 2.1), accumulated on the device, one chunk per call. */
+typedef struct {
+  uint64_t n_tokens; /* tokens seen                                  */
+  uint64_t n_active; /* sum over tokens of |experts active for it|   */
+  uint64_t n_chunks; /* chunks seen                                  */
+  uint64_t n_union;  /* sum over chunks of |Union|                   */
+} blockffn_stats;
+
+/* Per-call flags. */
+#define BLOCKFFN_CALL_ACCUMULATE 1 /* out += FFN(x) (residual, fp32) instead of out = FFN(x)     */
+#define BLOCKFFN_CALL_INDEPENDENT 2 /* promise: scores, union_ids, n_union and the weights of this
+                                       call were NOT written by the work enqueued just before it
+                                       on `stream`; only x and out may depend on it. Lets the call's
+                                       weight fetch start while the previous kernel drains.        */
+
+typedef struct blockffn_ctx* blockffn_handle;
+
+/* Creates a handle on the current CUDA device and allocates its workspace there
+ * (the only allocation the library ever makes). Returns WORKSPACE if that fails. */
+BLOCKFFN_API blockffn_status blockffn_create(const blockffn_config* cfg, blockffn_handle* out);
+/* Frees the workspace. The caller synchronises outstanding work first. */
+BLOCKFFN_API blockffn_status blockffn_destroy(blockffn_handle h);
+
+/* Eq. 3. scores[t][i] = gain[i] * a1 / sqrt(mean_i(a1^2) + rms_eps), a1 = max(0, x_t . W_r[i] + bias[i]);
+ * tok_mask[t][w] bit b = (scores[t][32 w + b] != 0), bits at and beyond E zero
+ * (tok_mask: u32 [L][ceil(E/32)], may be NULL). The mean runs over all E entries.      */
+BLOCKFFN_API blockffn_status blockffn_router(blockffn_handle h, const blockffn_weights* w,
+                                             const void* x, int32_t L, float* scores,
+                                             uint32_t* tok_mask, void* stream);
+
+/* Sec. 3.3 Union(x) from a score matrix: union_mask u32 [ceil(E/32)] (may be NULL);
+ * union_ids i32 [E], ascending expert ids, entries from n_union on are -1; n_union i32 [1]
+ * (device). stats (device, may be NULL) is advanced by this chunk (Sec. 2.1 counters). */
+BLOCKFFN_API blockffn_status blockffn_chunk_union(blockffn_handle h, const float* scores, int32_t L,
+                                                  uint32_t* union_mask, int32_t* union_ids,
+                                                  int32_t* n_union, blockffn_stats* stats,
+                                                  void* stream);
+
+/* Eq. 1 + Eq. 2 restricted to the listed experts: reads U_i, D_i only for
+ * i in union_ids[0 .. *n_union). out = (out +) sum_i scores[t][i] * D_i Swish(U_i x_t).
+ * x_next (bf16 [L][d], may be NULL, must not alias x) receives the bf16 rounding of the
+ * final out: the next layer's input when out is a running fp32 residual.
+ * An expert missing from the list contributes nothing, whatever its score.              */
+BLOCKFFN_API blockffn_status blockffn_expert_ffn(blockffn_handle h, const blockffn_weights* w,
+                                                 const void* x, const float* scores, int32_t L,
+                                                 const int32_t* union_ids, const int32_t* n_union,
+                                                 float* out, void* x_next, int32_t call_flags,
+                                                 void* stream);
+
+/* Whole layer, router on: Eq. 3 -> Union(x) -> Eq. 1/2, everything device side.
+ * The scores, masks, ids and count land in the handle's workspace
+ * (blockffn_read_routing). stats may be NULL.                                            */
+BLOCKFFN_API blockffn_status blockffn_layer_forward(blockffn_handle h, const blockffn_weights* w,
+                                                    const void* x, int32_t L, float* out,
+                                                    void* x_next, blockffn_stats* stats,
+                                                    int32_t call_flags, void* stream);
+
+/* Whole layer from precomputed router scores (the scores-in entry): Union(x) -> Eq. 1/2. */
+BLOCKFFN_API blockffn_status blockffn_layer_forward_scores(blockffn_handle h,
+                                                           const blockffn_weights* w, const void* x,
+                                                           const float* scores, int32_t L,
+                                                           float* out, void* x_next,
+                                                           blockffn_stats* stats,
+                                                           int32_t call_flags, void* stream);
+
+/* Enqueues device-to-device copies of what the last layer call on this handle derived
+ * (kept in the handle's workspace until the next call overwrites it) into caller buffers:
+ * scores f32 [L][E] and tok_mask u32 [L][ceil(E/32)] (router-on calls only),
+ * union_mask u32 [ceil(E/32)], union_ids i32 [E], n_union i32 [1]. Any may be NULL. */
+BLOCKFFN_API blockffn_status blockffn_read_routing(blockffn_handle h, int32_t L, float* scores,
+                                                   uint32_t* tok_mask, uint32_t* union_mask,
+                                                   int32_t* union_ids, int32_t* n_union,
+                                                   void* stream);
+
+/* Synchronises `stream`, then returns OK if the device status word is zero, DEVICE otherwise;
+ * *bits (may be NULL) receives the BLOCKFFN_DEV_* bits; clear != 0 resets the word.      */
+BLOCKFFN_API blockffn_status blockffn_last_status(blockffn_handle h, uint32_t* bits, int32_t clear,
+                                                  void* stream);
+
+/* Sec. 2.1, from a HOST copy of the counters: TLS = 1 - n_active / (n_tokens E),
+ * CLS_L = 1 - n_union / (n_chunks E) with L the chunk length of the calls counted.      */
+BLOCKFFN_API double blockffn_tls(const blockffn_stats* host_stats, int32_t E);
+BLOCKFFN_API double blockffn_cls(const blockffn_stats* host_stats, int32_t E);
+
+/* Number of kernels the library has launched through this handle (host counter). */
+BLOCKFFN_API uint64_t blockffn_launch_count(blockffn_handle h);
+
+/* Human-readable name of a status code (static storage). */
+BLOCKFFN_API const char* blockffn_status_string(blockffn_status s);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* BLOCKFFN_H_ */

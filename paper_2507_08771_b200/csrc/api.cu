@@ -1,0 +1,259 @@
+// C ABI of the BlockFFN library: argument checks, workspace, dispatch.
+#include <new>
+
+#include "common.cuh"
+
+namespace {
+
+inline bool misaligned(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) != 0; }
+inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+blockffn_status check_call(blockffn_ctx* c, int L) {
+  if (!c) return BLOCKFFN_ERR_INVALID_ARG;
+  if (L < 1 || L > c->cfg.L_max) return BLOCKFFN_ERR_INVALID_ARG;
+  return BLOCKFFN_OK;
+}
+
+blockffn_status expert_dispatch(blockffn_ctx* c, const blockffn_weights* w, const void* x,
+                                const float* scores, int L, const int32_t* union_ids,
+                                const int32_t* n_union, float* out, void* x_next, int call_flags,
+                                cudaStream_t st) {
+  cudaError_t e;
+  if (expert_mma_supported(c, L) && c->cfg.variant != BLOCKFFN_VARIANT_SIMT)
+    e = launch_expert_mma(c, w, x, scores, L, union_ids, n_union, out, x_next, call_flags, st);
+  else
+    e = launch_expert_simt(c, w, x, scores, L, union_ids, n_union, out, x_next, call_flags, st);
+  return e == cudaSuccess ? BLOCKFFN_OK : BLOCKFFN_ERR_CUDA;
+}
+
+}  // namespace
+
+extern "C" {
+
+blockffn_status blockffn_create(const blockffn_config* cfg, blockffn_handle* out) {
+  if (!cfg || !out) return BLOCKFFN_ERR_INVALID_ARG;
+  *out = nullptr;
+  if (cfg->d < 8 || cfg->d_e < 8 || cfg->E < 1 || cfg->L_max < 1) return BLOCKFFN_ERR_INVALID_ARG;
+  if (cfg->d % 8 || cfg->d_e % 8 || cfg->E > 1024 || cfg->L_max > 32 || cfg->d > (1 << 20) ||
+      cfg->d_e > (1 << 16))
+    return BLOCKFFN_ERR_UNSUPPORTED;
+  if (!(cfg->rms_eps >= 0.0f)) return BLOCKFFN_ERR_INVALID_ARG;
+  if (cfg->variant < BLOCKFFN_VARIANT_AUTO || cfg->variant > BLOCKFFN_VARIANT_MMA)
+    return BLOCKFFN_ERR_INVALID_ARG;
+  blockffn_ctx* c = new (std::nothrow) blockffn_ctx();
+  if (!c) return BLOCKFFN_ERR_WORKSPACE;
+  c->cfg = *cfg;
+  c->words = (cfg->E + 31) / 32;
+  c->launches = 0;
+  if (cudaGetDevice(&c->device) != cudaSuccess ||
+      cudaDeviceGetAttribute(&c->num_sms, cudaDevAttrMultiProcessorCount, c->device) !=
+          cudaSuccess) {
+    delete c;
+    return BLOCKFFN_ERR_CUDA;
+  }
+  const size_t E = cfg->E, L = cfg->L_max, d_e = cfg->d_e, W = c->words;
+  size_t off = 0;
+  auto take = [&](size_t bytes) {
+    size_t o = off;
+    off = align_up(off + bytes, 256);
+    return o;
+  };
+  const size_t o_a0 = take(sizeof(float) * L * E);
+  const size_t o_sc = take(sizeof(float) * L * E);
+  const size_t o_tm = take(sizeof(uint32_t) * L * W);
+  const size_t o_um = take(sizeof(uint32_t) * W);
+  const size_t o_id = take(sizeof(int32_t) * E);
+  const size_t o_nu = take(sizeof(int32_t));
+  const size_t o_h32 = take(sizeof(float) * E * L * d_e);
+  const size_t o_h16 = take(expert_mma_h_bytes(cfg));
+  const size_t o_tk = take(sizeof(unsigned int) * 8);
+  const size_t o_st = take(sizeof(uint32_t));
+  void* base = nullptr;
+  if (cudaMalloc(&base, off) != cudaSuccess) {
+    cudaGetLastError();
+    delete c;
+    return BLOCKFFN_ERR_WORKSPACE;
+  }
+  if (cudaMemset(base, 0, off) != cudaSuccess) {
+    cudaFree(base);
+    delete c;
+    return BLOCKFFN_ERR_CUDA;
+  }
+  char* b = static_cast<char*>(base);
+  c->ws_base = base;
+  c->a0 = reinterpret_cast<float*>(b + o_a0);
+  c->scores = reinterpret_cast<float*>(b + o_sc);
+  c->tok_mask = reinterpret_cast<uint32_t*>(b + o_tm);
+  c->union_mask = reinterpret_cast<uint32_t*>(b + o_um);
+  c->union_ids = reinterpret_cast<int32_t*>(b + o_id);
+  c->n_union = reinterpret_cast<int32_t*>(b + o_nu);
+  c->h32 = reinterpret_cast<float*>(b + o_h32);
+  c->h16 = b + o_h16;
+  c->ticket = reinterpret_cast<unsigned int*>(b + o_tk);
+  c->status = reinterpret_cast<uint32_t*>(b + o_st);
+  if (expert_mma_setup(c) != cudaSuccess) {
+    cudaFree(base);
+    delete c;
+    return BLOCKFFN_ERR_CUDA;
+  }
+  *out = c;
+  return BLOCKFFN_OK;
+}
+
+blockffn_status blockffn_destroy(blockffn_handle h) {
+  if (!h) return BLOCKFFN_ERR_INVALID_ARG;
+  cudaError_t e = cudaFree(h->ws_base);
+  delete h;
+  return e == cudaSuccess ? BLOCKFFN_OK : BLOCKFFN_ERR_CUDA;
+}
+
+blockffn_status blockffn_router(blockffn_handle h, const blockffn_weights* w, const void* x,
+                                int32_t L, float* scores, uint32_t* tok_mask, void* stream) {
+  blockffn_status s = check_call(h, L);
+  if (s != BLOCKFFN_OK) return s;
+  if (!w || !w->W_r || !w->gain || !x || !scores) return BLOCKFFN_ERR_INVALID_ARG;
+  if (misaligned(w->W_r) || misaligned(x) || misaligned(scores) ||
+      (reinterpret_cast<uintptr_t>(w->gain) & 3u) || (reinterpret_cast<uintptr_t>(w->bias) & 3u) ||
+      (reinterpret_cast<uintptr_t>(tok_mask) & 3u))
+    return BLOCKFFN_ERR_INVALID_ARG;
+  cudaError_t e =
+      launch_router(h, w, x, L, scores, tok_mask, false, nullptr, static_cast<cudaStream_t>(stream));
+  return e == cudaSuccess ? BLOCKFFN_OK : BLOCKFFN_ERR_CUDA;
+}
+
+blockffn_status blockffn_chunk_union(blockffn_handle h, const float* scores, int32_t L,
+                                     uint32_t* union_mask, int32_t* union_ids, int32_t* n_union,
+                                     blockffn_stats* stats, void* stream) {
+  blockffn_status s = check_call(h, L);
+  if (s != BLOCKFFN_OK) return s;
+  if (!scores || !union_ids || !n_union) return BLOCKFFN_ERR_INVALID_ARG;
+  if ((reinterpret_cast<uintptr_t>(scores) & 3u) || (reinterpret_cast<uintptr_t>(union_mask) & 3u) ||
+      (reinterpret_cast<uintptr_t>(union_ids) & 3u) || (reinterpret_cast<uintptr_t>(n_union) & 3u) ||
+      (reinterpret_cast<uintptr_t>(stats) & 7u))
+    return BLOCKFFN_ERR_INVALID_ARG;
+  cudaError_t e = launch_chunk_union(h, scores, L, union_mask, union_ids, n_union, stats,
+                                     static_cast<cudaStream_t>(stream));
+  return e == cudaSuccess ? BLOCKFFN_OK : BLOCKFFN_ERR_CUDA;
+}
+
+blockffn_status blockffn_expert_ffn(blockffn_handle h, const blockffn_weights* w, const void* x,
+                                    const float* scores, int32_t L, const int32_t* union_ids,
+                                    const int32_t* n_union, float* out, void* x_next,
+                                    int32_t call_flags, void* stream) {
+  blockffn_status s = check_call(h, L);
+  if (s != BLOCKFFN_OK) return s;
+  if (!w || !w->U || !w->D || !x || !scores || !union_ids || !n_union || !out)
+    return BLOCKFFN_ERR_INVALID_ARG;
+  if (misaligned(w->U) || misaligned(w->D) || misaligned(x) || misaligned(out) ||
+      misaligned(x_next) || (reinterpret_cast<uintptr_t>(scores) & 3u) ||
+      (reinterpret_cast<uintptr_t>(union_ids) & 3u) || (reinterpret_cast<uintptr_t>(n_union) & 3u))
+    return BLOCKFFN_ERR_INVALID_ARG;
+  if (x_next == x) return BLOCKFFN_ERR_INVALID_ARG;
+  if (call_flags & ~(BLOCKFFN_CALL_ACCUMULATE | BLOCKFFN_CALL_INDEPENDENT))
+    return BLOCKFFN_ERR_INVALID_ARG;
+  return expert_dispatch(h, w, x, scores, L, union_ids, n_union, out, x_next, call_flags,
+                         static_cast<cudaStream_t>(stream));
+}
+
+blockffn_status blockffn_layer_forward(blockffn_handle h, const blockffn_weights* w, const void* x,
+                                       int32_t L, float* out, void* x_next, blockffn_stats* stats,
+                                       int32_t call_flags, void* stream) {
+  blockffn_status s = check_call(h, L);
+  if (s != BLOCKFFN_OK) return s;
+  if (!w || !w->W_r || !w->gain || !w->U || !w->D || !x || !out) return BLOCKFFN_ERR_INVALID_ARG;
+  if (misaligned(w->W_r) || misaligned(w->U) || misaligned(w->D) || misaligned(x) ||
+      misaligned(out) || misaligned(x_next) || (reinterpret_cast<uintptr_t>(w->gain) & 3u) ||
+      (reinterpret_cast<uintptr_t>(w->bias) & 3u) || (reinterpret_cast<uintptr_t>(stats) & 7u))
+    return BLOCKFFN_ERR_INVALID_ARG;
+  if (x_next == x) return BLOCKFFN_ERR_INVALID_ARG;
+  if (call_flags & ~(BLOCKFFN_CALL_ACCUMULATE | BLOCKFFN_CALL_INDEPENDENT))
+    return BLOCKFFN_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  // The router writes the scores this very call consumes: never "independent".
+  const int flags = call_flags & ~BLOCKFFN_CALL_INDEPENDENT;
+  if (launch_router(h, w, x, L, h->scores, h->tok_mask, true, stats, st) != cudaSuccess)
+    return BLOCKFFN_ERR_CUDA;
+  return expert_dispatch(h, w, x, h->scores, L, h->union_ids, h->n_union, out, x_next, flags, st);
+}
+
+blockffn_status blockffn_layer_forward_scores(blockffn_handle h, const blockffn_weights* w,
+                                              const void* x, const float* scores, int32_t L,
+                                              float* out, void* x_next, blockffn_stats* stats,
+                                              int32_t call_flags, void* stream) {
+  blockffn_status s = check_call(h, L);
+  if (s != BLOCKFFN_OK) return s;
+  if (!w || !w->U || !w->D || !x || !scores || !out) return BLOCKFFN_ERR_INVALID_ARG;
+  if (misaligned(w->U) || misaligned(w->D) || misaligned(x) || misaligned(out) ||
+      misaligned(x_next) || misaligned(scores) || (reinterpret_cast<uintptr_t>(stats) & 7u))
+    return BLOCKFFN_ERR_INVALID_ARG;
+  if (x_next == x) return BLOCKFFN_ERR_INVALID_ARG;
+  if (call_flags & ~(BLOCKFFN_CALL_ACCUMULATE | BLOCKFFN_CALL_INDEPENDENT))
+    return BLOCKFFN_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (launch_chunk_union(h, scores, L, h->union_mask, h->union_ids, h->n_union, stats, st) !=
+      cudaSuccess)
+    return BLOCKFFN_ERR_CUDA;
+  // The union list is produced inside this call: the expert stage must wait for it.
+  const int flags = call_flags & ~BLOCKFFN_CALL_INDEPENDENT;
+  return expert_dispatch(h, w, x, scores, L, h->union_ids, h->n_union, out, x_next, flags, st);
+}
+
+blockffn_status blockffn_read_routing(blockffn_handle h, int32_t L, float* scores,
+                                      uint32_t* tok_mask, uint32_t* union_mask,
+                                      int32_t* union_ids, int32_t* n_union, void* stream) {
+  blockffn_status s = check_call(h, L);
+  if (s != BLOCKFFN_OK) return s;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const size_t E = h->cfg.E, W = h->words;
+  cudaError_t e = cudaSuccess;
+  auto copy = [&](void* dst, const void* src, size_t n) {
+    if (dst && e == cudaSuccess) e = cudaMemcpyAsync(dst, src, n, cudaMemcpyDeviceToDevice, st);
+  };
+  copy(scores, h->scores, sizeof(float) * L * E);
+  copy(tok_mask, h->tok_mask, sizeof(uint32_t) * L * W);
+  copy(union_mask, h->union_mask, sizeof(uint32_t) * W);
+  copy(union_ids, h->union_ids, sizeof(int32_t) * E);
+  copy(n_union, h->n_union, sizeof(int32_t));
+  return e == cudaSuccess ? BLOCKFFN_OK : BLOCKFFN_ERR_CUDA;
+}
+
+blockffn_status blockffn_last_status(blockffn_handle h, uint32_t* bits, int32_t clear,
+                                     void* stream) {
+  if (!h) return BLOCKFFN_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  uint32_t v = 0;
+  if (cudaMemcpyAsync(&v, h->status, sizeof v, cudaMemcpyDeviceToHost, st) != cudaSuccess ||
+      cudaStreamSynchronize(st) != cudaSuccess)
+    return BLOCKFFN_ERR_CUDA;
+  if (clear && v) {
+    if (cudaMemsetAsync(h->status, 0, sizeof v, st) != cudaSuccess) return BLOCKFFN_ERR_CUDA;
+  }
+  if (bits) *bits = v;
+  return v ? BLOCKFFN_ERR_DEVICE : BLOCKFFN_OK;
+}
+
+double blockffn_tls(const blockffn_stats* s, int32_t E) {
+  if (!s || E < 1 || s->n_tokens == 0) return 0.0;
+  return 1.0 - (double)s->n_active / ((double)s->n_tokens * (double)E);
+}
+
+double blockffn_cls(const blockffn_stats* s, int32_t E) {
+  if (!s || E < 1 || s->n_chunks == 0) return 0.0;
+  return 1.0 - (double)s->n_union / ((double)s->n_chunks * (double)E);
+}
+
+uint64_t blockffn_launch_count(blockffn_handle h) { return h ? h->launches : 0; }
+
+const char* blockffn_status_string(blockffn_status s) {
+  switch (s) {
+    case BLOCKFFN_OK: return "ok";
+    case BLOCKFFN_ERR_INVALID_ARG: return "invalid argument";
+    case BLOCKFFN_ERR_UNSUPPORTED: return "unsupported shape";
+    case BLOCKFFN_ERR_WORKSPACE: return "workspace allocation failed";
+    case BLOCKFFN_ERR_CUDA: return "CUDA error";
+    case BLOCKFFN_ERR_DEVICE: return "device status word set";
+  }
+  return "unknown";
+}
+
+}  // extern "C"

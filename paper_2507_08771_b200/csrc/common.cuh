@@ -1,0 +1,61 @@
+// Shared declarations of the BlockFFN CUDA library (sm_100a).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "blockffn.h"
+
+struct blockffn_ctx {
+  blockffn_config cfg;
+  int device;
+  int num_sms;
+  int words;            // ceil(E / 32)
+  uint64_t launches;    // host-side count of kernels launched through this handle
+  // ---- workspace (device) ----
+  void* ws_base;
+  float* a0;            // [L_max][E] router logits
+  float* scores;        // [L_max][E]
+  uint32_t* tok_mask;   // [L_max][words]
+  uint32_t* union_mask; // [words]
+  int32_t* union_ids;   // [E]
+  int32_t* n_union;     // [1]
+  float* h32;           // [E][L_max][d_e] fp32 intermediate (SIMT variant)
+  void* h16;            // bf16 intermediate (MMA variant), slot-major padded rows
+  unsigned int* ticket; // last-block-done counters [8]
+  uint32_t* status;     // sticky device status word
+};
+
+// ---- device helpers -------------------------------------------------------
+__device__ __forceinline__ float bf16_lo(uint32_t packed) { return __uint_as_float(packed << 16); }
+__device__ __forceinline__ float bf16_hi(uint32_t packed) {
+  return __uint_as_float(packed & 0xffff0000u);
+}
+// float -> bf16 bits, round to nearest even, NaN kept quiet
+__device__ __forceinline__ uint32_t f32_to_bf16_bits(float f) {
+  uint32_t w = __float_as_uint(f);
+  if ((w & 0x7fffffffu) > 0x7f800000u) return (w >> 16) | 0x40u;
+  return (w + 0x7fffu + ((w >> 16) & 1u)) >> 16;
+}
+__device__ __forceinline__ float swish(float z) { return z / (1.0f + __expf(-z)); }
+
+// ---- launchers (each returns the cudaError_t of its launch) ----------------
+cudaError_t launch_router(blockffn_ctx* c, const blockffn_weights* w, const void* x, int L,
+                          float* scores, uint32_t* tok_mask, bool fuse_union,
+                          blockffn_stats* stats, cudaStream_t st);
+cudaError_t launch_chunk_union(blockffn_ctx* c, const float* scores, int L, uint32_t* union_mask,
+                               int32_t* union_ids, int32_t* n_union, blockffn_stats* stats,
+                               cudaStream_t st);
+cudaError_t launch_expert_simt(blockffn_ctx* c, const blockffn_weights* w, const void* x,
+                               const float* scores, int L, const int32_t* union_ids,
+                               const int32_t* n_union, float* out, void* x_next, int call_flags,
+                               cudaStream_t st);
+
+// Tensor-core / bulk-copy variant of the expert stage.
+bool expert_mma_supported(const blockffn_ctx* c, int L);
+size_t expert_mma_h_bytes(const blockffn_config* cfg);
+cudaError_t expert_mma_setup(blockffn_ctx* c);
+cudaError_t launch_expert_mma(blockffn_ctx* c, const blockffn_weights* w, const void* x,
+                              const float* scores, int L, const int32_t* union_ids,
+                              const int32_t* n_union, float* out, void* x_next, int call_flags,
+                              cudaStream_t st);

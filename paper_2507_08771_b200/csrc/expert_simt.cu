@@ -1,0 +1,185 @@
+// Expert stage (Eq. 1, Eq. 2 restricted to Union(x), Sec. 3.3), CUDA-core variant.
+//
+// Two kernels. expert_up: each warp owns 4 neuron rows of one union expert, streams
+// their bf16 weights with 128-bit loads, multiplies them with every token of the
+// chunk (fp32 FMA, tokens tiled by LT), reduces over the warp, applies Swish and the
+// token's router score and stores the fp32 intermediate h[slot][t][j].
+// expert_down: each warp owns one output column, runs over all union experts'
+// rows of D for that column and over h, reduces, and writes out[t][c] (optionally
+// accumulating into an fp32 residual and emitting its bf16 rounding).
+// No atomics: every output element has exactly one writer.
+#include "common.cuh"
+
+namespace {
+
+constexpr int kThreads = 256;
+constexpr int kWarps = kThreads / 32;
+constexpr int kRows = 4;  // neuron rows per warp task
+
+__device__ __forceinline__ int load_union(const int32_t* union_ids, const int32_t* n_union, int E,
+                                          int* ids_sm, uint32_t* status) {
+  int nu = *n_union;
+  if (nu < 0 || nu > E) {
+    if (threadIdx.x == 0) atomicOr(status, BLOCKFFN_DEV_BAD_UNION_COUNT);
+    nu = nu < 0 ? 0 : E;
+  }
+  for (int q = threadIdx.x; q < nu; q += blockDim.x) {
+    int id = union_ids[q];
+    if (id < 0 || id >= E) {
+      atomicOr(status, BLOCKFFN_DEV_BAD_UNION_ID);
+      id = -1;
+    }
+    ids_sm[q] = id;
+  }
+  __syncthreads();
+  return nu;
+}
+
+template <int LT>
+__global__ void __launch_bounds__(kThreads)
+expert_up_simt(const uint16_t* __restrict__ x, const uint16_t* __restrict__ U,
+               const float* __restrict__ scores, const int32_t* __restrict__ union_ids,
+               const int32_t* __restrict__ n_union, float* __restrict__ h, int L, int d, int E,
+               int d_e, int L_max, uint32_t* status) {
+  extern __shared__ int ids_sm[];
+  const int nu = load_union(union_ids, n_union, E, ids_sm, status);
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int groups = d_e / kRows;
+  const int tasks = nu * groups;
+  const int chunks = d >> 3;
+  for (int task = blockIdx.x * kWarps + warp; task < tasks; task += gridDim.x * kWarps) {
+    const int q = task / groups, j0 = (task % groups) * kRows;
+    const int id = ids_sm[q];
+    if (id < 0) continue;
+    const uint4* wrow[kRows];
+#pragma unroll
+    for (int r = 0; r < kRows; ++r)
+      wrow[r] = reinterpret_cast<const uint4*>(U + ((size_t)id * d_e + j0 + r) * d);
+    for (int t0 = 0; t0 < L; t0 += LT) {
+      float acc[kRows][LT];
+#pragma unroll
+      for (int r = 0; r < kRows; ++r)
+#pragma unroll
+        for (int t = 0; t < LT; ++t) acc[r][t] = 0.0f;
+      for (int c = lane; c < chunks; c += 32) {
+        uint4 wv[kRows];
+#pragma unroll
+        for (int r = 0; r < kRows; ++r) wv[r] = __ldg(wrow[r] + c);
+#pragma unroll
+        for (int t = 0; t < LT; ++t) {
+          if (t0 + t < L) {
+            const uint4 xv = __ldg(reinterpret_cast<const uint4*>(x + (size_t)(t0 + t) * d) + c);
+            const uint32_t xp[4] = {xv.x, xv.y, xv.z, xv.w};
+#pragma unroll
+            for (int r = 0; r < kRows; ++r) {
+              const uint32_t wp[4] = {wv[r].x, wv[r].y, wv[r].z, wv[r].w};
+#pragma unroll
+              for (int p = 0; p < 4; ++p) {
+                acc[r][t] = fmaf(bf16_lo(wp[p]), bf16_lo(xp[p]), acc[r][t]);
+                acc[r][t] = fmaf(bf16_hi(wp[p]), bf16_hi(xp[p]), acc[r][t]);
+              }
+            }
+          }
+        }
+      }
+#pragma unroll
+      for (int r = 0; r < kRows; ++r)
+#pragma unroll
+        for (int t = 0; t < LT; ++t) {
+          float v = acc[r][t];
+#pragma unroll
+          for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+          if (lane == r * LT + t && t0 + t < L) {
+            const float s = scores[(size_t)(t0 + t) * E + id];
+            h[((size_t)q * L_max + t0 + t) * d_e + j0 + r] = s * swish(v);
+          }
+        }
+    }
+  }
+}
+
+template <int LT>
+__global__ void __launch_bounds__(kThreads)
+expert_down_simt(const uint16_t* __restrict__ D, const float* __restrict__ h,
+                 const int32_t* __restrict__ union_ids, const int32_t* __restrict__ n_union,
+                 float* __restrict__ out, uint16_t* __restrict__ x_next, int L, int d, int E,
+                 int d_e, int L_max, int accumulate, uint32_t* status) {
+  extern __shared__ int ids_sm[];
+  const int nu = load_union(union_ids, n_union, E, ids_sm, status);
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int K = nu * d_e;
+  for (int c = blockIdx.x * kWarps + warp; c < d; c += gridDim.x * kWarps) {
+    for (int t0 = 0; t0 < L; t0 += LT) {
+      float acc[LT];
+#pragma unroll
+      for (int t = 0; t < LT; ++t) acc[t] = 0.0f;
+      for (int kk = lane * 4; kk < K; kk += 128) {
+        const int q = kk / d_e, j = kk - q * d_e;
+        const int id = ids_sm[q];
+        if (id < 0) continue;
+        const uint2 wv = __ldg(reinterpret_cast<const uint2*>(D + ((size_t)id * d + c) * d_e + j));
+        const float w0 = bf16_lo(wv.x), w1 = bf16_hi(wv.x), w2 = bf16_lo(wv.y), w3 = bf16_hi(wv.y);
+#pragma unroll
+        for (int t = 0; t < LT; ++t) {
+          if (t0 + t < L) {
+            const float4 hv =
+                *reinterpret_cast<const float4*>(h + ((size_t)q * L_max + t0 + t) * d_e + j);
+            acc[t] = fmaf(hv.x, w0, acc[t]);
+            acc[t] = fmaf(hv.y, w1, acc[t]);
+            acc[t] = fmaf(hv.z, w2, acc[t]);
+            acc[t] = fmaf(hv.w, w3, acc[t]);
+          }
+        }
+      }
+#pragma unroll
+      for (int t = 0; t < LT; ++t) {
+        float v = acc[t];
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+        if (lane == t && t0 + t < L) {
+          const size_t p = (size_t)(t0 + t) * d + c;
+          if (accumulate) v += out[p];
+          out[p] = v;
+          if (x_next) x_next[p] = (uint16_t)f32_to_bf16_bits(v);
+        }
+      }
+    }
+  }
+}
+
+template <int LT>
+cudaError_t launch_lt(blockffn_ctx* c, const blockffn_weights* w, const void* x,
+                      const float* scores, int L, const int32_t* union_ids,
+                      const int32_t* n_union, float* out, void* x_next, int call_flags,
+                      cudaStream_t st) {
+  const int E = c->cfg.E, d = c->cfg.d, d_e = c->cfg.d_e;
+  const size_t sm = sizeof(int) * (size_t)E;
+  const int up_tasks = E * (d_e / kRows);
+  int grid_up = (up_tasks + kWarps - 1) / kWarps;
+  if (grid_up > c->num_sms * 4) grid_up = c->num_sms * 4;
+  int grid_dn = (d + kWarps - 1) / kWarps;
+  if (grid_dn > c->num_sms * 4) grid_dn = c->num_sms * 4;
+  expert_up_simt<LT><<<grid_up, kThreads, sm, st>>>(
+      static_cast<const uint16_t*>(x), static_cast<const uint16_t*>(w->U), scores, union_ids,
+      n_union, c->h32, L, d, E, d_e, c->cfg.L_max, c->status);
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return e;
+  expert_down_simt<LT><<<grid_dn, kThreads, sm, st>>>(
+      static_cast<const uint16_t*>(w->D), c->h32, union_ids, n_union, out,
+      static_cast<uint16_t*>(x_next), L, d, E, d_e, c->cfg.L_max,
+      (call_flags & BLOCKFFN_CALL_ACCUMULATE) ? 1 : 0, c->status);
+  c->launches += 2;
+  return cudaGetLastError();
+}
+
+}  // namespace
+
+cudaError_t launch_expert_simt(blockffn_ctx* c, const blockffn_weights* w, const void* x,
+                               const float* scores, int L, const int32_t* union_ids,
+                               const int32_t* n_union, float* out, void* x_next, int call_flags,
+                               cudaStream_t st) {
+  if (L <= 1) return launch_lt<1>(c, w, x, scores, L, union_ids, n_union, out, x_next, call_flags, st);
+  if (L <= 2) return launch_lt<2>(c, w, x, scores, L, union_ids, n_union, out, x_next, call_flags, st);
+  if (L <= 4) return launch_lt<4>(c, w, x, scores, L, union_ids, n_union, out, x_next, call_flags, st);
+  return launch_lt<8>(c, w, x, scores, L, union_ids, n_union, out, x_next, call_flags, st);
+}

@@ -1,0 +1,190 @@
+// Router (Eq. 3) and chunk union (Sec. 3.3) kernels.
+//
+// router_kernel: one block per expert computes that expert's logit for every
+// token of the chunk (x . W_r[i] + bias[i]) with 128-bit loads and fp32 FMAs; the
+// block that finishes last (a ticket counter, no waiting) applies ReLU and RMSNorm
+// with the per-expert gain, writes the scores and the per-token nonzero masks
+// (warp ballot), and, for the fused layer call, derives the chunk union right away.
+//
+// union_kernel: one block ORs the per-token nonzero patterns of a score matrix,
+// compacts the union's expert ids in ascending order with a warp prefix count, and
+// advances the TLS / CLS counters (Sec. 2.1).
+#include "common.cuh"
+
+namespace {
+
+constexpr int kThreads = 256;
+constexpr int kWarps = kThreads / 32;
+constexpr int kMaxWords = 32;  // E <= 1024
+
+// All 256 threads of the block take part. sm: >= 3 * kMaxWords ints.
+__device__ void chunk_union_block(const float* scores, int L, int E, uint32_t* union_mask,
+                                  int32_t* union_ids, int32_t* n_union, blockffn_stats* stats,
+                                  int* sm) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int words = (E + 31) >> 5;
+  int* cnt = sm;                                   // popcount of each union word
+  int* act = sm + kMaxWords;                       // active (token, expert) pairs per word
+  uint32_t* um = reinterpret_cast<uint32_t*>(sm + 2 * kMaxWords);
+  for (int w = warp; w < words; w += kWarps) {
+    const int e = 32 * w + lane;
+    uint32_t un = 0;
+    int nact = 0;
+    for (int t = 0; t < L; ++t) {
+      float v = (e < E) ? scores[(size_t)t * E + e] : 0.0f;
+      uint32_t m = __ballot_sync(0xffffffffu, v != 0.0f);
+      un |= m;
+      nact += __popc(m);
+    }
+    if (lane == 0) {
+      cnt[w] = __popc(un);
+      act[w] = nact;
+      um[w] = un;
+      if (union_mask) union_mask[w] = un;
+    }
+  }
+  __syncthreads();
+  int total = 0, total_act = 0;
+  for (int w = 0; w < words; ++w) {
+    total += cnt[w];
+    total_act += act[w];
+  }
+  for (int w = warp; w < words; w += kWarps) {
+    int off = 0;
+    for (int v = 0; v < w; ++v) off += cnt[v];
+    const uint32_t un = um[w];
+    if ((un >> lane) & 1u) union_ids[off + __popc(un & ((1u << lane) - 1u))] = 32 * w + lane;
+  }
+  for (int idx = total + threadIdx.x; idx < E; idx += kThreads) union_ids[idx] = -1;
+  if (threadIdx.x == 0) {
+    *n_union = total;
+    if (stats) {
+      atomicAdd(reinterpret_cast<unsigned long long*>(&stats->n_tokens), (unsigned long long)L);
+      atomicAdd(reinterpret_cast<unsigned long long*>(&stats->n_active),
+                (unsigned long long)total_act);
+      atomicAdd(reinterpret_cast<unsigned long long*>(&stats->n_chunks), 1ull);
+      atomicAdd(reinterpret_cast<unsigned long long*>(&stats->n_union), (unsigned long long)total);
+    }
+  }
+}
+
+__global__ void __launch_bounds__(kThreads)
+union_kernel(const float* __restrict__ scores, int L, int E, uint32_t* union_mask,
+             int32_t* union_ids, int32_t* n_union, blockffn_stats* stats) {
+  __shared__ int sm[3 * kMaxWords];
+  chunk_union_block(scores, L, E, union_mask, union_ids, n_union, stats, sm);
+}
+
+__global__ void __launch_bounds__(kThreads)
+router_kernel(const uint16_t* __restrict__ x, const uint16_t* __restrict__ W_r,
+              const float* __restrict__ gain, const float* __restrict__ bias, float* a0,
+              float* scores, uint32_t* tok_mask, int L, int d, int E, float eps,
+              unsigned int* ticket, int fuse_union, uint32_t* union_mask, int32_t* union_ids,
+              int32_t* n_union, blockffn_stats* stats) {
+  __shared__ float red[kWarps][8];
+  __shared__ int sm[3 * kMaxWords];
+  __shared__ int is_last;
+  const int i = blockIdx.x;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int chunks = d >> 3;
+  const uint4* wrow = reinterpret_cast<const uint4*>(W_r + (size_t)i * d);
+  const float b = bias ? bias[i] : 0.0f;
+
+  for (int t0 = 0; t0 < L; t0 += 8) {
+    float acc[8];
+#pragma unroll
+    for (int t = 0; t < 8; ++t) acc[t] = 0.0f;
+    for (int c = threadIdx.x; c < chunks; c += kThreads) {
+      const uint4 wv = __ldg(wrow + c);
+      const uint32_t wp[4] = {wv.x, wv.y, wv.z, wv.w};
+#pragma unroll
+      for (int t = 0; t < 8; ++t) {
+        if (t0 + t < L) {
+          const uint4 xv = __ldg(reinterpret_cast<const uint4*>(x + (size_t)(t0 + t) * d) + c);
+          const uint32_t xp[4] = {xv.x, xv.y, xv.z, xv.w};
+#pragma unroll
+          for (int p = 0; p < 4; ++p) {
+            acc[t] = fmaf(bf16_lo(wp[p]), bf16_lo(xp[p]), acc[t]);
+            acc[t] = fmaf(bf16_hi(wp[p]), bf16_hi(xp[p]), acc[t]);
+          }
+        }
+      }
+    }
+#pragma unroll
+    for (int t = 0; t < 8; ++t) {
+      float v = acc[t];
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+      if (lane == 0) red[warp][t] = v;
+    }
+    __syncthreads();
+    if (threadIdx.x < 8 && t0 + threadIdx.x < L) {
+      float v = b;
+#pragma unroll
+      for (int w = 0; w < kWarps; ++w) v += red[w][threadIdx.x];
+      a0[(size_t)(t0 + threadIdx.x) * E + i] = v;
+    }
+    __syncthreads();
+  }
+
+  // last block done: normalise. The ticket is reset for the next call.
+  __threadfence();
+  if (threadIdx.x == 0) {
+    unsigned int tk = atomicAdd(ticket, 1u);
+    is_last = (tk == gridDim.x - 1);
+    if (is_last) *ticket = 0u;
+  }
+  __syncthreads();
+  if (!is_last) return;
+  __threadfence();
+
+  const int words = (E + 31) >> 5;
+  for (int t = warp; t < L; t += kWarps) {
+    float ss = 0.0f;
+    for (int e = lane; e < E; e += 32) {
+      float v = __ldcg(a0 + (size_t)t * E + e);
+      v = v > 0.0f ? v : 0.0f;
+      ss = fmaf(v, v, ss);
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
+    const float r = 1.0f / sqrtf(ss / (float)E + eps);
+    for (int w = 0; w < words; ++w) {
+      const int e = 32 * w + lane;
+      float s = 0.0f;
+      if (e < E) {
+        float v = __ldcg(a0 + (size_t)t * E + e);
+        v = v > 0.0f ? v : 0.0f;
+        s = gain[e] * v * r;
+        scores[(size_t)t * E + e] = s;
+      }
+      const uint32_t m = __ballot_sync(0xffffffffu, s != 0.0f);
+      if (tok_mask && lane == 0) tok_mask[(size_t)t * words + w] = m;
+    }
+  }
+  if (fuse_union) {
+    __syncthreads();
+    chunk_union_block(scores, L, E, union_mask, union_ids, n_union, stats, sm);
+  }
+}
+
+}  // namespace
+
+cudaError_t launch_router(blockffn_ctx* c, const blockffn_weights* w, const void* x, int L,
+                          float* scores, uint32_t* tok_mask, bool fuse_union,
+                          blockffn_stats* stats, cudaStream_t st) {
+  router_kernel<<<c->cfg.E, kThreads, 0, st>>>(
+      static_cast<const uint16_t*>(x), static_cast<const uint16_t*>(w->W_r), w->gain, w->bias,
+      c->a0, scores, tok_mask, L, c->cfg.d, c->cfg.E, c->cfg.rms_eps, c->ticket,
+      fuse_union ? 1 : 0, c->union_mask, c->union_ids, c->n_union, stats);
+  c->launches += 1;
+  return cudaGetLastError();
+}
+
+cudaError_t launch_chunk_union(blockffn_ctx* c, const float* scores, int L, uint32_t* union_mask,
+                               int32_t* union_ids, int32_t* n_union, blockffn_stats* stats,
+                               cudaStream_t st) {
+  union_kernel<<<1, kThreads, 0, st>>>(scores, L, c->cfg.E, union_mask, union_ids, n_union, stats);
+  c->launches += 1;
+  return cudaGetLastError();
+}
