@@ -119,8 +119,8 @@ def make_weights(W_r=None, gain=None, bias=None, U=None, D=None) -> Weights:
 
 
 # ---- entry points, same names as the C ABI ------------------------------------
-def blockffn_create(d, E, d_e, L_max, rms_eps=1e-6, variant=VARIANT_AUTO):
-    cfg = Config(d, E, d_e, L_max, rms_eps, variant, 0)
+def blockffn_create(d, E, d_e, L_max, rms_eps=1e-6, variant=VARIANT_AUTO, flags=0):
+    cfg = Config(d, E, d_e, L_max, rms_eps, variant, flags)
     h = ctypes.c_void_p()
     _check(load().blockffn_create(ctypes.byref(cfg), ctypes.byref(h)), "blockffn_create")
     return h
@@ -220,11 +220,12 @@ class LayerOutput:
 class Layer:
     """Owns one library handle and output buffers; forwards to the C entry points."""
 
-    def __init__(self, d, E, d_e, L_max=32, rms_eps=1e-6, variant=VARIANT_AUTO, device="cuda"):
+    def __init__(self, d, E, d_e, L_max=32, rms_eps=1e-6, variant=VARIANT_AUTO, device="cuda",
+                 flags=0):
         self.d, self.E, self.d_e, self.L_max = d, E, d_e, L_max
         self.words = (E + 31) // 32
         self.device = torch.device(device)
-        self.h = blockffn_create(d, E, d_e, L_max, rms_eps, variant)
+        self.h = blockffn_create(d, E, d_e, L_max, rms_eps, variant, flags)
         self.stats = torch.zeros(4, dtype=torch.int64, device=self.device)
 
     def close(self):

@@ -14,13 +14,19 @@ blockffn_status check_call(blockffn_ctx* c, int L) {
   return BLOCKFFN_OK;
 }
 
+bool use_mma(const blockffn_ctx* c, int L) {
+  return c->cfg.variant != BLOCKFFN_VARIANT_SIMT && expert_mma_supported(c, L);
+}
+
+// Expert stage from a given union list.
 blockffn_status expert_dispatch(blockffn_ctx* c, const blockffn_weights* w, const void* x,
                                 const float* scores, int L, const int32_t* union_ids,
                                 const int32_t* n_union, float* out, void* x_next, int call_flags,
                                 cudaStream_t st) {
   cudaError_t e;
-  if (expert_mma_supported(c, L) && c->cfg.variant != BLOCKFFN_VARIANT_SIMT)
-    e = launch_expert_mma(c, w, x, scores, L, union_ids, n_union, out, x_next, call_flags, st);
+  if (use_mma(c, L))
+    e = launch_expert_mma(c, w, x, scores, L, union_ids, n_union, out, x_next, call_flags, nullptr,
+                          st);
   else
     e = launch_expert_simt(c, w, x, scores, L, union_ids, n_union, out, x_next, call_flags, st);
   return e == cudaSuccess ? BLOCKFFN_OK : BLOCKFFN_ERR_CUDA;
@@ -40,6 +46,7 @@ blockffn_status blockffn_create(const blockffn_config* cfg, blockffn_handle* out
   if (!(cfg->rms_eps >= 0.0f)) return BLOCKFFN_ERR_INVALID_ARG;
   if (cfg->variant < BLOCKFFN_VARIANT_AUTO || cfg->variant > BLOCKFFN_VARIANT_MMA)
     return BLOCKFFN_ERR_INVALID_ARG;
+  if (cfg->flags & ~0xffff) return BLOCKFFN_ERR_INVALID_ARG;
   blockffn_ctx* c = new (std::nothrow) blockffn_ctx();
   if (!c) return BLOCKFFN_ERR_WORKSPACE;
   c->cfg = *cfg;
@@ -190,6 +197,15 @@ blockffn_status blockffn_layer_forward_scores(blockffn_handle h, const blockffn_
   if (call_flags & ~(BLOCKFFN_CALL_ACCUMULATE | BLOCKFFN_CALL_INDEPENDENT))
     return BLOCKFFN_ERR_INVALID_ARG;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (use_mma(h, L)) {
+    // The expert kernels derive Union(x) from the scores themselves (every CTA needs the
+    // list before it can fetch a weight byte) and CTA 0 publishes it: no separate launch.
+    const RoutingOut pub{h->union_mask, h->union_ids, h->n_union, stats};
+    return launch_expert_mma(h, w, x, scores, L, nullptr, nullptr, out, x_next, call_flags, &pub,
+                             st) == cudaSuccess
+               ? BLOCKFFN_OK
+               : BLOCKFFN_ERR_CUDA;
+  }
   if (launch_chunk_union(h, scores, L, h->union_mask, h->union_ids, h->n_union, stats, st) !=
       cudaSuccess)
     return BLOCKFFN_ERR_CUDA;

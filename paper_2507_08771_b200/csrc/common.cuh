@@ -51,11 +51,20 @@ cudaError_t launch_expert_simt(blockffn_ctx* c, const blockffn_weights* w, const
                                const int32_t* n_union, float* out, void* x_next, int call_flags,
                                cudaStream_t st);
 
-// Tensor-core / bulk-copy variant of the expert stage.
+// Where a kernel that derives Union(x) itself publishes it (each pointer may be NULL).
+struct RoutingOut {
+  uint32_t* union_mask;
+  int32_t* union_ids;
+  int32_t* n_union;
+  blockffn_stats* stats;
+};
+
+// Tensor-core / bulk-copy variant of the expert stage. union_ids == NULL: the kernels derive
+// the union from the nonzero pattern of scores and publish it through pub.
 bool expert_mma_supported(const blockffn_ctx* c, int L);
 size_t expert_mma_h_bytes(const blockffn_config* cfg);
 cudaError_t expert_mma_setup(blockffn_ctx* c);
 cudaError_t launch_expert_mma(blockffn_ctx* c, const blockffn_weights* w, const void* x,
                               const float* scores, int L, const int32_t* union_ids,
                               const int32_t* n_union, float* out, void* x_next, int call_flags,
-                              cudaStream_t st);
+                              const RoutingOut* pub, cudaStream_t st);
