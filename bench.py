@@ -44,6 +44,8 @@ def parse():
     p.add_argument("--L", type=int, default=None, help="chunk length (default: the config's)")
     p.add_argument("--chunks", type=int, default=256, help="chunks per step")
     p.add_argument("--variant", type=int, default=0, help="0 auto, 1 CUDA-core, 2 tensor-core")
+    p.add_argument("--flags", type=lambda v: int(v, 0), default=0,
+                   help="blockffn_config.flags (ring depths, BLOCKFFN_CFG_* bits)")
     p.add_argument("--no-cpu-baseline", action="store_true")
     p.add_argument("--sweep", action="store_true", help="also report every L of the sweep (config 2)")
     return p.parse_args()
@@ -123,7 +125,7 @@ class ClockSampler:
 class Workload:
     """Device-resident synthetic inputs for one benchmark configuration."""
 
-    def __init__(self, cfg_index, L, chunks, variant, device):
+    def __init__(self, cfg_index, L, chunks, variant, device, flags=0):
         import torch
         from paper_2507_08771_b200 import binding as B
         self.torch, self.B = torch, B
@@ -133,7 +135,8 @@ class Workload:
         seed = I.config_seed(cfg_index)
         self.u = sh.u
         self.active_bytes = sh.active_bytes()
-        self.layer = B.Layer(sh.d, sh.E, sh.d_e, L_max=max(self.L, 8), variant=variant, device=device)
+        self.layer = B.Layer(sh.d, sh.E, sh.d_e, L_max=max(self.L, 8), variant=variant, device=device,
+                             flags=flags)
         if cfg_index == 4:
             self.n_copies = I.STACK_LAYERS          # 24 distinct layers, 1.6 GB >> L2
             host = [I.make_experts(sh.d, sh.E, sh.d_e, seed, layer=l) for l in range(self.n_copies)]
@@ -329,7 +332,7 @@ def run_ours(args):
             dist.barrier()
         torch.cuda.synchronize()
 
-    wl = Workload(args.config, args.L, args.chunks, args.variant, device)
+    wl = Workload(args.config, args.L, args.chunks, args.variant, device, args.flags)
     sh = wl.sh
     stream = torch.cuda.Stream(device)
     lay = wl.layer
@@ -405,7 +408,7 @@ def run_ours(args):
             "l2": f"inputs larger than L2: {wl.n_copies} weight copies rotated, "
                   f"{wl.n_copies * wl.active_bytes / 1e6:.0f} MB streamed between reuses",
             "replicas": "independent replicas per GPU, no collective" if world > 1 else "single GPU",
-            "variant": args.variant,
+            "variant": args.variant, "flags": args.flags,
         },
         "clocks": clocks,
         "e2e": {"value": e2e, "unit": "GB/s", "h2d_bytes_per_step": wl.h2d_bytes,

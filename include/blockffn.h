@@ -71,8 +71,15 @@ typedef struct {
   int32_t L_max;   /* largest chunk length a call may pass (<= 32)             */
   float rms_eps;   /* RMSNorm epsilon, added to the mean square (Eq. 3); 1e-6  */
   int32_t variant; /* BLOCKFFN_VARIANT_*                                       */
-  int32_t flags;   /* reserved, 0                                              */
+  int32_t flags;   /* tuning, 0 = defaults: bits 0-7 ring depth of the up-projection
+                      kernel, bits 8-15 of the down-projection kernel (stages of shared
+                      memory, 0 = chosen from the shape), BLOCKFFN_CFG_* bits        */
 } blockffn_config;
+
+/* The tensor-core kernels are normally launched so that a kernel may start fetching its
+ * weights while the kernel enqueued before it on the stream is still finishing
+ * (programmatic dependent launch); this bit launches them fully serialised instead. */
+#define BLOCKFFN_CFG_NO_CHAINING 0x10000
 
 /* Layer parameters: device pointers, caller-owned, read-only to the library. */
 typedef struct {

@@ -1,81 +1,86 @@
-// Expert stage (Eq. 1, Eq. 2 restricted to Union(x), Sec. 3.3): bulk-copy staged,
+// Expert stage (Eq. 1, Eq. 2 restricted to Union(x), Sec. 3.3): asynchronously staged,
 // tensor-core variant.
 //
 // Two kernels per call, one CTA per SM each, chained by programmatic dependent
 // launch so that the weight fetch of a kernel overlaps the tail of the one before:
 //
 //   expert_up_mma    CTA b owns an equal share of the union's neuron rows (u * d_e
-//                    rows of U, d contiguous bf16 each). One producer lane gathers the
-//                    rows into a shared-memory ring with 1-D bulk async copies that
-//                    complete on mbarriers; eight consumer warps split K, multiply the
-//                    16-row tile with all L tokens on mma.sync m16n8k16 (weights are
-//                    the M operand, tokens the N operand), reduce across warps, apply
-//                    Swish and the token's router score and store the bf16 intermediate
+//                    rows of U, d contiguous bf16 each). All 256 threads gather the
+//                    share into shared memory with 16-byte asynchronous copies
+//                    (cp.async, L2 only), a few rows per stage; the eight warps split K,
+//                    multiply a stage of up to 16
+//                    rows with all L tokens on mma.sync m16n8k16 (weights are the M
+//                    operand, tokens the N operand), reduce across warps, apply Swish
+//                    and the token's router score and store the bf16 intermediate
 //                    h[q][t][j] to the handle's workspace.
 //   expert_down_mma  CTA b owns a block of <= 16 output columns. For every union expert
-//                    it bulk-copies the contiguous [columns x d_e] slab of D and the
-//                    expert's h chunk, accumulates out[t][c] over all experts on the
-//                    tensor cores and writes each output element exactly once
-//                    (no atomics; results are run-to-run identical).
+//                    it stages the contiguous [columns x d_e] slab of D and the expert's
+//                    h rows, accumulates out[t][c] over all experts on the tensor cores
+//                    and writes each output element exactly once (no atomics; results
+//                    are run-to-run identical).
 //
 // The D slabs (and, for calls flagged independent, the U rows) are requested before
 // griddepcontrol.wait, i.e. while the previous kernel is still running; everything a
 // previous kernel may have produced (x, h, out) is touched only after it.
 //
-// The k index of each 32-wide block is permuted identically for both mma operands
-// (lane tg owns 8 consecutive k), so every fragment is one 128-bit shared-memory load.
-// Every wait on an mbarrier is bounded: on expiry the kernel sets
-// BLOCKFFN_DEV_WAIT_EXPIRED, keeps its control flow (so all barriers are met), drains
-// its own outstanding copies with a bound and returns.
+// Why cp.async and not bulk (TMA) copies: the pieces are small (a D slab is
+// columns * 2 d_e bytes, 3.5 KB at d = 2048) and a bulk copy costs its issuing thread a
+// few hundred nanoseconds whatever its size, which measured 0.56 / 2.2 / 7.0 TB/s device
+// wide for 1 / 4 / 16 KB pieces; 16-byte cp.async from 256 threads with 64 KB in flight
+// per SM measured 7.2 TB/s.
+//
+// Fragments: the k index of each 64-wide block is permuted identically for both mma
+// operands (lane tg owns 8 consecutive k of each 32-wide half), so a fragment is a
+// 128-bit shared-memory load; rows are staged unpadded (row strides are multiples of
+// 128 bytes) and lanes of odd rows read the two halves in the opposite order, which
+// keeps every quarter-warp on 32 distinct banks.
+// Completion is tracked with cp.async commit groups and CTA barriers only: no thread ever
+// spins on memory, so nothing here can wait forever.
 #include "common.cuh"
 
 namespace {
 
-constexpr int kConsumerWarps = 8;
-constexpr int kConsumerThreads = kConsumerWarps * 32;
-constexpr int kThreads = kConsumerThreads + 32;  // + one producer warp
-constexpr int kKC = 512;                         // k columns per up-projection stage
-constexpr int kPad = 64;                         // padding bytes per staged row (bank skew)
-constexpr int kMaxStages = 32;
-constexpr long long kWaitCycles = 2000000000ll;  // about one second
+constexpr int kWarps = 8;
+constexpr int kThreads = kWarps * 32;
+constexpr int kMaxStages = 32;                   // slots of the down kernel's ring
+constexpr int kUpStages = 3;                     // slots of the up kernel's ring
 constexpr int kSmemMax = 232448;                 // 227 KB per CTA
 constexpr int kSmemHalf = 113 * 1024;            // lets an up and a down CTA share one SM
 
 // ---- shared-memory layout ----------------------------------------------------
 __host__ __device__ inline int align128(int v) { return (v + 127) & ~127; }
 
-struct SmemLayout {
-  int off_ctl, off_ids, off_red, off_x, off_ring, slot_bytes, slot_h_off, total;
-};
-// bars: full[kMaxStages], empty[kMaxStages], xbar
-constexpr int kOffBars = 0;
-constexpr int kBarBytes = 1024;
-constexpr int kCtlBytes = 512;  // ints: [0] nu, [1] abort, [2] n_active, [3] bad bits, [5] abort of the
-                                // final drain; [8..40) union mask words; [40..72), [72..104) scratch
+constexpr int kCtlBytes = 512;  // ints: [0] nu, [2] n_active, [3] bad bits; [8..40) union mask
+                                // words; [40..72), [72..104) scratch
+constexpr int kOffCtl = 0;
+constexpr int kOffIds = kOffCtl + kCtlBytes;
 
-__host__ __device__ inline SmemLayout up_layout(int d, int E, int NT, int ns) {
-  SmemLayout s;
-  s.off_ctl = kBarBytes;
-  s.off_ids = s.off_ctl + kCtlBytes;
-  s.off_red = s.off_ids + align128(E * 4);
-  s.off_x = s.off_red + kConsumerWarps * 16 * 8 * NT * 4;
-  s.off_ring = s.off_x + align128(8 * NT * (2 * d + kPad));
-  s.slot_bytes = 16 * (2 * kKC + kPad);
-  s.slot_h_off = 0;
-  s.total = s.off_ring + ns * s.slot_bytes;
+struct UpLayout {
+  int off_red, off_x, off_ring, total;
+};
+// red: per warp a 32 x (8 NT) tile; x: L rows of 2d bytes; ring: ring_rows rows of 2d bytes
+__host__ __device__ inline UpLayout up_layout(int d, int E, int NT, int L, int ring_rows) {
+  UpLayout s;
+  s.off_red = kOffIds + align128(E * 4);
+  s.off_x = s.off_red + kWarps * 32 * 8 * NT * 4;
+  s.off_ring = s.off_x + align128(L * 2 * d);
+  s.total = s.off_ring + ring_rows * 2 * d;
   return s;
 }
 
-__host__ __device__ inline SmemLayout down_layout(int d_e, int E, int NT, int ns) {
-  SmemLayout s;
-  s.off_ctl = kBarBytes;
-  s.off_ids = s.off_ctl + kCtlBytes;
-  s.off_red = s.off_ids + align128(E * 4);
-  s.off_x = s.off_red + kConsumerWarps * 16 * 8 * NT * 4;
-  s.off_ring = s.off_x;
-  s.slot_h_off = align128(16 * 2 * d_e);
-  s.slot_bytes = s.slot_h_off + align128(8 * NT * (2 * d_e + kPad));
-  s.total = s.off_ring + ns * s.slot_bytes;
+struct DownLayout {
+  int off_red, off_h, off_d, slot_h, slot_d, total;
+};
+// h ring: ns slots of L rows of 2 d_e bytes; D ring: ns slots of max_cols rows of 2 d_e bytes
+__host__ __device__ inline DownLayout down_layout(int d_e, int E, int NT, int L, int ns,
+                                                  int max_cols) {
+  DownLayout s;
+  s.off_red = kOffIds + align128(E * 4);
+  s.off_h = s.off_red + kWarps * 16 * 8 * NT * 4;
+  s.slot_h = L * 2 * d_e;
+  s.slot_d = max_cols * 2 * d_e;
+  s.off_d = s.off_h + align128(ns * s.slot_h);
+  s.total = s.off_d + ns * s.slot_d;
   return s;
 }
 
@@ -83,115 +88,102 @@ __host__ __device__ inline SmemLayout down_layout(int d_e, int E, int NT, int ns
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
   return static_cast<uint32_t>(__cvta_generic_to_shared(p));
 }
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
-  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+// 16-byte asynchronous copy global -> shared, cached in L2 only.
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
 }
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes)
-               : "memory");
+__device__ __forceinline__ void cp_async_commit() {
+  asm volatile("cp.async.commit_group;" ::: "memory");
 }
-__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
-  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+// Waits until at most N of this thread's most recent commit groups are still in flight.
+template <int N>
+__device__ __forceinline__ void cp_async_wait_group() {
+  asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
 }
-__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile(
-      "{\n"
-      ".reg .pred p;\n"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
-      "selp.u32 %0, 1, 0, p;\n"
-      "}\n"
-      : "=r"(ok)
-      : "r"(bar), "r"(parity)
-      : "memory");
-  return ok != 0;
+__device__ __forceinline__ void cp_async_wait_all() {
+  asm volatile("cp.async.wait_all;" ::: "memory");
 }
-// Bounded wait. Returns false if it gave up (or another thread already had).
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* ctl,
-                                          uint32_t* status) {
-  if (mbar_try_wait(bar, parity)) return true;
-  const long long t0 = clock64();
-  while (true) {
-    if (mbar_try_wait(bar, parity)) return true;
-    if (ctl[1]) return false;
-    if (clock64() - t0 > kWaitCycles) {
-      ctl[1] = 1;
-      atomicOr(status, BLOCKFFN_DEV_WAIT_EXPIRED);
-      return false;
-    }
+// Contiguous run of bytes (a multiple of 16), spread over the CTA's threads. Runs should be
+// long: consecutive cp.async of one thread only overlap when the loop is unrolled (distinct
+// address registers), so many short runs issue several times slower than one long one.
+__device__ __forceinline__ void copy_run(uint32_t dst, const void* src, int bytes) {
+  const char* s = static_cast<const char*>(src);
+#pragma unroll 4
+  for (int o = threadIdx.x * 16; o < bytes; o += kThreads * 16) cp_async16(dst + o, s + o);
+}
+// n_pieces pieces of piece_bytes each (a multiple of 16), piece i from src(i) to
+// dst0 + i * dst_stride. The loop over the pieces is the unrolled one (a loop nested inside
+// it would stop the unrolling and with it the overlap of the copies).
+template <class SrcOf>
+__device__ __forceinline__ void copy_pieces(uint32_t dst0, int dst_stride, int n_pieces,
+                                            int piece_bytes, SrcOf src) {
+  for (int o = threadIdx.x * 16; o < piece_bytes; o += kThreads * 16) {
+#pragma unroll 4
+    for (int i = 0; i < n_pieces; ++i) cp_async16(dst0 + i * dst_stride + o, src(i) + o);
   }
-}
-// 1-D bulk async copy global -> shared, completion counted in bytes on an mbarrier.
-// dst, src and bytes are multiples of 16.
-__device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t bytes,
-                                         uint32_t bar) {
-  asm volatile(
-      "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::
-          "r"(dst),
-      "l"(src), "r"(bytes), "r"(bar)
-      : "memory");
 }
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void pdl_trigger() {
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 }
-__device__ __forceinline__ void consumer_sync() {
-  asm volatile("bar.sync 1, %0;" ::"n"(kConsumerThreads) : "memory");
-}
-__device__ __forceinline__ uint4 lds128(uint32_t addr) {
-  uint4 v;
-  asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];"
-               : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
-               : "r"(addr));
-  return v;
-}
-// D(16x8, f32) += A(16x16, bf16, row) * B(16x8, bf16, col)
+// D(16x8, f32) += A(16x16, bf16, row) * B(16x8, bf16, col). Not volatile: the compiler is
+// free to interleave independent mma chains and the shared-memory loads that feed them.
 __device__ __forceinline__ void mma_bf16(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2,
                                          uint32_t a3, uint32_t b0, uint32_t b1) {
-  asm volatile(
-      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, "
+  asm("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, "
       "{%8,%9}, {%0,%1,%2,%3};"
       : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
       : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
+__device__ __forceinline__ float swish_fast(float z) { return __fdividef(z, 1.0f + __expf(-z)); }
 
 // ---- Union(x) inside the CTA -----------------------------------------------------
-// Fills ids_sm[0 .. nu) with the ascending valid expert ids and returns nu.
+// Fills ids_sm[0 .. nu) with the ascending valid expert ids and returns nu. All global
+// loads of one call are independent of each other, so the routine costs one memory latency.
 // ids_in == NULL: derived from the nonzero pattern of scores (Sec. 3.3); ctl[2] then holds
 // the number of active (token, expert) pairs and ctl[8 ..] the union mask words.
-// ids_in != NULL: taken from the caller's list; entries out of range are dropped and
-// reported, a count out of range is clamped and reported.
+// ids_in != NULL: taken from the caller's list (E entries are readable); entries out of
+// range are dropped and reported, a count out of range is clamped and reported.
+// tm: scratch of at least L * ceil(E/32) words of shared memory.
 __device__ int derive_union(const float* scores, const int32_t* ids_in, const int32_t* n_in,
-                            int L, int E, int* ids_sm, int* ctl, uint32_t* status) {
+                            int L, int E, int* ids_sm, int* ctl, uint32_t* tm) {
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int nwarps = blockDim.x >> 5;
   const int words = (E + 31) >> 5;
   int* cnt = ctl + 40;
   int* act = ctl + 72;
+  uint32_t* um = reinterpret_cast<uint32_t*>(ctl + 8);
   if (ids_in == nullptr) {
-    uint32_t* um = reinterpret_cast<uint32_t*>(ctl + 8);
-    for (int w = warp; w < words; w += nwarps) {
-      const int e = 32 * w + lane;
-      uint32_t un = 0;
-      int nact = 0;
-      for (int t = 0; t < L; ++t) {
-        const float v = (e < E) ? __ldcg(scores + (size_t)t * E + e) : 0.0f;
-        const uint32_t m = __ballot_sync(0xffffffffu, v != 0.0f);
-        un |= m;
-        nact += __popc(m);
-      }
-      if (lane == 0) {
-        cnt[w] = __popc(un);
-        act[w] = nact;
-        um[w] = un;
+    // warp -> tokens warp, warp + nwarps, ...; four mask words in flight per step
+    for (int t = warp; t < L; t += nwarps) {
+      for (int w0 = 0; w0 < words; w0 += 4) {
+        float v[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          const int e = 32 * (w0 + u) + lane;
+          v[u] = e < E ? __ldcg(scores + (size_t)t * E + e) : 0.0f;
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          const uint32_t m = __ballot_sync(0xffffffffu, v[u] != 0.0f);
+          if (lane == 0 && w0 + u < words) tm[t * words + w0 + u] = m;
+        }
       }
     }
     __syncthreads();
-    int total = 0, total_act = 0;
-    for (int w = 0; w < words; ++w) {
-      total += cnt[w];
-      total_act += act[w];
+    if (threadIdx.x < words) {
+      uint32_t un = 0;
+      int nact = 0;
+      for (int t = 0; t < L; ++t) {
+        const uint32_t m = tm[t * words + threadIdx.x];
+        un |= m;
+        nact += __popc(m);
+      }
+      cnt[threadIdx.x] = __popc(un);
+      act[threadIdx.x] = nact;
+      um[threadIdx.x] = un;
     }
+    __syncthreads();
     for (int w = warp; w < words; w += nwarps) {
       int off = 0;
       for (int v = 0; v < w; ++v) off += cnt[v];
@@ -199,30 +191,91 @@ __device__ int derive_union(const float* scores, const int32_t* ids_in, const in
       if ((un >> lane) & 1u) ids_sm[off + __popc(un & ((1u << lane) - 1u))] = 32 * w + lane;
     }
     if (threadIdx.x == 0) {
+      int total = 0, total_act = 0;
+      for (int w = 0; w < words; ++w) {
+        total += cnt[w];
+        total_act += act[w];
+      }
       ctl[0] = total;
       ctl[2] = total_act;
     }
   } else {
-    if (threadIdx.x == 0) {
-      int n = __ldcg(n_in), bad = 0;
-      if (n < 0 || n > E) {
-        bad |= BLOCKFFN_DEV_BAD_UNION_COUNT;
-        n = n < 0 ? 0 : E;
-      }
+    int n = __ldcg(n_in);
+    for (int q = threadIdx.x; q < E; q += blockDim.x) ids_sm[q] = __ldcg(ids_in + q);
+    int bad = 0;
+    if (n < 0 || n > E) {
+      bad = BLOCKFFN_DEV_BAD_UNION_COUNT;
+      n = n < 0 ? 0 : E;
+    }
+    __syncthreads();
+    if (warp == 0) {   // in-place ordered compaction of the valid entries
       int k = 0;
-      for (int q = 0; q < n; ++q) {
-        const int id = __ldcg(ids_in + q);
-        if (id < 0 || id >= E)
-          bad |= BLOCKFFN_DEV_BAD_UNION_ID;
-        else
-          ids_sm[k++] = id;
+      for (int base = 0; base < n; base += 32) {
+        const int q = base + lane;
+        const int id = q < n ? ids_sm[q] : 0;
+        const bool in = q < n, ok = in && id >= 0 && id < E;
+        const uint32_t m = __ballot_sync(0xffffffffu, ok);
+        if (__ballot_sync(0xffffffffu, in && !ok)) bad |= BLOCKFFN_DEV_BAD_UNION_ID;
+        if (ok) ids_sm[k + __popc(m & ((1u << lane) - 1u))] = id;
+        k += __popc(m);
       }
-      ctl[0] = k;
-      ctl[3] = bad;
+      if (lane == 0) {
+        ctl[0] = k;
+        ctl[3] = bad;
+      }
     }
   }
   __syncthreads();
   return ctl[0];
+}
+
+// One 64-wide k block of a 16-row operand tile: rows row_a / row_b (byte addresses of the
+// block within the row), this lane's 16 bytes of each 32-wide half. Lanes of odd rows
+// read the halves in the opposite order (bank spread) and swap them back.
+struct Frag64 {
+  uint4 lo, hi;   // first / second 32-wide half
+};
+// row: shared-memory address of the 64-wide block inside the operand row (128-byte aligned)
+__device__ __forceinline__ Frag64 load_frag64(const unsigned char* row, int par, int tg) {
+  const uint4 first = *reinterpret_cast<const uint4*>(row + 64 * par + 16 * tg);
+  const uint4 second = *reinterpret_cast<const uint4*>(row + 64 * (par ^ 1) + 16 * tg);
+  Frag64 f;
+  f.lo = par ? second : first;
+  f.hi = par ? first : second;
+  return f;
+}
+// acc0 takes the first 32-wide half, acc1 the second: two independent dependency chains.
+template <int NT>
+__device__ __forceinline__ void mma_block64(float (&acc0)[NT][4], float (&acc1)[NT][4],
+                                            const Frag64& ra, const Frag64& rb,
+                                            const Frag64 (&xb)[NT]) {
+#pragma unroll
+  for (int n = 0; n < NT; ++n) {
+    mma_bf16(acc0[n], ra.lo.x, rb.lo.x, ra.lo.y, rb.lo.y, xb[n].lo.x, xb[n].lo.y);
+    mma_bf16(acc1[n], ra.hi.x, rb.hi.x, ra.hi.y, rb.hi.y, xb[n].hi.x, xb[n].hi.y);
+    mma_bf16(acc0[n], ra.lo.z, rb.lo.z, ra.lo.w, rb.lo.w, xb[n].lo.z, xb[n].lo.w);
+    mma_bf16(acc1[n], ra.hi.z, rb.hi.z, ra.hi.w, rb.hi.w, xb[n].hi.z, xb[n].hi.w);
+  }
+}
+// The 16 x (8 NT) accumulator tile of one warp (both chains summed) -> mine[t * ld + m0 + .]
+template <int NT>
+__device__ __forceinline__ void store_partial(float* mine, int ld, int m0, const float (&a0)[NT][4],
+                                              const float (&a1)[NT][4], int g, int tg) {
+#pragma unroll
+  for (int n = 0; n < NT; ++n) {
+    const int t = 8 * n + 2 * tg;
+    mine[t * ld + m0 + g] = a0[n][0] + a1[n][0];
+    mine[(t + 1) * ld + m0 + g] = a0[n][1] + a1[n][1];
+    mine[t * ld + m0 + g + 8] = a0[n][2] + a1[n][2];
+    mine[(t + 1) * ld + m0 + g + 8] = a0[n][3] + a1[n][3];
+  }
+}
+template <int NT>
+__device__ __forceinline__ void zero_acc(float (&a)[NT][4]) {
+#pragma unroll
+  for (int n = 0; n < NT; ++n)
+#pragma unroll
+    for (int v = 0; v < 4; ++v) a[n][v] = 0.0f;
 }
 
 // ---- up projection ---------------------------------------------------------------
@@ -232,8 +285,8 @@ struct UpParams {
   const float* scores;     // f32 [L][E]
   const int32_t* ids_in;   // caller's union list, or NULL: derive from scores
   const int32_t* n_in;
-  uint16_t* h;             // bf16 [q][L][d_e + 32] intermediate
-  int L, d, E, d_e, ns, early;
+  uint16_t* h;             // bf16 [q][L][d_e] intermediate
+  int L, d, E, d_e, de_shift, ring_rows, early;   // de_shift: log2(d_e), or -1
   uint32_t* status;
   // what CTA 0 publishes when it derived the union itself (each may be NULL)
   uint32_t* pub_mask;
@@ -246,25 +299,16 @@ template <int NT>
 __global__ void __launch_bounds__(kThreads, 1) expert_up_mma_kernel(const UpParams p) {
   extern __shared__ __align__(128) unsigned char smem[];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const SmemLayout lay = up_layout(p.d, p.E, NT, p.ns);
+  const int d = p.d, d_e = p.d_e, L = p.L;
+  constexpr int ns = kUpStages;
+  const UpLayout lay = up_layout(d, p.E, NT, L, p.ring_rows);
   const uint32_t sbase = smem_u32(smem);
-  const uint32_t bar_full = sbase + kOffBars, bar_empty = bar_full + 8 * kMaxStages,
-                 bar_x = bar_empty + 8 * kMaxStages;
-  int* ctl = reinterpret_cast<int*>(smem + lay.off_ctl);
-  int* ids_sm = reinterpret_cast<int*>(smem + lay.off_ids);
+  int* ctl = reinterpret_cast<int*>(smem + kOffCtl);
+  int* ids_sm = reinterpret_cast<int*>(smem + kOffIds);
   float* red = reinterpret_cast<float*>(smem + lay.off_red);
-  const int d = p.d, d_e = p.d_e, L = p.L, ns = p.ns;
-  const int XS = 2 * d + kPad, RS = 2 * kKC + kPad;
+  const int row_bytes = 2 * d;
 
-  if (tid == 0) {
-    for (int s = 0; s < ns; ++s) {
-      mbar_init(bar_full + 8 * s, 1);
-      mbar_init(bar_empty + 8 * s, kConsumerWarps);
-    }
-    mbar_init(bar_x, 1);
-    for (int v = 0; v < 8; ++v) ctl[v] = 0;
-    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-  }
+  if (tid < 8) ctl[tid] = 0;
   if (p.early) {
     pdl_trigger();       // the next kernel may start fetching its weights right away
   } else {
@@ -272,146 +316,166 @@ __global__ void __launch_bounds__(kThreads, 1) expert_up_mma_kernel(const UpPara
     pdl_trigger();
   }
   __syncthreads();
-  const int nu = derive_union(p.scores, p.ids_in, p.n_in, L, p.E, ids_sm, ctl, p.status);
+  const int nu = derive_union(p.scores, p.ids_in, p.n_in, L, p.E, ids_sm, ctl,
+                              reinterpret_cast<uint32_t*>(red));
 
-  const long long R = (long long)nu * d_e;
-  const int r0 = (int)(R * blockIdx.x / gridDim.x), r1 = (int)(R * (blockIdx.x + 1) / gridDim.x);
-  const int nrows = r1 - r0;
-  const int mt = (nrows + 15) >> 4;
-  const int nkc = (d + kKC - 1) / kKC;
-  const int nstages = mt * nkc;
+  // This CTA's rows [r0, r1) of the u * d_e union rows (balanced: the first R % G CTAs take
+  // one row more). They are one stage when they fit the ring (the usual case), else stages
+  // of a third of the ring that are refilled as they free.
+  const int R = nu * d_e, G = gridDim.x, bx = blockIdx.x;
+  const int rq = R / G, rrem = R - rq * G;
+  const int r0 = bx * rq + min(bx, rrem), nrows = rq + (bx < rrem ? 1 : 0), r1 = r0 + nrows;
+  const bool single = nrows <= min(32, p.ring_rows);
+  const int slot_rows = single ? max(nrows, 1) : min(32, p.ring_rows / ns);
+  const int ngroups = (nrows + slot_rows - 1) / slot_rows;
+  const int rpg = ngroups ? (nrows + ngroups - 1) / ngroups : 0;
+  const int slot_bytes = slot_rows * row_bytes;
+  const int sh = p.de_shift;
+  auto row_q = [&](int r) { return sh >= 0 ? r >> sh : r / d_e; };
 
-  if (warp == kConsumerWarps) {
-    // ===== producer warp: lane m copies row m of the stage's tile =====
-    auto issue = [&](int s) {
-      const int slot = s % ns, tile = s / nkc, kc = s - tile * nkc;
-      const int k0 = kc * kKC, klen = min(kKC, d - k0);
-      const int rows = min(16, nrows - tile * 16);
-      if (lane == 0) mbar_expect_tx(bar_full + 8 * slot, (uint32_t)(rows * klen * 2));
-      __syncwarp();
-      if (lane < rows) {
-        const int r = r0 + tile * 16 + lane;
-        const int q = r / d_e, j = r - q * d_e;
-        const uint16_t* src = p.U + ((size_t)ids_sm[q] * d_e + j) * d + k0;
-        bulk_g2s(sbase + lay.off_ring + slot * lay.slot_bytes + lane * RS, src,
-                 (uint32_t)(klen * 2), bar_full + 8 * slot);
+  // stage gi: rows [r0 + gi rpg, ...) -> slot gi % ns; one run per expert the rows fall in
+  auto issue = [&](int gi) {
+    int ra = r0 + gi * rpg;
+    const int rb = min(r1, ra + rpg);
+    uint32_t dst = sbase + lay.off_ring + (gi % ns) * slot_bytes;
+    int q = row_q(ra), j = ra - q * d_e;
+    while (ra < rb) {
+      const int n = min(rb - ra, d_e - j);
+      copy_run(dst, p.U + ((size_t)ids_sm[q] * d_e + j) * d, n * row_bytes);
+      dst += n * row_bytes;
+      ra += n;
+      ++q;
+      j = 0;
+    }
+  };
+  // The router score, expert slot and neuron of each element this thread finishes in a stage
+  // (element e = t * 32 + m: token t, row m of the stage).
+  float sc[NT];
+  int hq[NT], hj[NT];
+  auto prepare = [&](int gi) {
+    const int ra = r0 + gi * rpg, rows = min(r1, ra + rpg) - ra;
+#pragma unroll
+    for (int i = 0; i < NT; ++i) {
+      const int e = tid + i * kThreads, t = e >> 5, m = e & 31;
+      sc[i] = 0.0f;
+      hq[i] = -1;
+      if (t < L && m < rows) {
+        hq[i] = row_q(ra + m);
+        hj[i] = ra + m - hq[i] * d_e;
+        sc[i] = __ldcg(p.scores + (size_t)t * p.E + ids_sm[hq[i]]);
       }
-    };
-    const int s_pre = p.early ? min(nstages, ns) : 0;
-    for (int s = 0; s < s_pre; ++s) issue(s);
-    pdl_wait();          // x may come from the kernel just before
-    if (nstages > 0) {
-      if (lane == 0) mbar_expect_tx(bar_x, (uint32_t)(L * d * 2));
-      __syncwarp();
-      for (int t = lane; t < L; t += 32)
-        bulk_g2s(sbase + lay.off_x + t * XS, p.x + (size_t)t * d, (uint32_t)(d * 2), bar_x);
     }
-    for (int s = s_pre; s < nstages; ++s) {
-      if (s >= ns) mbar_wait(bar_empty + 8 * (s % ns), ((s / ns) - 1) & 1, ctl, p.status);
-      issue(s);
-    }
-    // Outstanding copies: every stage issued is also awaited by the consumers; if they
-    // gave up, wait here (bounded) so that no copy lands after the CTA is gone.
-    if (ctl[1]) {
-      for (int s = max(0, nstages - ns); s < nstages; ++s)
-        mbar_wait(bar_full + 8 * (s % ns), (s / ns) & 1, ctl + 4, p.status);
-      if (nstages > 0) mbar_wait(bar_x, 0, ctl + 4, p.status);
-    }
-  } else {
-    // ===== consumer warps =====
-    pdl_wait();
-    const int g = lane >> 2, tg = lane & 3;
-    if (nstages > 0) mbar_wait(bar_x, 0, ctl, p.status);
-    for (int tile = 0; tile < mt; ++tile) {
-      float acc[NT][4];
+  };
+  const int g = lane >> 2, tg = lane & 3, par = g & 1;
+  const int npairs = d >> 6;   // 64-wide k blocks
+  const unsigned char* x_row[NT];
 #pragma unroll
-      for (int n = 0; n < NT; ++n)
-#pragma unroll
-        for (int v = 0; v < 4; ++v) acc[n][v] = 0.0f;
-      for (int kc = 0; kc < nkc; ++kc) {
-        const int s = tile * nkc + kc, slot = s % ns;
-        const int k0 = kc * kKC, nsb = min(kKC, d - k0) >> 5;
-        mbar_wait(bar_full + 8 * slot, (s / ns) & 1, ctl, p.status);
-        const uint32_t a_base = sbase + lay.off_ring + slot * lay.slot_bytes + g * RS + tg * 16;
-        const uint32_t b_base = sbase + lay.off_x + g * XS + k0 * 2 + tg * 16;
+  for (int n = 0; n < NT; ++n) x_row[n] = smem + lay.off_x + min(8 * n + g, L - 1) * row_bytes;
+
+  const int g_first = min(ngroups, ns);
+  if (p.early) {
+    for (int gi = 0; gi < g_first; ++gi) issue(gi);
+    if (ngroups > 0) prepare(0);
+  }
+  pdl_wait();            // x may come from the kernel just before; h may still be read by it
+  if (ngroups > 0) copy_run(sbase + lay.off_x, p.x, L * row_bytes);
+  if (!p.early) {
+    for (int gi = 0; gi < g_first; ++gi) issue(gi);
+    if (ngroups > 0) prepare(0);
+  }
+  cp_async_commit();
+  cp_async_wait_group<0>();
+  __syncthreads();
+
+  for (int gi = 0; gi < ngroups; ++gi) {
+    const int rows = min(r1, r0 + (gi + 1) * rpg) - (r0 + gi * rpg);
+    const unsigned char* slot = smem + lay.off_ring + (gi % ns) * slot_bytes;
+    const bool two = rows > 16;   // second block of 16 rows
+    const unsigned char* ra0 = slot + min(g, rows - 1) * row_bytes;
+    const unsigned char* rb0 = slot + min(g + 8, rows - 1) * row_bytes;
+    const unsigned char* ra1 = slot + min(g + 16, rows - 1) * row_bytes;
+    const unsigned char* rb1 = slot + min(g + 24, rows - 1) * row_bytes;
+    float a00[NT][4], a01[NT][4], a10[NT][4], a11[NT][4];
+    zero_acc<NT>(a00);
+    zero_acc<NT>(a01);
+    zero_acc<NT>(a10);
+    zero_acc<NT>(a11);
 #pragma unroll 2
-        for (int sb = warp; sb < nsb; sb += kConsumerWarps) {
-          const uint4 ra = lds128(a_base + sb * 64);
-          const uint4 rb = lds128(a_base + 8 * RS + sb * 64);
+    for (int pp = warp; pp < npairs; pp += kWarps) {
+      Frag64 fx[NT];
 #pragma unroll
-          for (int n = 0; n < NT; ++n) {
-            const uint4 xb = lds128(b_base + n * 8 * XS + sb * 64);
-            mma_bf16(acc[n], ra.x, rb.x, ra.y, rb.y, xb.x, xb.y);
-            mma_bf16(acc[n], ra.z, rb.z, ra.w, rb.w, xb.z, xb.w);
-          }
-        }
-        __syncwarp();
-        if (lane == 0) mbar_arrive(bar_empty + 8 * slot);
+      for (int n = 0; n < NT; ++n) fx[n] = load_frag64(x_row[n] + 128 * pp, par, tg);
+      const Frag64 fa = load_frag64(ra0 + 128 * pp, par, tg);
+      const Frag64 fb = load_frag64(rb0 + 128 * pp, par, tg);
+      mma_block64<NT>(a00, a01, fa, fb, fx);
+      if (two) {
+        const Frag64 fc = load_frag64(ra1 + 128 * pp, par, tg);
+        const Frag64 fd = load_frag64(rb1 + 128 * pp, par, tg);
+        mma_block64<NT>(a10, a11, fc, fd, fx);
       }
-      // cross-warp reduction of the K split, then Swish, score, store
-      float* mine = red + warp * (16 * 8 * NT);
-#pragma unroll
-      for (int n = 0; n < NT; ++n) {
-        const int t = 8 * n + 2 * tg;
-        mine[t * 16 + g] = acc[n][0];
-        mine[(t + 1) * 16 + g] = acc[n][1];
-        mine[t * 16 + g + 8] = acc[n][2];
-        mine[(t + 1) * 16 + g + 8] = acc[n][3];
-      }
-      consumer_sync();
-      const int rows = min(16, nrows - tile * 16);
-      for (int e = tid; e < 16 * 8 * NT; e += kConsumerThreads) {
-        const int t = e >> 4, m = e & 15;
-        if (t < L && m < rows) {
-          float v = 0.0f;
-#pragma unroll
-          for (int w = 0; w < kConsumerWarps; ++w) v += red[w * (16 * 8 * NT) + e];
-          const int r = r0 + tile * 16 + m;
-          const int q = r / d_e, j = r - q * d_e;
-          const float s = __ldcg(p.scores + (size_t)t * p.E + ids_sm[q]);
-          p.h[((size_t)q * L + t) * (d_e + 32) + j] = (uint16_t)f32_to_bf16_bits(s * swish(v));
-        }
-      }
-      consumer_sync();
     }
-    // CTA 0 publishes the routing it derived (after the wait: earlier readers are done)
-    if (blockIdx.x == 0) {
-      if (p.ids_in == nullptr) {
-        const int words = (p.E + 31) >> 5;
-        const uint32_t* um = reinterpret_cast<const uint32_t*>(ctl + 8);
-        for (int e = tid; e < p.E; e += kConsumerThreads) {
-          if (p.pub_ids) p.pub_ids[e] = e < nu ? ids_sm[e] : -1;
-          if (p.pub_mask && e < words) p.pub_mask[e] = um[e];
-        }
-        if (tid == 0) {
-          if (p.pub_n) *p.pub_n = nu;
-          if (p.stats) {
-            atomicAdd(reinterpret_cast<unsigned long long*>(&p.stats->n_tokens),
-                      (unsigned long long)L);
-            atomicAdd(reinterpret_cast<unsigned long long*>(&p.stats->n_active),
-                      (unsigned long long)ctl[2]);
-            atomicAdd(reinterpret_cast<unsigned long long*>(&p.stats->n_chunks), 1ull);
-            atomicAdd(reinterpret_cast<unsigned long long*>(&p.stats->n_union),
-                      (unsigned long long)nu);
-          }
-        }
-      } else if (tid == 0 && ctl[3]) {
-        atomicOr(p.status, (uint32_t)ctl[3]);
+    // cross-warp reduction of the K split, then Swish, score, store
+    float* mine = red + warp * (32 * 8 * NT);
+    store_partial<NT>(mine, 32, 0, a00, a01, g, tg);
+    if (two) store_partial<NT>(mine, 32, 16, a10, a11, g, tg);
+    __syncthreads();     // every warp is done with the slot: refill it
+    if (gi + ns < ngroups) issue(gi + ns);
+    cp_async_commit();   // one group per stage, empty or not, keeps the count below uniform
+#pragma unroll
+    for (int i = 0; i < NT; ++i) {
+      if (hq[i] >= 0) {
+        const int e = tid + i * kThreads;
+        float v = 0.0f;
+#pragma unroll
+        for (int w = 0; w < kWarps; ++w) v += red[w * (32 * 8 * NT) + e];
+        p.h[((size_t)hq[i] * L + (e >> 5)) * d_e + hj[i]] =
+            (uint16_t)f32_to_bf16_bits(sc[i] * swish_fast(v));
       }
+    }
+    if (gi + 1 < ngroups) prepare(gi + 1);
+    // stage gi + 1, if it is a refill, was committed ns - 1 groups ago
+    if (gi + 1 >= ns) cp_async_wait_group<ns - 1>();
+    __syncthreads();
+  }
+  // CTA 0 publishes the routing it derived (after the wait: earlier readers are done)
+  if (blockIdx.x == 0) {
+    if (p.ids_in == nullptr) {
+      const int words = (p.E + 31) >> 5;
+      const uint32_t* um = reinterpret_cast<const uint32_t*>(ctl + 8);
+      for (int e = tid; e < p.E; e += kThreads) {
+        if (p.pub_ids) p.pub_ids[e] = e < nu ? ids_sm[e] : -1;
+        if (p.pub_mask && e < words) p.pub_mask[e] = um[e];
+      }
+      if (tid == 0) {
+        if (p.pub_n) *p.pub_n = nu;
+        if (p.stats) {
+          atomicAdd(reinterpret_cast<unsigned long long*>(&p.stats->n_tokens),
+                    (unsigned long long)L);
+          atomicAdd(reinterpret_cast<unsigned long long*>(&p.stats->n_active),
+                    (unsigned long long)ctl[2]);
+          atomicAdd(reinterpret_cast<unsigned long long*>(&p.stats->n_chunks), 1ull);
+          atomicAdd(reinterpret_cast<unsigned long long*>(&p.stats->n_union),
+                    (unsigned long long)nu);
+        }
+      }
+    } else if (tid == 0 && ctl[3]) {
+      atomicOr(p.status, (uint32_t)ctl[3]);
     }
   }
+  cp_async_wait_all();
 }
 
 // ---- down projection ---------------------------------------------------------------
 struct DownParams {
   const uint16_t* D;       // bf16 [E][d][d_e]
-  const uint16_t* h;       // bf16 [q][L][d_e + 32]
+  const uint16_t* h;       // bf16 [q][L][d_e]
   const float* scores;
   const int32_t* ids_in;
   const int32_t* n_in;
   float* out;              // f32 [L][d]
   uint16_t* x_next;        // bf16 [L][d] or NULL
-  int L, d, E, d_e, ns, accumulate;
+  int L, d, E, d_e, ns, max_cols, per, accumulate;
+  int cols_q, cols_rem;    // the d columns over G * per tiles: tile w has cols_q + (w < cols_rem)
   uint32_t* status;
 };
 
@@ -419,176 +483,224 @@ template <int NT>
 __global__ void __launch_bounds__(kThreads, 1) expert_down_mma_kernel(const DownParams p) {
   extern __shared__ __align__(128) unsigned char smem[];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const SmemLayout lay = down_layout(p.d_e, p.E, NT, p.ns);
+  const int d = p.d, d_e = p.d_e, L = p.L, per = p.per;
+  const DownLayout lay = down_layout(d_e, p.E, NT, L, p.ns, p.max_cols);
   const uint32_t sbase = smem_u32(smem);
-  const uint32_t bar_full = sbase + kOffBars, bar_empty = bar_full + 8 * kMaxStages;
-  int* ctl = reinterpret_cast<int*>(smem + lay.off_ctl);
-  int* ids_sm = reinterpret_cast<int*>(smem + lay.off_ids);
+  int* ctl = reinterpret_cast<int*>(smem + kOffCtl);
+  int* ids_sm = reinterpret_cast<int*>(smem + kOffIds);
   float* red = reinterpret_cast<float*>(smem + lay.off_red);
-  const int d = p.d, d_e = p.d_e, L = p.L, ns = p.ns;
-  const int DS = 2 * d_e, HS = 2 * d_e + kPad;   // bytes per staged D row / h row
-  const uint32_t h_bytes = (uint32_t)(L * HS);
+  const int row_bytes = 2 * d_e;
 
-  if (tid == 0) {
-    for (int s = 0; s < ns; ++s) {
-      mbar_init(bar_full + 8 * s, 1);
-      mbar_init(bar_empty + 8 * s, kConsumerWarps);
-    }
-    for (int v = 0; v < 8; ++v) ctl[v] = 0;
-    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-  }
+  if (tid < 8) ctl[tid] = 0;
   pdl_trigger();
   __syncthreads();
   // The routing inputs were final before the up kernel of this call passed its own wait.
-  const int nu = derive_union(p.scores, p.ids_in, p.n_in, L, p.E, ids_sm, ctl, p.status);
+  const int nu = derive_union(p.scores, p.ids_in, p.n_in, L, p.E, ids_sm, ctl,
+                              reinterpret_cast<uint32_t*>(red));
 
-  // column tiles: W = G * ceil(d / 16G) tiles of at most 16 columns, tile w -> CTA w % G
+  // Column tiles: G * per tiles of at most max_cols (<= 16) columns, tile w -> CTA w % G,
+  // tile w = columns [w cols_q + min(w, cols_rem), ...). Per tile, the experts go through
+  // the ring in rounds: all of them at once when they fit (the usual case), else half a
+  // ring per round, the next round in flight during the math.
   const int G = gridDim.x;
-  const int per = (d + 16 * G - 1) / (16 * G);
-  const long long W = (long long)G * per;
-  auto tile_c0 = [&](int ti) { return (int)((long long)d * (blockIdx.x + (long long)ti * G) / W); };
-  auto tile_c1 = [&](int ti) {
-    return (int)((long long)d * (blockIdx.x + (long long)ti * G + 1) / W);
+  const int rsz = (per == 1 && nu <= p.ns) ? max(nu, 1) : max(1, min(nu, p.ns / 2));
+  const int rpt = (nu + rsz - 1) / rsz;                  // rounds per tile
+  const int nrounds = per * rpt;
+  const char* dptr = reinterpret_cast<const char*>(p.D);
+  const size_t estride = (size_t)d * d_e * 2;
+  const char* hptr = reinterpret_cast<const char*>(p.h);
+  auto tile_c0 = [&](int ti) {
+    const int w = blockIdx.x + ti * G;
+    return w * p.cols_q + min(w, p.cols_rem);
   };
-  const int nstages = per * nu;   // empty tiles keep their stages (h only), which is rare
+  auto tile_nc = [&](int ti) { return p.cols_q + ((int)blockIdx.x + ti * G < p.cols_rem ? 1 : 0); };
+  // (i_ti, i_rr): tile and round-in-tile of the next round to request; (c_ti, c_rr): to compute
+  int i_r = 0, i_ti = 0, i_rr = 0;
+  auto issue_d = [&]() {
+    const int q0 = i_rr * rsz, n = min(rsz, nu - q0);
+    const char* base = dptr + (size_t)tile_c0(i_ti) * row_bytes;
+    copy_pieces(sbase + lay.off_d + (i_r & 1) * rsz * lay.slot_d, lay.slot_d, n,
+                tile_nc(i_ti) * row_bytes,
+                [&](int i) { return base + (size_t)ids_sm[q0 + i] * estride; });
+  };
+  auto issue_h = [&](int r, int rr) {
+    const int q0 = rr * rsz, n = min(rsz, nu - q0);
+    copy_run(sbase + lay.off_h + (r & 1) * rsz * lay.slot_h, hptr + (size_t)q0 * lay.slot_h,
+             n * lay.slot_h);
+  };
+  auto advance = [&]() {
+    ++i_r;
+    if (++i_rr == rpt) {
+      i_rr = 0;
+      ++i_ti;
+    }
+  };
+  const int g = lane >> 2, tg = lane & 3, par = g & 1;
+  const int npairs = d_e >> 6;         // 64-wide k blocks per expert
+  const int pshift = (npairs & (npairs - 1)) == 0 ? __ffs(npairs) - 1 : -1;
+  int h_off[NT];
+#pragma unroll
+  for (int n = 0; n < NT; ++n) h_off[n] = min(8 * n + g, L - 1) * row_bytes;
 
-  if (warp == kConsumerWarps) {
-    // ===== producer lane =====
-    if (lane == 0) {
-      auto issue_d = [&](int s) {
-        const int slot = s % ns, ti = s / nu, q = s - ti * nu;
-        const int c0 = tile_c0(ti), ncols = tile_c1(ti) - c0;
-        const uint32_t d_bytes = (uint32_t)(ncols * DS);
-        mbar_expect_tx(bar_full + 8 * slot, d_bytes + h_bytes);
-        if (ncols > 0)
-          bulk_g2s(sbase + lay.off_ring + slot * lay.slot_bytes,
-                   p.D + ((size_t)ids_sm[q] * d + c0) * d_e, d_bytes, bar_full + 8 * slot);
-      };
-      auto issue_h = [&](int s) {
-        const int slot = s % ns, q = s % nu;
-        bulk_g2s(sbase + lay.off_ring + slot * lay.slot_bytes + lay.slot_h_off,
-                 p.h + (size_t)q * L * (d_e + 32), h_bytes, bar_full + 8 * slot);
-      };
-      const int s_pre = min(nstages, ns);
-      for (int s = 0; s < s_pre; ++s) issue_d(s);
-      pdl_wait();        // h is complete and visible from here on
-      for (int s = 0; s < s_pre; ++s) issue_h(s);
-      for (int s = s_pre; s < nstages; ++s) {
-        mbar_wait(bar_empty + 8 * (s % ns), ((s / ns) - 1) & 1, ctl, p.status);
-        issue_d(s);
-        issue_h(s);
-      }
-      if (ctl[1]) {
-        for (int s = max(0, nstages - ns); s < nstages; ++s)
-          mbar_wait(bar_full + 8 * (s % ns), (s / ns) & 1, ctl + 4, p.status);
+  // before the wait: the weights of the first two rounds; after it: their h
+  const int npre = min(nrounds, 2);
+  const int rr1 = rpt > 1 ? 1 : 0;     // round-in-tile of round 1
+  for (int r = 0; r < npre; ++r) {
+    issue_d();
+    advance();
+    cp_async_commit();
+  }
+  pdl_wait();            // h, out and x_next are safe to touch from here on
+  if (npre > 0) {
+    issue_h(0, 0);
+    cp_async_commit();
+  }
+  if (npre > 1) {
+    issue_h(1, rr1);
+    cp_async_commit();
+  }
+
+  float acc0[NT][4], acc1[NT][4];
+  int c_ti = 0, c_rr = 0;
+  for (int r = 0; r < nrounds; ++r) {
+    const int q0 = c_rr * rsz, n = min(rsz, nu - q0);
+    const int c0 = tile_c0(c_ti), ncols = tile_nc(c_ti);
+    if (c_rr == 0) {
+      zero_acc<NT>(acc0);
+      zero_acc<NT>(acc1);
+    }
+    // everything but the newest group has to have landed (the newest is the next round's)
+    if (r + 1 < nrounds) cp_async_wait_group<1>(); else cp_async_wait_group<0>();
+    __syncthreads();
+    if (ncols > 0) {
+      const int off_a = min(g, ncols - 1) * row_bytes, off_b = min(g + 8, ncols - 1) * row_bytes;
+      const unsigned char* d_base = smem + lay.off_d + (r & 1) * rsz * lay.slot_d;
+      const unsigned char* h_base = smem + lay.off_h + (r & 1) * rsz * lay.slot_h;
+      // the 64-wide k blocks of the round's experts are dealt round-robin to the warps
+      const int nblk = n * npairs;
+#pragma unroll 2
+      for (int b = warp; b < nblk; b += kWarps) {
+        const int i = pshift >= 0 ? b >> pshift : b / npairs, pp = b - i * npairs;
+        const unsigned char* da = d_base + i * lay.slot_d + 128 * pp;
+        const unsigned char* ha = h_base + i * lay.slot_h + 128 * pp;
+        const Frag64 fa = load_frag64(da + off_a, par, tg);
+        const Frag64 fb = load_frag64(da + off_b, par, tg);
+        Frag64 fx[NT];
+#pragma unroll
+        for (int nn = 0; nn < NT; ++nn) fx[nn] = load_frag64(ha + h_off[nn], par, tg);
+        mma_block64<NT>(acc0, acc1, fa, fb, fx);
       }
     }
-  } else {
-    // ===== consumer warps =====
-    pdl_wait();
-    const int g = lane >> 2, tg = lane & 3;
-    const int nsb = d_e >> 5;            // 32-wide k blocks per expert
-    for (int ti = 0; ti < per; ++ti) {
-      const int c0 = tile_c0(ti), ncols = tile_c1(ti) - c0;
-      float acc[NT][4];
-#pragma unroll
-      for (int n = 0; n < NT; ++n)
-#pragma unroll
-        for (int v = 0; v < 4; ++v) acc[n][v] = 0.0f;
-      for (int q = 0; q < nu; ++q) {
-        const int s = ti * nu + q, slot = s % ns;
-        mbar_wait(bar_full + 8 * slot, (s / ns) & 1, ctl, p.status);
-        const uint32_t a_base = sbase + lay.off_ring + slot * lay.slot_bytes + g * DS + tg * 16;
-        const uint32_t b_base =
-            sbase + lay.off_ring + slot * lay.slot_bytes + lay.slot_h_off + g * HS + tg * 16;
-        // k blocks of all experts are dealt round-robin to the warps
-        for (int sb = (warp - q * nsb) & (kConsumerWarps - 1); sb < nsb; sb += kConsumerWarps) {
-          const uint4 ra = lds128(a_base + sb * 64);
-          const uint4 rb = lds128(a_base + 8 * DS + sb * 64);
-#pragma unroll
-          for (int n = 0; n < NT; ++n) {
-            const uint4 xb = lds128(b_base + n * 8 * HS + sb * 64);
-            mma_bf16(acc[n], ra.x, rb.x, ra.y, rb.y, xb.x, xb.y);
-            mma_bf16(acc[n], ra.z, rb.z, ra.w, rb.w, xb.z, xb.w);
-          }
-        }
-        __syncwarp();
-        if (lane == 0) mbar_arrive(bar_empty + 8 * slot);
-      }
-      float* mine = red + warp * (16 * 8 * NT);
-#pragma unroll
-      for (int n = 0; n < NT; ++n) {
-        const int t = 8 * n + 2 * tg;
-        mine[t * 16 + g] = acc[n][0];
-        mine[(t + 1) * 16 + g] = acc[n][1];
-        mine[t * 16 + g + 8] = acc[n][2];
-        mine[(t + 1) * 16 + g + 8] = acc[n][3];
-      }
-      consumer_sync();
-      for (int e = tid; e < 16 * 8 * NT; e += kConsumerThreads) {
+    if (r + 2 < nrounds) {       // refill this round's half of the ring
+      __syncthreads();
+      issue_d();
+      issue_h(i_r, i_rr);
+      advance();
+      cp_async_commit();
+    }
+    if (c_rr == rpt - 1) {       // the tile is complete: reduce across warps and store
+      store_partial<NT>(red + warp * (16 * 8 * NT), 16, 0, acc0, acc1, g, tg);
+      __syncthreads();
+      for (int e = tid; e < 16 * 8 * NT; e += kThreads) {
         const int t = e >> 4, m = e & 15;
         if (t < L && m < ncols) {
           float v = 0.0f;
 #pragma unroll
-          for (int w = 0; w < kConsumerWarps; ++w) v += red[w * (16 * 8 * NT) + e];
+          for (int w = 0; w < kWarps; ++w) v += red[w * (16 * 8 * NT) + e];
           const size_t o = (size_t)t * d + c0 + m;
           if (p.accumulate) v += __ldcg(p.out + o);
           p.out[o] = v;
           if (p.x_next) p.x_next[o] = (uint16_t)f32_to_bf16_bits(v);
         }
       }
-      consumer_sync();
+      __syncthreads();
+    }
+    if (++c_rr == rpt) {
+      c_rr = 0;
+      ++c_ti;
     }
   }
+  if (nu == 0) {               // empty union: FFN(x) = 0
+    for (int ti = 0; ti < per; ++ti) {
+      const int c0 = tile_c0(ti), ncols = tile_nc(ti);
+      for (int e = tid; e < L * ncols; e += kThreads) {
+        const int t = e / ncols, m = e - t * ncols;
+        const size_t o = (size_t)t * d + c0 + m;
+        const float v = p.accumulate ? __ldcg(p.out + o) : 0.0f;
+        p.out[o] = v;
+        if (p.x_next) p.x_next[o] = (uint16_t)f32_to_bf16_bits(v);
+      }
+    }
+  }
+  cp_async_wait_all();
 }
 
 // ---- host side -----------------------------------------------------------------------
 struct MmaPlan {
-  int NT, ns_up, ns_down, smem_up, smem_down;
+  int NT, ring_rows, ns_down, max_cols, per, cols_q, cols_rem, smem_up, smem_down;
   bool ok;
 };
 
-MmaPlan make_plan(const blockffn_config& cfg, int L) {
+// Shapes the kernels take: d and d_e multiples of 64 (whole 64-wide k blocks, row strides
+// multiples of 128 bytes) and shared memory for x plus two stages of rows / two expert slabs.
+MmaPlan make_plan(const blockffn_config& cfg, int L, int grid) {
   MmaPlan pl{};
   pl.ok = false;
-  if (L < 1 || L > 32) return pl;
-  if (cfg.d % 32 || cfg.d_e % 32 || cfg.E > 1024) return pl;
-  if (cfg.d_e > 2048 || cfg.d > 65536) return pl;
-  if ((long long)32 * (2 * cfg.d_e + kPad) + 16 * 2 * cfg.d_e >= (1 << 20)) return pl;  // tx count
+  const int d = cfg.d, d_e = cfg.d_e, E = cfg.E;
+  if (L < 1 || L > 32 || grid < 1) return pl;
+  if (d % 64 || d_e % 64 || E > 1024 || d > 32768 || d_e > 4096) return pl;
   pl.NT = (L + 7) / 8;
   const int want_up = cfg.flags & 0xff, want_down = (cfg.flags >> 8) & 0xff;
-  auto pick = [&](auto layout_of, int want) {
-    const SmemLayout one = layout_of(1);
-    const int base = one.total - one.slot_bytes;
-    int ns = (kSmemHalf - base) / one.slot_bytes;        // share the SM with the other kernel
-    if (ns < 2) ns = (kSmemMax - base) / one.slot_bytes; // or take it alone
-    if (want) ns = want;
-    if (ns > kMaxStages) ns = kMaxStages;
-    if (base + ns * one.slot_bytes > kSmemMax) ns = (kSmemMax - base) / one.slot_bytes;
-    return ns;
-  };
-  pl.ns_up = pick([&](int ns) { return up_layout(cfg.d, cfg.E, pl.NT, ns); }, want_up);
-  pl.ns_down = pick([&](int ns) { return down_layout(cfg.d_e, cfg.E, pl.NT, ns); }, want_down);
-  if (pl.ns_up < 2 || pl.ns_down < 2) return pl;
-  if (pl.ns_up > 8) pl.ns_up = want_up ? pl.ns_up : 8;
-  pl.smem_up = up_layout(cfg.d, cfg.E, pl.NT, pl.ns_up).total;
-  pl.smem_down = down_layout(cfg.d_e, cfg.E, pl.NT, pl.ns_down).total;
+  // down: column tiles
+  pl.per = (d + 16 * grid - 1) / (16 * grid);
+  const int W = grid * pl.per;
+  pl.cols_q = d / W;
+  pl.cols_rem = d % W;
+  pl.max_cols = pl.cols_q + (pl.cols_rem ? 1 : 0);
+  // up: x resident, the rest of the budget is the ring
+  const int up_base = up_layout(d, E, pl.NT, L, 0).total;
+  const int down_base = down_layout(d_e, E, pl.NT, L, 0, pl.max_cols).total;
+  const int slot_dn = L * 2 * d_e + pl.max_cols * 2 * d_e;
+  // Paired: both kernels fit one SM together when x plus a modest ring fit half of it.
+  const bool paired = up_base + 12 * 2 * d <= kSmemHalf && down_base + 4 * slot_dn <= kSmemHalf;
+  const int budget = paired ? kSmemHalf : kSmemMax;
+  pl.ring_rows = (budget - up_base) / (2 * d);
+  if (want_up && want_up < pl.ring_rows) pl.ring_rows = want_up;
+  if (pl.ring_rows > 96) pl.ring_rows = 96;
+  if (pl.ring_rows < kUpStages) return pl;
+  pl.ns_down = (budget - down_base - 128) / slot_dn;
+  if (want_down) pl.ns_down = want_down;
+  if (pl.ns_down > kMaxStages) pl.ns_down = kMaxStages;
+  if (pl.ns_down > E) pl.ns_down = E < 2 ? 2 : E;
+  if (pl.ns_down < 2) return pl;
+  if (pl.ns_down < E) pl.ns_down &= ~1;   // halves when the union does not fit at once
+  pl.smem_up = up_layout(d, E, pl.NT, L, pl.ring_rows).total;
+  pl.smem_down = down_layout(d_e, E, pl.NT, L, pl.ns_down, pl.max_cols).total;
+  if (pl.smem_up > kSmemMax || pl.smem_down > kSmemMax) return pl;
   pl.ok = true;
   return pl;
 }
 
+// Both kernels ask for the largest shared-memory carve-out: an SM keeps its carve-out while
+// any CTA runs on it, so a down CTA can only join an up CTA (and the next call's up CTA the
+// down CTA) if the first of them already configured the SM for both.
 template <int NT>
 cudaError_t set_attrs() {
-  cudaError_t e = cudaFuncSetAttribute(expert_up_mma_kernel<NT>,
-                                       cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemMax);
-  if (e != cudaSuccess) return e;
-  return cudaFuncSetAttribute(expert_down_mma_kernel<NT>,
-                              cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemMax);
+  const void* fns[2] = {reinterpret_cast<const void*>(&expert_up_mma_kernel<NT>),
+                        reinterpret_cast<const void*>(&expert_down_mma_kernel<NT>)};
+  for (const void* f : fns) {
+    cudaError_t e = cudaFuncSetAttribute(f, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemMax);
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(f, cudaFuncAttributePreferredSharedMemoryCarveout,
+                             cudaSharedmemCarveoutMaxShared);
+    if (e != cudaSuccess) return e;
+  }
+  return cudaSuccess;
 }
 
 template <int NT>
 cudaError_t launch_nt(const MmaPlan& pl, int grid, const UpParams& up, const DownParams& dn,
-                      cudaStream_t st) {
+                      bool chained, cudaStream_t st) {
   cudaLaunchAttribute attr[1];
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[0].val.programmaticStreamSerializationAllowed = 1;
@@ -597,7 +709,7 @@ cudaError_t launch_nt(const MmaPlan& pl, int grid, const UpParams& up, const Dow
   lc.blockDim = dim3(kThreads);
   lc.stream = st;
   lc.attrs = attr;
-  lc.numAttrs = 1;
+  lc.numAttrs = chained ? 1 : 0;
   lc.dynamicSmemBytes = pl.smem_up;
   cudaError_t e = cudaLaunchKernelEx(&lc, expert_up_mma_kernel<NT>, up);
   if (e != cudaSuccess) return e;
@@ -607,10 +719,12 @@ cudaError_t launch_nt(const MmaPlan& pl, int grid, const UpParams& up, const Dow
 
 }  // namespace
 
-bool expert_mma_supported(const blockffn_ctx* c, int L) { return make_plan(c->cfg, L).ok; }
+bool expert_mma_supported(const blockffn_ctx* c, int L) {
+  return make_plan(c->cfg, L, c->num_sms).ok;
+}
 
 size_t expert_mma_h_bytes(const blockffn_config* cfg) {
-  return sizeof(uint16_t) * (size_t)cfg->E * cfg->L_max * (cfg->d_e + 32) + 256;
+  return sizeof(uint16_t) * (size_t)cfg->E * cfg->L_max * cfg->d_e + 256;
 }
 
 cudaError_t expert_mma_setup(blockffn_ctx*) {
@@ -625,7 +739,7 @@ cudaError_t launch_expert_mma(blockffn_ctx* c, const blockffn_weights* w, const 
                               const float* scores, int L, const int32_t* union_ids,
                               const int32_t* n_union, float* out, void* x_next, int call_flags,
                               const RoutingOut* pub, cudaStream_t st) {
-  const MmaPlan pl = make_plan(c->cfg, L);
+  const MmaPlan pl = make_plan(c->cfg, L, c->num_sms);
   if (!pl.ok) return cudaErrorNotSupported;
   UpParams up{};
   up.x = static_cast<const uint16_t*>(x);
@@ -638,7 +752,8 @@ cudaError_t launch_expert_mma(blockffn_ctx* c, const blockffn_weights* w, const 
   up.d = c->cfg.d;
   up.E = c->cfg.E;
   up.d_e = c->cfg.d_e;
-  up.ns = pl.ns_up;
+  up.ring_rows = pl.ring_rows;
+  up.de_shift = (c->cfg.d_e & (c->cfg.d_e - 1)) == 0 ? __builtin_ctz(c->cfg.d_e) : -1;
   up.early = (call_flags & BLOCKFFN_CALL_INDEPENDENT) ? 1 : 0;
   up.status = c->status;
   if (pub) {
@@ -660,14 +775,19 @@ cudaError_t launch_expert_mma(blockffn_ctx* c, const blockffn_weights* w, const 
   dn.E = c->cfg.E;
   dn.d_e = c->cfg.d_e;
   dn.ns = pl.ns_down;
+  dn.max_cols = pl.max_cols;
+  dn.per = pl.per;
+  dn.cols_q = pl.cols_q;
+  dn.cols_rem = pl.cols_rem;
   dn.accumulate = (call_flags & BLOCKFFN_CALL_ACCUMULATE) ? 1 : 0;
   dn.status = c->status;
+  const bool chained = !(c->cfg.flags & BLOCKFFN_CFG_NO_CHAINING);
   cudaError_t e;
   switch (pl.NT) {
-    case 1: e = launch_nt<1>(pl, c->num_sms, up, dn, st); break;
-    case 2: e = launch_nt<2>(pl, c->num_sms, up, dn, st); break;
-    case 3: e = launch_nt<3>(pl, c->num_sms, up, dn, st); break;
-    default: e = launch_nt<4>(pl, c->num_sms, up, dn, st); break;
+    case 1: e = launch_nt<1>(pl, c->num_sms, up, dn, chained, st); break;
+    case 2: e = launch_nt<2>(pl, c->num_sms, up, dn, chained, st); break;
+    case 3: e = launch_nt<3>(pl, c->num_sms, up, dn, chained, st); break;
+    default: e = launch_nt<4>(pl, c->num_sms, up, dn, chained, st); break;
   }
   if (e == cudaSuccess) c->launches += 2;
   return e;
