@@ -46,6 +46,7 @@ constexpr int kMaxStages = 32;                   // slots of the down kernel's r
 constexpr int kUpStages = 3;                     // slots of the up kernel's ring
 constexpr int kSmemMax = 232448;                 // 227 KB per CTA
 constexpr int kSmemHalf = 113 * 1024;            // lets an up and a down CTA share one SM
+// (registers too: for L <= 16 the kernels are compiled for two CTAs per SM, 128 per thread)
 
 // ---- shared-memory layout ----------------------------------------------------
 __host__ __device__ inline int align128(int v) { return (v + 127) & ~127; }
@@ -296,7 +297,7 @@ struct UpParams {
 };
 
 template <int NT>
-__global__ void __launch_bounds__(kThreads, 1) expert_up_mma_kernel(const UpParams p) {
+__global__ void __launch_bounds__(kThreads, NT <= 2 ? 2 : 1) expert_up_mma_kernel(const UpParams p) {
   extern __shared__ __align__(128) unsigned char smem[];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int d = p.d, d_e = p.d_e, L = p.L;
@@ -480,7 +481,7 @@ struct DownParams {
 };
 
 template <int NT>
-__global__ void __launch_bounds__(kThreads, 1) expert_down_mma_kernel(const DownParams p) {
+__global__ void __launch_bounds__(kThreads, NT <= 2 ? 2 : 1) expert_down_mma_kernel(const DownParams p) {
   extern __shared__ __align__(128) unsigned char smem[];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int d = p.d, d_e = p.d_e, L = p.L, per = p.per;
@@ -673,7 +674,6 @@ MmaPlan make_plan(const blockffn_config& cfg, int L, int grid) {
   if (pl.ns_down > kMaxStages) pl.ns_down = kMaxStages;
   if (pl.ns_down > E) pl.ns_down = E < 2 ? 2 : E;
   if (pl.ns_down < 2) return pl;
-  if (pl.ns_down < E) pl.ns_down &= ~1;   // halves when the union does not fit at once
   pl.smem_up = up_layout(d, E, pl.NT, L, pl.ring_rows).total;
   pl.smem_down = down_layout(d_e, E, pl.NT, L, pl.ns_down, pl.max_cols).total;
   if (pl.smem_up > kSmemMax || pl.smem_down > kSmemMax) return pl;
