@@ -179,6 +179,37 @@ BLOCKFFN_API double blockffn_cls(const blockffn_stats* host_stats, int32_t E);
 /* Number of kernels the library has launched through this handle (host counter). */
 BLOCKFFN_API uint64_t blockffn_launch_count(blockffn_handle h);
 
+/* Largest fp32 intermediate blockffn_expert_ffn_noalloc can hold: E * L * d_e * 4 bytes of a
+ * call must not exceed it (1 MiB: E = 64, d_e = 128 up to L = 32). */
+#define BLOCKFFN_NOALLOC_SCRATCH_BYTES (1 << 20)
+
+/* The paper has no counterpart of this entry point; it exists for deployment reasons only.
+ * It is blockffn_expert_ffn (Eq. 1 + Eq. 2 over the listed experts, same arguments, same
+ * result as the CUDA-core variant) for callers that are not allowed to allocate device
+ * memory and therefore cannot call blockffn_create, whose workspace comes from cudaMalloc:
+ * for instance a plug-in that runs inside a host application which has handed all device
+ * memory to its own pool (an allocation would fail, or would stall every stream of the
+ * process while the driver maps it), or code on a latency-critical path where an
+ * allocator call is forbidden by policy. It takes the shape in a blockffn_config
+ * (d, E, d_e, rms_eps unused; L_max, variant and flags are ignored) instead of a handle and
+ * makes no call that allocates or frees memory.
+ *   - Its intermediate lives in a fixed array inside the library image, which every GPU that
+ *     loads the library keeps until the process exits: BLOCKFFN_NOALLOC_SCRATCH_BYTES plus a
+ *     256-byte header. A call whose E * L * d_e * 4 exceeds that size returns
+ *     BLOCKFFN_ERR_WORKSPACE and enqueues nothing.
+ *   - The first call on a device looks up the array's device address (with that device
+ *     current) and caches it; make that first call outside any stream capture.
+ *   - All calls on a device share the one array. Calls enqueued on the same stream are safe;
+ *     two calls that may run on the GPU at the same time (different streams, or graph
+ *     branches) race on it and give wrong results. Nothing in the array carries over from
+ *     one call to the next: the part a call reads is rewritten by that call first.
+ *   - Out-of-range union entries are skipped as in blockffn_expert_ffn but are not reported:
+ *     there is no handle whose status word could be read.                                  */
+BLOCKFFN_API blockffn_status blockffn_expert_ffn_noalloc(
+    const blockffn_config* cfg, const blockffn_weights* w, const void* x, const float* scores,
+    int32_t L, const int32_t* union_ids, const int32_t* n_union, float* out, void* x_next,
+    int32_t call_flags, void* stream);
+
 /* Human-readable name of a status code (static storage). */
 BLOCKFFN_API const char* blockffn_status_string(blockffn_status s);
 

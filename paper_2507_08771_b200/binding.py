@@ -28,8 +28,9 @@ EXPORTS = [
     "blockffn_create", "blockffn_destroy", "blockffn_router", "blockffn_chunk_union",
     "blockffn_expert_ffn", "blockffn_layer_forward", "blockffn_layer_forward_scores",
     "blockffn_read_routing", "blockffn_last_status", "blockffn_tls", "blockffn_cls",
-    "blockffn_launch_count", "blockffn_status_string",
+    "blockffn_launch_count", "blockffn_status_string", "blockffn_expert_ffn_noalloc",
 ]
+NOALLOC_SCRATCH_BYTES = 1 << 20
 
 
 class Config(ctypes.Structure):
@@ -74,6 +75,8 @@ def load():
     lib.blockffn_layer_forward_scores.argtypes = [vp, ctypes.POINTER(Weights), vp, vp, i32, vp, vp,
                                                   vp, i32, vp]
     lib.blockffn_read_routing.argtypes = [vp, i32, vp, vp, vp, vp, vp, vp]
+    lib.blockffn_expert_ffn_noalloc.argtypes = [ctypes.POINTER(Config), ctypes.POINTER(Weights), vp,
+                                                vp, i32, vp, vp, vp, vp, i32, vp]
     lib.blockffn_last_status.argtypes = [vp, ctypes.POINTER(ctypes.c_uint32), i32, vp]
     lib.blockffn_tls.argtypes = [ctypes.POINTER(Stats), i32]
     lib.blockffn_tls.restype = ctypes.c_double
@@ -146,6 +149,16 @@ def blockffn_expert_ffn(h, w: Weights, x, scores, L, union_ids, n_union, out, x_
     _check(load().blockffn_expert_ffn(h, ctypes.byref(w), _ptr(x), _ptr(scores), L,
                                       _ptr(union_ids), _ptr(n_union), _ptr(out), _ptr(x_next),
                                       call_flags, _stream(stream)), "blockffn_expert_ffn")
+
+
+def blockffn_expert_ffn_noalloc(cfg: Config, w: Weights, x, scores, L, union_ids, n_union, out,
+                                x_next=None, call_flags=0, stream=None):
+    """Expert stage for callers that may not allocate device memory: no handle, the
+    intermediate lives in a fixed array inside the library (see the header for its limits)."""
+    _check(load().blockffn_expert_ffn_noalloc(ctypes.byref(cfg), ctypes.byref(w), _ptr(x),
+                                              _ptr(scores), L, _ptr(union_ids), _ptr(n_union),
+                                              _ptr(out), _ptr(x_next), call_flags,
+                                              _stream(stream)), "blockffn_expert_ffn_noalloc")
 
 
 def blockffn_layer_forward(h, w: Weights, x, L, out, x_next=None, stats=None, call_flags=0,

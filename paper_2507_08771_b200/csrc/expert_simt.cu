@@ -183,3 +183,73 @@ cudaError_t launch_expert_simt(blockffn_ctx* c, const blockffn_weights* w, const
   if (L <= 4) return launch_lt<4>(c, w, x, scores, L, union_ids, n_union, out, x_next, call_flags, st);
   return launch_lt<8>(c, w, x, scores, L, union_ids, n_union, out, x_next, call_flags, st);
 }
+
+// ---- expert stage without a handle and without any allocation ---------------------------
+//
+// Scratch for blockffn_expert_ffn_noalloc: the fp32 intermediate h[q][t][j] of the two
+// CUDA-core kernels above, preceded by a 256-byte header whose first word is the status word
+// those kernels want. The array is part of the library image: every GPU that loads the
+// library holds these bytes until the process exits.
+#define BLOCKFFN_NOALLOC_HEADER 256
+static __device__ __align__(256) unsigned char
+    g_noalloc_scratch[BLOCKFFN_NOALLOC_HEADER + BLOCKFFN_NOALLOC_SCRATCH_BYTES];
+
+namespace {
+constexpr int kMaxDevices = 64;
+// Device address of g_noalloc_scratch per device, looked up once per device. In host code
+// the array's name is only a handle for the runtime, never an address a kernel may be given.
+unsigned char* g_noalloc_ptr[kMaxDevices] = {};
+int g_noalloc_sms[kMaxDevices] = {};
+}  // namespace
+
+extern "C" blockffn_status blockffn_expert_ffn_noalloc(
+    const blockffn_config* cfg, const blockffn_weights* w, const void* x, const float* scores,
+    int32_t L, const int32_t* union_ids, const int32_t* n_union, float* out, void* x_next,
+    int32_t call_flags, void* stream) {
+  auto bad16 = [](const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) != 0; };
+  auto bad4 = [](const void* p) { return (reinterpret_cast<uintptr_t>(p) & 3u) != 0; };
+  if (!cfg || !w || !w->U || !w->D || !x || !scores || !union_ids || !n_union || !out)
+    return BLOCKFFN_ERR_INVALID_ARG;
+  if (cfg->d < 8 || cfg->d_e < 8 || cfg->E < 1 || L < 1) return BLOCKFFN_ERR_INVALID_ARG;
+  if (cfg->d % 8 || cfg->d_e % 8 || cfg->E > 1024 || L > 32 || cfg->d > (1 << 20) ||
+      cfg->d_e > (1 << 16))
+    return BLOCKFFN_ERR_UNSUPPORTED;
+  // the intermediate of this call must fit the fixed scratch
+  if ((size_t)cfg->E * (size_t)L * (size_t)cfg->d_e * sizeof(float) >
+      (size_t)BLOCKFFN_NOALLOC_SCRATCH_BYTES)
+    return BLOCKFFN_ERR_WORKSPACE;
+  if (bad16(w->U) || bad16(w->D) || bad16(x) || bad16(out) || bad16(x_next) || bad4(scores) ||
+      bad4(union_ids) || bad4(n_union) || x_next == x)
+    return BLOCKFFN_ERR_INVALID_ARG;
+  if (call_flags & ~(BLOCKFFN_CALL_ACCUMULATE | BLOCKFFN_CALL_INDEPENDENT))
+    return BLOCKFFN_ERR_INVALID_ARG;
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return BLOCKFFN_ERR_CUDA;
+  if (!g_noalloc_ptr[dev]) {   // first call on this device, with this device current
+    unsigned char* ptr = nullptr;
+    int sms = 0;
+    if (cudaGetSymbolAddress(reinterpret_cast<void**>(&ptr), g_noalloc_scratch) != cudaSuccess ||
+        !ptr ||
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) {
+      cudaGetLastError();
+      return BLOCKFFN_ERR_CUDA;
+    }
+    g_noalloc_sms[dev] = sms;
+    g_noalloc_ptr[dev] = ptr;
+  }
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  // The status word is shared by all calls and keeps its last value: start it at zero.
+  if (cudaMemsetAsync(g_noalloc_ptr[dev], 0, BLOCKFFN_NOALLOC_HEADER, st) != cudaSuccess)
+    return BLOCKFFN_ERR_CUDA;
+  blockffn_ctx tmp{};          // a view for the launcher: nothing in it owns memory
+  tmp.cfg = *cfg;
+  tmp.cfg.L_max = L;           // h is laid out [q][L][d_e]
+  tmp.device = dev;
+  tmp.num_sms = g_noalloc_sms[dev];
+  tmp.words = (cfg->E + 31) / 32;
+  tmp.status = reinterpret_cast<uint32_t*>(g_noalloc_ptr[dev]);
+  tmp.h32 = reinterpret_cast<float*>(g_noalloc_ptr[dev] + BLOCKFFN_NOALLOC_HEADER);
+  const cudaError_t e =
+      launch_expert_simt(&tmp, w, x, scores, L, union_ids, n_union, out, x_next, call_flags, st);
+  return e == cudaSuccess ? BLOCKFFN_OK : BLOCKFFN_ERR_CUDA;
+}
