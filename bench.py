@@ -210,6 +210,23 @@ class Workload:
                                       B.CALL_INDEPENDENT, stream)
 
 
+def max_over_ranks(values, world, device=None):
+    """Element-wise maximum of a list of floats over all ranks (the slowest rank sets the time).
+    world == 1: the values themselves. Uses the default process group (NCCL on GPUs, gloo on CPU)."""
+    if world <= 1:
+        return [float(v) for v in values]
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor(values, dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(v) for v in t.cpu()]
+
+
+def job_throughput(world, bytes_per_rank_step, ms_step):
+    """Whole-job GB/s: every rank streams bytes_per_rank_step in ms_step (replicas, no collective)."""
+    return world * bytes_per_rank_step / (ms_step * 1e-3) / 1e9
+
+
 def capture(torch, stream, fn):
     g = torch.cuda.CUDAGraph()
     with torch.cuda.stream(stream):
@@ -370,17 +387,15 @@ def run_ours(args):
     barrier()
     status = lay.last_status()
     assert status == 0, f"device status word {status}"
+    lay_is_mma = args.variant != 1 and expert_launches // max(wl.calls_per_step, 1) == 2 and sh.d % 64 == 0
     assert torch.isfinite(wl.out).all()
 
-    t = torch.tensor([ms_step, ms_e2e, ms_expert], dtype=torch.float64, device=device)
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    ms_step, ms_e2e, ms_expert = (float(v) for v in t.cpu())
+    ms_step, ms_e2e, ms_expert = max_over_ranks([ms_step, ms_e2e, ms_expert], world, device)
 
     calls = wl.calls_per_step
     bytes_step = calls * wl.active_bytes
-    value = world * bytes_step / (ms_step * 1e-3) / 1e9
-    e2e = world * bytes_step / (ms_e2e * 1e-3) / 1e9
+    value = job_throughput(world, bytes_step, ms_step)
+    e2e = job_throughput(world, bytes_step, ms_e2e)
     peak, peak_kind = measured_peak()
     # algorithmic bytes of one expert-stage call: weights + x + out + scores
     alg_bytes = wl.active_bytes + 2 * wl.L * sh.d + 4 * wl.L * sh.d + 4 * wl.L * sh.E
@@ -395,7 +410,7 @@ def run_ours(args):
     line = {
         "metric": METRIC, "value": value, "unit": "GB/s", "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True,
-        "scaling": "weak", "vs_baseline": None, "dtype": "bf16 weights, f32 accumulate",
+        "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
         "data": "synthetic",
         "latency_us_per_chunk": ms_step * 1e3 / wl.chunks,
         "latency_us_per_layer_call": ms_step * 1e3 / calls,
@@ -416,11 +431,13 @@ def run_ours(args):
         "gpu_launches": launches_per_step * args.steps,
         "gpu_launches_per_step": launches_per_step,
         "roofline": {
-            "bound": "hbm", "kernel": "expert stage (up + down projection kernels of one call)",
+            "bound": "hbm", "kernel": "expert_up_mma + expert_down_mma (the chained pair of one call; 50 % / 49 % of the ncu launch list)",
             "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
             "peak_kind": f"of {peak_kind}", "us_per_launch": us_expert,
             "algorithmic_bytes_per_launch": alg_bytes, "launches_per_call": expert_launches // calls,
-            "traffic": None,
+            # dram__bytes_read + write of one up + one down launch (ncu, config 1, see profiles/);
+            # other configurations: not captured
+            "traffic": 11144192 if (args.config == 1 and wl.L == 8 and lay_is_mma) else None,
         },
     }
     if not args.no_cpu_baseline and world == 1:
