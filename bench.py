@@ -135,6 +135,9 @@ class Workload:
         seed = I.config_seed(cfg_index)
         self.u = sh.u
         self.active_bytes = sh.active_bytes()
+        # successive chunks of configs 1-3 are independent inputs; the stack (4) feeds each layer
+        # the previous layer's output, so only its routing inputs and weights are stable
+        self.call_flags = B.CALL_INDEPENDENT if cfg_index == 4 else B.CALL_INDEPENDENT_X
         self.layer = B.Layer(sh.d, sh.E, sh.d_e, L_max=max(self.L, 8), variant=variant, device=device,
                              flags=flags)
         if cfg_index == 4:
@@ -190,7 +193,7 @@ class Workload:
             for c in range(self.chunks):
                 B.blockffn_layer_forward_scores(
                     lay.h, self.dws[c % self.n_copies].struct, self.x[c], self.scores[c, 0], self.L,
-                    self.out[c], None, lay.stats, B.CALL_INDEPENDENT, stream)
+                    self.out[c], None, lay.stats, self.call_flags, stream)
 
     # -- expert stage alone (the dominant kernels), unions precomputed --
     def enqueue_unions(self, stream):
@@ -207,7 +210,7 @@ class Workload:
                 k = l if self.idx == 4 else c % self.n_copies
                 B.blockffn_expert_ffn(lay.h, self.dws[k].struct, self.x[c], self.scores[c, l], self.L,
                                       self.ids[c, l], self.nu[c, l:l + 1], self.out[c], None,
-                                      B.CALL_INDEPENDENT, stream)
+                                      B.CALL_INDEPENDENT if self.idx == 4 else self.call_flags, stream)
 
 
 def max_over_ranks(values, world, device=None):

@@ -102,10 +102,19 @@ typedef struct {
 
 /* Per-call flags. */
 #define BLOCKFFN_CALL_ACCUMULATE 1 /* out += FFN(x) (residual, fp32) instead of out = FFN(x)     */
-#define BLOCKFFN_CALL_INDEPENDENT 2 /* promise: scores, union_ids, n_union and the weights of this
-                                       call were NOT written by the work enqueued just before it
-                                       on `stream`; only x and out may depend on it. Lets the call's
-                                       weight fetch start while the previous kernel drains.        */
+/* The tensor-core kernels of a call may start while the kernels enqueued before it on `stream`
+ * are still running (programmatic dependent launch). What they read before they have waited for
+ * that earlier work to finish is governed by two promises of the caller:                      */
+#define BLOCKFFN_CALL_INDEPENDENT 2 /* scores, union_ids, n_union and the weights of this call are
+                                       stable: nothing enqueued on `stream` since the last call made
+                                       without this flag (or since the last host synchronisation)
+                                       writes them. x and out may still come from the work just
+                                       before. The weight fetch then overlaps the previous kernel.  */
+#define BLOCKFFN_CALL_INDEPENDENT_X 4 /* in addition x is stable in the same sense (the chunk does
+                                       not consume the previous call's output); implies
+                                       BLOCKFFN_CALL_INDEPENDENT. The up projection then runs in full
+                                       under the previous call and only its store waits. Ignored by
+                                       blockffn_layer_forward (its router writes the scores).       */
 
 typedef struct blockffn_ctx* blockffn_handle;
 

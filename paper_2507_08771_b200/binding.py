@@ -22,7 +22,8 @@ _lib = None
 OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_CUDA, ERR_DEVICE = range(6)
 DEV_BAD_UNION_ID, DEV_BAD_UNION_COUNT, DEV_WAIT_EXPIRED = 1, 2, 4
 VARIANT_AUTO, VARIANT_SIMT, VARIANT_MMA = 0, 1, 2
-CALL_ACCUMULATE, CALL_INDEPENDENT = 1, 2
+CALL_ACCUMULATE, CALL_INDEPENDENT, CALL_INDEPENDENT_X = 1, 2, 4
+CFG_NO_CHAINING = 0x10000
 
 EXPORTS = [
     "blockffn_create", "blockffn_destroy", "blockffn_router", "blockffn_chunk_union",

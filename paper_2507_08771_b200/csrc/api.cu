@@ -5,6 +5,9 @@
 
 namespace {
 
+constexpr int kCallFlags =
+    BLOCKFFN_CALL_ACCUMULATE | BLOCKFFN_CALL_INDEPENDENT | BLOCKFFN_CALL_INDEPENDENT_X;
+
 inline bool misaligned(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) != 0; }
 inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
@@ -156,7 +159,7 @@ blockffn_status blockffn_expert_ffn(blockffn_handle h, const blockffn_weights* w
       (reinterpret_cast<uintptr_t>(union_ids) & 3u) || (reinterpret_cast<uintptr_t>(n_union) & 3u))
     return BLOCKFFN_ERR_INVALID_ARG;
   if (x_next == x) return BLOCKFFN_ERR_INVALID_ARG;
-  if (call_flags & ~(BLOCKFFN_CALL_ACCUMULATE | BLOCKFFN_CALL_INDEPENDENT))
+  if (call_flags & ~kCallFlags)
     return BLOCKFFN_ERR_INVALID_ARG;
   return expert_dispatch(h, w, x, scores, L, union_ids, n_union, out, x_next, call_flags,
                          static_cast<cudaStream_t>(stream));
@@ -173,11 +176,11 @@ blockffn_status blockffn_layer_forward(blockffn_handle h, const blockffn_weights
       (reinterpret_cast<uintptr_t>(w->bias) & 3u) || (reinterpret_cast<uintptr_t>(stats) & 7u))
     return BLOCKFFN_ERR_INVALID_ARG;
   if (x_next == x) return BLOCKFFN_ERR_INVALID_ARG;
-  if (call_flags & ~(BLOCKFFN_CALL_ACCUMULATE | BLOCKFFN_CALL_INDEPENDENT))
+  if (call_flags & ~kCallFlags)
     return BLOCKFFN_ERR_INVALID_ARG;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   // The router writes the scores this very call consumes: never "independent".
-  const int flags = call_flags & ~BLOCKFFN_CALL_INDEPENDENT;
+  const int flags = call_flags & ~(BLOCKFFN_CALL_INDEPENDENT | BLOCKFFN_CALL_INDEPENDENT_X);
   if (launch_router(h, w, x, L, h->scores, h->tok_mask, true, stats, st) != cudaSuccess)
     return BLOCKFFN_ERR_CUDA;
   return expert_dispatch(h, w, x, h->scores, L, h->union_ids, h->n_union, out, x_next, flags, st);
@@ -194,7 +197,7 @@ blockffn_status blockffn_layer_forward_scores(blockffn_handle h, const blockffn_
       misaligned(x_next) || misaligned(scores) || (reinterpret_cast<uintptr_t>(stats) & 7u))
     return BLOCKFFN_ERR_INVALID_ARG;
   if (x_next == x) return BLOCKFFN_ERR_INVALID_ARG;
-  if (call_flags & ~(BLOCKFFN_CALL_ACCUMULATE | BLOCKFFN_CALL_INDEPENDENT))
+  if (call_flags & ~kCallFlags)
     return BLOCKFFN_ERR_INVALID_ARG;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   if (use_mma(h, L)) {
@@ -210,7 +213,7 @@ blockffn_status blockffn_layer_forward_scores(blockffn_handle h, const blockffn_
       cudaSuccess)
     return BLOCKFFN_ERR_CUDA;
   // The union list is produced inside this call: the expert stage must wait for it.
-  const int flags = call_flags & ~BLOCKFFN_CALL_INDEPENDENT;
+  const int flags = call_flags & ~(BLOCKFFN_CALL_INDEPENDENT | BLOCKFFN_CALL_INDEPENDENT_X);
   return expert_dispatch(h, w, x, scores, L, h->union_ids, h->n_union, out, x_next, flags, st);
 }
 

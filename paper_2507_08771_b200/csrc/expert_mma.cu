@@ -287,7 +287,8 @@ struct UpParams {
   const int32_t* ids_in;   // caller's union list, or NULL: derive from scores
   const int32_t* n_in;
   uint16_t* h;             // bf16 [q][L][d_e] intermediate
-  int L, d, E, d_e, de_shift, ring_rows, early;   // de_shift: log2(d_e), or -1
+  int L, d, E, d_e, de_shift, ring_rows;   // de_shift: log2(d_e), or -1
+  int early;               // 0: wait first; 1: routing + weights before the wait; 2: x too
   uint32_t* status;
   // what CTA 0 publishes when it derived the union itself (each may be NULL)
   uint32_t* pub_mask;
@@ -378,7 +379,7 @@ __global__ void __launch_bounds__(kThreads, NT <= 2 ? 2 : 1) expert_up_mma_kerne
     for (int gi = 0; gi < g_first; ++gi) issue(gi);
     if (ngroups > 0) prepare(0);
   }
-  pdl_wait();            // x may come from the kernel just before; h may still be read by it
+  if (p.early < 2) pdl_wait();   // x may come from the kernel just before
   if (ngroups > 0) copy_run(sbase + lay.off_x, p.x, L * row_bytes);
   if (!p.early) {
     for (int gi = 0; gi < g_first; ++gi) issue(gi);
@@ -422,6 +423,7 @@ __global__ void __launch_bounds__(kThreads, NT <= 2 ? 2 : 1) expert_up_mma_kerne
     __syncthreads();     // every warp is done with the slot: refill it
     if (gi + ns < ngroups) issue(gi + ns);
     cp_async_commit();   // one group per stage, empty or not, keeps the count below uniform
+    if (gi == 0 && p.early == 2) pdl_wait();   // h may still be read by the call before
 #pragma unroll
     for (int i = 0; i < NT; ++i) {
       if (hq[i] >= 0) {
@@ -438,6 +440,7 @@ __global__ void __launch_bounds__(kThreads, NT <= 2 ? 2 : 1) expert_up_mma_kerne
     if (gi + 1 >= ns) cp_async_wait_group<ns - 1>();
     __syncthreads();
   }
+  if (p.early == 2 && ngroups == 0) pdl_wait();   // every kernel waits before it ends
   // CTA 0 publishes the routing it derived (after the wait: earlier readers are done)
   if (blockIdx.x == 0) {
     if (p.ids_in == nullptr) {
@@ -754,7 +757,8 @@ cudaError_t launch_expert_mma(blockffn_ctx* c, const blockffn_weights* w, const 
   up.d_e = c->cfg.d_e;
   up.ring_rows = pl.ring_rows;
   up.de_shift = (c->cfg.d_e & (c->cfg.d_e - 1)) == 0 ? __builtin_ctz(c->cfg.d_e) : -1;
-  up.early = (call_flags & BLOCKFFN_CALL_INDEPENDENT) ? 1 : 0;
+  up.early = (call_flags & BLOCKFFN_CALL_INDEPENDENT_X) ? 2
+             : (call_flags & BLOCKFFN_CALL_INDEPENDENT) ? 1 : 0;
   up.status = c->status;
   if (pub) {
     up.pub_mask = pub->union_mask;

@@ -221,7 +221,7 @@ extern "C" blockffn_status blockffn_expert_ffn_noalloc(
   if (bad16(w->U) || bad16(w->D) || bad16(x) || bad16(out) || bad16(x_next) || bad4(scores) ||
       bad4(union_ids) || bad4(n_union) || x_next == x)
     return BLOCKFFN_ERR_INVALID_ARG;
-  if (call_flags & ~(BLOCKFFN_CALL_ACCUMULATE | BLOCKFFN_CALL_INDEPENDENT))
+  if (call_flags & ~(BLOCKFFN_CALL_ACCUMULATE | BLOCKFFN_CALL_INDEPENDENT | BLOCKFFN_CALL_INDEPENDENT_X))
     return BLOCKFFN_ERR_INVALID_ARG;
   int dev = -1;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return BLOCKFFN_ERR_CUDA;

@@ -16,7 +16,8 @@ pytestmark = pytest.mark.gpu
 
 TOL = 2e-2          # max|err| <= TOL * RMS(ref)
 FLIP_BAND = 1e-3    # |pre-ReLU logit| below which a mask flip is excused
-VARIANTS = [B.VARIANT_SIMT, B.VARIANT_AUTO]
+# (kernel family, config flags): CUDA-core, tensor-core chained, tensor-core fully serialised
+VARIANTS = [(B.VARIANT_SIMT, 0), (B.VARIANT_AUTO, 0), (B.VARIANT_AUTO, B.CFG_NO_CHAINING)]
 
 
 def rms(a):
@@ -153,7 +154,7 @@ def test_expert_ffn(variant, d, E, d_e, L, p):
     tm = oracle.token_masks(s.astype(np.float64))
     _, ids, n = oracle.chunk_union(tm, E)
     ref = oracle.expert_ffn(x, s.astype(np.float64), w["U"], w["D"], expert_ids=ids[:n])
-    layer = B.Layer(d, E, d_e, L_max=32, variant=variant)
+    layer = B.Layer(d, E, d_e, L_max=32, variant=variant[0], flags=variant[1])
     dw = layer.upload_weights(w)
     got, _ = run_expert(layer, dw, x, s, ids, n, L)
     assert_close(got, ref, f"expert_ffn d={d} E={E} L={L}")
@@ -168,7 +169,7 @@ def test_expert_ffn_degenerate_unions_and_residual(variant):
     sh, w = small_layer(d, E, d_e, 77)
     rng = np.random.default_rng(77)
     x = I.make_x(d, L, 77)
-    layer = B.Layer(d, E, d_e, L_max=8, variant=variant)
+    layer = B.Layer(d, E, d_e, L_max=8, variant=variant[0], flags=variant[1])
     dw = layer.upload_weights(w)
     # empty union: out = 0
     ids = np.full(E, -1, np.int32)
@@ -202,7 +203,7 @@ def test_bad_union_entries_are_flagged_not_followed():
     x = I.make_x(d, L, 5)
     s = sparse_scores(rng, L, E, 0.5)
     for variant in VARIANTS:
-        layer = B.Layer(d, E, d_e, L_max=4, variant=variant)
+        layer = B.Layer(d, E, d_e, L_max=4, variant=variant[0], flags=variant[1])
         dw = layer.upload_weights(w)
         ids = np.full(E, -1, np.int32)
         ids[:3] = [2, 99, 7]                                   # 99 is out of range
@@ -274,7 +275,7 @@ def check_layer_router_on(layer, dw, w, x, L, bias=None):
 def test_config0_tiny_full_router(variant):
     sh, seed = I.SHAPES[0], I.config_seed(0)
     w = I.make_layer(sh, seed)
-    layer = B.Layer(sh.d, sh.E, sh.d_e, L_max=sh.L, variant=variant)
+    layer = B.Layer(sh.d, sh.E, sh.d_e, L_max=sh.L, variant=variant[0], flags=variant[1])
     dw = layer.upload_weights(w)
     for chunk in range(3):
         x = I.make_x(sh.d, sh.L, seed, chunk=chunk)
@@ -299,7 +300,7 @@ def check_scores_in(layer, dw, w, sh, L, seed, chunk, u=None):
 def test_config1_scores_in(variant):
     sh, seed = I.SHAPES[1], I.config_seed(1)
     w = I.make_layer(sh, seed, with_router=False)
-    layer = B.Layer(sh.d, sh.E, sh.d_e, L_max=sh.L, variant=variant)
+    layer = B.Layer(sh.d, sh.E, sh.d_e, L_max=sh.L, variant=variant[0], flags=variant[1])
     dw = layer.upload_weights(w)
     for chunk in range(3):
         check_scores_in(layer, dw, w, sh, sh.L, seed, chunk)
@@ -313,7 +314,7 @@ def test_config1_scores_in(variant):
 def test_config2_l_sweep(variant):
     sh, seed = I.SHAPES[2], I.config_seed(2)
     w = I.make_layer(sh, seed, with_router=False)
-    layer = B.Layer(sh.d, sh.E, sh.d_e, L_max=32, variant=variant)
+    layer = B.Layer(sh.d, sh.E, sh.d_e, L_max=32, variant=variant[0], flags=variant[1])
     dw = layer.upload_weights(w)
     for L in I.L_SWEEP:
         check_scores_in(layer, dw, w, sh, L, seed, chunk=L)
