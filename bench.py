@@ -47,7 +47,9 @@ def parse():
     p.add_argument("--flags", type=lambda v: int(v, 0), default=0,
                    help="blockffn_config.flags (ring depths, BLOCKFFN_CFG_* bits)")
     p.add_argument("--no-cpu-baseline", action="store_true")
-    p.add_argument("--sweep", action="store_true", help="also report every L of the sweep (config 2)")
+    p.add_argument("--no-extras", action="store_true",
+                   help="skip the other configurations (L sweep, router-on layer and union sweep, "
+                        "24-layer stack), which add about two minutes to a single-GPU run")
     return p.parse_args()
 
 
@@ -125,7 +127,7 @@ class ClockSampler:
 class Workload:
     """Device-resident synthetic inputs for one benchmark configuration."""
 
-    def __init__(self, cfg_index, L, chunks, variant, device, flags=0):
+    def __init__(self, cfg_index, L, chunks, variant, device, flags=0, u=None):
         import torch
         from paper_2507_08771_b200 import binding as B
         self.torch, self.B = torch, B
@@ -133,8 +135,8 @@ class Workload:
         self.sh = sh = I.SHAPES[cfg_index]
         self.L = L or sh.L
         seed = I.config_seed(cfg_index)
-        self.u = sh.u
-        self.active_bytes = sh.active_bytes()
+        self.u = sh.u if u is None else u
+        self.active_bytes = sh.active_bytes(self.u)
         # successive chunks of configs 1-3 are independent inputs; the stack (4) feeds each layer
         # the previous layer's output, so only its routing inputs and weights are stable
         self.call_flags = B.CALL_INDEPENDENT if cfg_index == 4 else B.CALL_INDEPENDENT_X
@@ -157,11 +159,11 @@ class Workload:
         if cfg_index == 4:
             # chunk c runs through all 24 layers; scores differ per (layer, chunk)
             self.calls_per_chunk = self.n_copies
-            sc = np.stack([np.stack([I.make_scores(sh.E, self.L, sh.u, seed, layer=l, chunk=c)
+            sc = np.stack([np.stack([I.make_scores(sh.E, self.L, self.u, seed, layer=l, chunk=c)
                                      for l in range(self.n_copies)]) for c in range(n)])
         else:
             self.calls_per_chunk = 1
-            sc = np.stack([I.make_scores(sh.E, self.L, sh.u, seed, chunk=c) for c in range(n)])[:, None]
+            sc = np.stack([I.make_scores(sh.E, self.L, self.u, seed, chunk=c) for c in range(n)])[:, None]
         xs = np.stack([I.make_x(sh.d, self.L, seed, chunk=c) for c in range(n)])
         self.scores_host = torch.from_numpy(sc).pin_memory()
         self.x_host = torch.from_numpy(xs.view(np.int16)).pin_memory()
@@ -449,31 +451,126 @@ def run_ours(args):
             "value": gbs, "unit": "GB/s", "cores": 1, "kind": "oracle", "us_per_chunk": us,
             "sample": f"{n} chunks of the same workload (one layer call each), union-restricted "
                       f"sum, float64, single thread"}
-    if args.sweep and args.config == 2:
-        line["sweep"] = sweep(args, torch, device)
+    if not args.no_extras and world == 1:
+        del wl, g_step, g_expert
+        torch.cuda.empty_cache()
+        line["extras"] = extras(args, torch, device, peak)
     print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()
 
 
-def sweep(args, torch, device):
+class RouterWorkload:
+    """Config 3 with the router on: blockffn_layer_forward over correlated or iid chunks."""
+
+    def __init__(self, chunks, device, rho, n_copies):
+        import torch
+        from paper_2507_08771_b200 import binding as B
+        self.torch, self.B, self.chunks = torch, B, chunks
+        self.sh = sh = I.SHAPES[3]
+        seed = I.config_seed(3)
+        self.layer = B.Layer(sh.d, sh.E, sh.d_e, L_max=sh.L, device=device)
+        w = I.make_layer(sh, seed, bias_shift=I.ROUTER_BIAS_SHIFT)
+        first = self.layer.upload_weights(w)
+        self.dws = [first]
+        for _ in range(n_copies - 1):          # distinct addresses for the expert weights only
+            tU, tD = B.to_device_bf16(w["U"], device), B.to_device_bf16(w["D"], device)
+            t = dict(first.tensors, U=tU, D=tD)
+            self.dws.append(B.DeviceWeights(B.make_weights(t["W_r"], t["gain"], t["bias"], tU, tD), t))
+        if rho is None:
+            xs = np.stack([I.make_x(sh.d, sh.L, seed, chunk=c) for c in range(chunks)])
+        else:
+            xs = np.stack([I.make_correlated_x(sh.d, sh.L, rho, seed, chunk=c) for c in range(chunks)])
+        self.x = torch.from_numpy(xs.view(np.int16)).to(device).view(torch.bfloat16)
+        self.out = torch.zeros(chunks, sh.L, sh.d, dtype=torch.float32, device=device)
+
+    def enqueue_step(self, stream):
+        B, lay = self.B, self.layer
+        for c in range(self.chunks):
+            B.blockffn_layer_forward(lay.h, self.dws[c % len(self.dws)].struct, self.x[c], self.sh.L,
+                                     self.out[c], None, lay.stats, 0, stream)
+
+    def sparsity(self):
+        hs = self.layer.stats_host()
+        return (self.B.blockffn_tls(hs, self.sh.E), 1.0 - self.B.blockffn_cls(hs, self.sh.E))
+
+
+def extras(args, torch, device, peak):
+    """The other configurations, each as us per call and GB/s of active expert bytes."""
+    out = {}
+    chunks = min(args.chunks, 64)
+
+    def timed(wl):
+        stream = torch.cuda.Stream(device)
+        g = capture(torch, stream, wl.enqueue_step)
+        ms = time_replays(torch, stream, g, max(3, args.steps // 2), 3)
+        assert wl.layer.last_status() == 0
+        return ms
+
+    # config 2: L sweep, tensor-core path against CUDA-core path
     rows = []
     for L in I.L_SWEEP:
-        for variant in (1, 2):
-            try:
-                wl = Workload(2, L, args.chunks, variant, device)
-            except Exception as e:  # a variant that does not support the shape
-                rows.append({"L": L, "variant": variant, "error": str(e)})
-                continue
-            stream = torch.cuda.Stream(device)
-            g = capture(torch, stream, wl.enqueue_step)
-            ms = time_replays(torch, stream, g, args.steps, args.warmup)
-            us = ms * 1e3 / wl.chunks
-            rows.append({"L": L, "variant": variant, "us_per_chunk": us,
-                         "GBps": wl.active_bytes / (us * 1e-6) / 1e9})
-            del wl, g
+        row = {"L": L}
+        for name, variant in (("tensor_core", 0), ("cuda_core", 1)):
+            wl = Workload(2, L, chunks, variant, device, args.flags)
+            us = timed(wl) * 1e3 / wl.calls_per_step
+            hs = wl.layer.stats_host()
+            row[name] = {"us_per_call": us, "GBps": wl.active_bytes / us / 1e3,
+                         "frac_of_measured": wl.active_bytes / us / 1e3 / peak}
+            row["tls"] = wl.B.blockffn_tls(hs, wl.sh.E)
+            del wl
             torch.cuda.empty_cache()
-    return rows
+        rows.append(row)
+    out["config2_L_sweep"] = rows
+
+    # config 3: router on (iid tokens, and correlated tokens whose union is about 30 %), then the
+    # scores-in union sweep against the dense all-experts layer
+    sh = I.SHAPES[3]
+    full = {}
+    n_copies = copies_needed(sh.active_bytes(sh.E))          # sized for the dense union
+    lo, hi, rho = 0.0, 1.0, 0.9
+    for _ in range(7):                                        # bisect rho on the library's own router
+        rho = 0.5 * (lo + hi)
+        probe = RouterWorkload(16, device, rho, 1)
+        probe.enqueue_step(torch.cuda.current_stream())
+        torch.cuda.synchronize()
+        frac = probe.sparsity()[1]
+        lo, hi = (rho, hi) if frac > 0.30 else (lo, rho)
+        del probe
+    for name, r in (("iid_tokens", None), ("correlated_tokens", rho)):
+        wl = RouterWorkload(chunks, device, r, n_copies)
+        ms = timed(wl)
+        hs = wl.layer.stats_host()
+        tls, ufrac = wl.sparsity()
+        us = ms * 1e3 / chunks
+        mean_u = ufrac * sh.E
+        full[name] = {"rho": r, "us_per_call": us, "tls": tls, "mean_union": mean_u,
+                      "GBps": mean_u * sh.expert_bytes / us / 1e3,
+                      "launches_per_call": 3}
+        del wl
+        torch.cuda.empty_cache()
+    sweep_rows, dense_us = [], None
+    for frac in (1.0, 0.9, 0.8, 0.7, 0.6, 0.5, 0.4, 0.3, 0.2, 0.1):
+        u = int(round(frac * sh.E))
+        wl = Workload(3, sh.L, chunks, 0, device, args.flags, u=u)
+        us = timed(wl) * 1e3 / wl.calls_per_step
+        dense_us = us if dense_us is None else dense_us
+        sweep_rows.append({"union_frac": frac, "u": u, "us_per_call": us,
+                           "GBps": wl.active_bytes / us / 1e3, "time_vs_dense": us / dense_us})
+        del wl
+        torch.cuda.empty_cache()
+    full["union_sweep"] = sweep_rows
+    out["config3_full_layer"] = full
+
+    # config 4: 24-layer stack, residual between layers
+    wl = Workload(4, None, min(args.chunks, I.STACK_CHUNKS), 0, device, args.flags)
+    ms = timed(wl)
+    us_chunk = ms * 1e3 / wl.chunks
+    out["config4_stack"] = {"layers": wl.n_copies, "chunks": wl.chunks, "us_per_chunk": us_chunk,
+                            "us_per_layer": us_chunk / wl.n_copies,
+                            "GBps": wl.n_copies * wl.active_bytes / us_chunk / 1e3,
+                            "frac_of_measured": wl.n_copies * wl.active_bytes / us_chunk / 1e3 / peak}
+    return out
 
 
 if __name__ == "__main__":
