@@ -29,7 +29,7 @@ blockffn_status expert_dispatch(blockffn_ctx* c, const blockffn_weights* w, cons
   cudaError_t e;
   if (use_mma(c, L))
     e = launch_expert_mma(c, w, x, scores, L, union_ids, n_union, out, x_next, call_flags, nullptr,
-                          st);
+                          nullptr, st);
   else
     e = launch_expert_simt(c, w, x, scores, L, union_ids, n_union, out, x_next, call_flags, st);
   return e == cudaSuccess ? BLOCKFFN_OK : BLOCKFFN_ERR_CUDA;
@@ -127,7 +127,8 @@ blockffn_status blockffn_router(blockffn_handle h, const blockffn_weights* w, co
       (reinterpret_cast<uintptr_t>(tok_mask) & 3u))
     return BLOCKFFN_ERR_INVALID_ARG;
   cudaError_t e =
-      launch_router(h, w, x, L, scores, tok_mask, false, nullptr, static_cast<cudaStream_t>(stream));
+      launch_router(h, w, x, L, scores, tok_mask, false, nullptr, false,
+                    static_cast<cudaStream_t>(stream));
   return e == cudaSuccess ? BLOCKFFN_OK : BLOCKFFN_ERR_CUDA;
 }
 
@@ -181,7 +182,20 @@ blockffn_status blockffn_layer_forward(blockffn_handle h, const blockffn_weights
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   // The router writes the scores this very call consumes: never "independent".
   const int flags = call_flags & ~(BLOCKFFN_CALL_INDEPENDENT | BLOCKFFN_CALL_INDEPENDENT_X);
-  if (launch_router(h, w, x, L, h->scores, h->tok_mask, true, stats, st) != cudaSuccess)
+  if (use_mma(h, L)) {
+    // The router kernel leaves the raw logits; the expert kernels (every CTA needs the union
+    // before it can fetch a weight byte) apply ReLU, RMSNorm and gain themselves and CTA 0
+    // publishes scores, masks, union and counters.
+    if (launch_router(h, w, x, L, h->scores, h->tok_mask, false, nullptr, true, st) != cudaSuccess)
+      return BLOCKFFN_ERR_CUDA;
+    const RoutingOut pub{h->union_mask, h->union_ids, h->n_union, stats, h->scores, h->tok_mask};
+    const RouterLogits lg{h->a0, w->gain, h->cfg.rms_eps};
+    return launch_expert_mma(h, w, x, h->scores, L, nullptr, nullptr, out, x_next, flags, &pub, &lg,
+                             st) == cudaSuccess
+               ? BLOCKFFN_OK
+               : BLOCKFFN_ERR_CUDA;
+  }
+  if (launch_router(h, w, x, L, h->scores, h->tok_mask, true, stats, false, st) != cudaSuccess)
     return BLOCKFFN_ERR_CUDA;
   return expert_dispatch(h, w, x, h->scores, L, h->union_ids, h->n_union, out, x_next, flags, st);
 }
@@ -203,9 +217,9 @@ blockffn_status blockffn_layer_forward_scores(blockffn_handle h, const blockffn_
   if (use_mma(h, L)) {
     // The expert kernels derive Union(x) from the scores themselves (every CTA needs the
     // list before it can fetch a weight byte) and CTA 0 publishes it: no separate launch.
-    const RoutingOut pub{h->union_mask, h->union_ids, h->n_union, stats};
+    const RoutingOut pub{h->union_mask, h->union_ids, h->n_union, stats, nullptr, nullptr};
     return launch_expert_mma(h, w, x, scores, L, nullptr, nullptr, out, x_next, call_flags, &pub,
-                             st) == cudaSuccess
+                             nullptr, st) == cudaSuccess
                ? BLOCKFFN_OK
                : BLOCKFFN_ERR_CUDA;
   }

@@ -42,7 +42,7 @@ __device__ __forceinline__ float swish(float z) { return z / (1.0f + __expf(-z))
 // ---- launchers (each returns the cudaError_t of its launch) ----------------
 cudaError_t launch_router(blockffn_ctx* c, const blockffn_weights* w, const void* x, int L,
                           float* scores, uint32_t* tok_mask, bool fuse_union,
-                          blockffn_stats* stats, cudaStream_t st);
+                          blockffn_stats* stats, bool raw, cudaStream_t st);
 cudaError_t launch_chunk_union(blockffn_ctx* c, const float* scores, int L, uint32_t* union_mask,
                                int32_t* union_ids, int32_t* n_union, blockffn_stats* stats,
                                cudaStream_t st);
@@ -57,14 +57,23 @@ struct RoutingOut {
   int32_t* union_ids;
   int32_t* n_union;
   blockffn_stats* stats;
+  float* scores;        // [L][E], written only when the kernel normalises router logits itself
+  uint32_t* tok_mask;   // [L][words], likewise
+};
+// Raw router logits (Eq. 3 before ReLU) for kernels that finish the router themselves.
+struct RouterLogits {
+  const float* a0;      // [L][E]
+  const float* gain;    // [E]
+  float eps;
 };
 
 // Tensor-core / bulk-copy variant of the expert stage. union_ids == NULL: the kernels derive
-// the union from the nonzero pattern of scores and publish it through pub.
+// the union from the nonzero pattern of scores and publish it through pub; with logits != NULL
+// they first turn the raw router logits into scores (ReLU, RMSNorm, gain) and scores is unused.
 bool expert_mma_supported(const blockffn_ctx* c, int L);
 size_t expert_mma_h_bytes(const blockffn_config* cfg);
 cudaError_t expert_mma_setup(blockffn_ctx* c);
 cudaError_t launch_expert_mma(blockffn_ctx* c, const blockffn_weights* w, const void* x,
                               const float* scores, int L, const int32_t* union_ids,
                               const int32_t* n_union, float* out, void* x_next, int call_flags,
-                              const RoutingOut* pub, cudaStream_t st);
+                              const RoutingOut* pub, const RouterLogits* logits, cudaStream_t st);

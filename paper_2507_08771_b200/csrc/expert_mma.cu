@@ -51,8 +51,8 @@ constexpr int kSmemHalf = 113 * 1024;            // lets an up and a down CTA sh
 // ---- shared-memory layout ----------------------------------------------------
 __host__ __device__ inline int align128(int v) { return (v + 127) & ~127; }
 
-constexpr int kCtlBytes = 512;  // ints: [0] nu, [2] n_active, [3] bad bits; [8..40) union mask
-                                // words; [40..72), [72..104) scratch
+constexpr int kCtlBytes = 640;  // ints: [0] nu, [2] n_active, [3] bad bits; [8..40) union mask
+                                // words; [40..72), [72..104) scratch; [104..136) 1/rms per token
 constexpr int kOffCtl = 0;
 constexpr int kOffIds = kOffCtl + kCtlBytes;
 
@@ -146,15 +146,43 @@ __device__ __forceinline__ float swish_fast(float z) { return __fdividef(z, 1.0f
 // ids_in != NULL: taken from the caller's list (E entries are readable); entries out of
 // range are dropped and reported, a count out of range is clamped and reported.
 // tm: scratch of at least L * ceil(E/32) words of shared memory.
-__device__ int derive_union(const float* scores, const int32_t* ids_in, const int32_t* n_in,
-                            int L, int E, int* ids_sm, int* ctl, uint32_t* tm) {
+__device__ int derive_union(const float* scores, const RouterLogits& lg, const int32_t* ids_in,
+                            const int32_t* n_in, int L, int E, int* ids_sm, int* ctl,
+                            uint32_t* tm) {
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int nwarps = blockDim.x >> 5;
   const int words = (E + 31) >> 5;
   int* cnt = ctl + 40;
   int* act = ctl + 72;
   uint32_t* um = reinterpret_cast<uint32_t*>(ctl + 8);
-  if (ids_in == nullptr) {
+  float* rinv = reinterpret_cast<float*>(ctl + 104);
+  if (lg.a0 != nullptr) {
+    // Raw router logits: finish Eq. 3 here (ReLU, RMSNorm over all E entries, gain), with the
+    // arithmetic of the router kernel's own normalisation, and take the nonzero pattern.
+    for (int t = warp; t < L; t += nwarps) {
+      float ss = 0.0f;
+      for (int e = lane; e < E; e += 32) {
+        float v = __ldcg(lg.a0 + (size_t)t * E + e);
+        v = v > 0.0f ? v : 0.0f;
+        ss = fmaf(v, v, ss);
+      }
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
+      const float r = 1.0f / sqrtf(ss / (float)E + lg.eps);
+      if (lane == 0) rinv[t] = r;
+      for (int w = 0; w < words; ++w) {
+        const int e = 32 * w + lane;
+        float s = 0.0f;
+        if (e < E) {
+          float v = __ldcg(lg.a0 + (size_t)t * E + e);
+          v = v > 0.0f ? v : 0.0f;
+          s = __ldg(lg.gain + e) * v * r;
+        }
+        const uint32_t m = __ballot_sync(0xffffffffu, s != 0.0f);
+        if (lane == 0) tm[t * words + w] = m;
+      }
+    }
+  } else if (ids_in == nullptr) {
     // warp -> tokens warp, warp + nwarps, ...; four mask words in flight per step
     for (int t = warp; t < L; t += nwarps) {
       for (int w0 = 0; w0 < words; w0 += 4) {
@@ -171,6 +199,8 @@ __device__ int derive_union(const float* scores, const int32_t* ids_in, const in
         }
       }
     }
+  }
+  if (lg.a0 != nullptr || ids_in == nullptr) {
     __syncthreads();
     if (threadIdx.x < words) {
       uint32_t un = 0;
@@ -283,8 +313,9 @@ __device__ __forceinline__ void zero_acc(float (&a)[NT][4]) {
 struct UpParams {
   const uint16_t* x;       // bf16 [L][d]
   const uint16_t* U;       // bf16 [E][d_e][d]
-  const float* scores;     // f32 [L][E]
-  const int32_t* ids_in;   // caller's union list, or NULL: derive from scores
+  const float* scores;     // f32 [L][E] (unused when lg.a0 is set)
+  RouterLogits lg;         // raw router logits to finish here, or a0 == NULL
+  const int32_t* ids_in;   // caller's union list, or NULL: derive from scores / logits
   const int32_t* n_in;
   uint16_t* h;             // bf16 [q][L][d_e] intermediate
   int L, d, E, d_e, de_shift, ring_rows;   // de_shift: log2(d_e), or -1
@@ -295,6 +326,8 @@ struct UpParams {
   int32_t* pub_ids;
   int32_t* pub_n;
   blockffn_stats* stats;
+  float* pub_scores;       // logits mode only
+  uint32_t* pub_tok;
 };
 
 template <int NT>
@@ -318,7 +351,7 @@ __global__ void __launch_bounds__(kThreads, NT <= 2 ? 2 : 1) expert_up_mma_kerne
     pdl_trigger();
   }
   __syncthreads();
-  const int nu = derive_union(p.scores, p.ids_in, p.n_in, L, p.E, ids_sm, ctl,
+  const int nu = derive_union(p.scores, p.lg, p.ids_in, p.n_in, L, p.E, ids_sm, ctl,
                               reinterpret_cast<uint32_t*>(red));
 
   // This CTA's rows [r0, r1) of the u * d_e union rows (balanced: the first R % G CTAs take
@@ -364,7 +397,14 @@ __global__ void __launch_bounds__(kThreads, NT <= 2 ? 2 : 1) expert_up_mma_kerne
       if (t < L && m < rows) {
         hq[i] = row_q(ra + m);
         hj[i] = ra + m - hq[i] * d_e;
-        sc[i] = __ldcg(p.scores + (size_t)t * p.E + ids_sm[hq[i]]);
+        const int id = ids_sm[hq[i]];
+        if (p.lg.a0 != nullptr) {      // gain * ReLU(logit) / rms, as in derive_union
+          float v = __ldcg(p.lg.a0 + (size_t)t * p.E + id);
+          v = v > 0.0f ? v : 0.0f;
+          sc[i] = __ldg(p.lg.gain + id) * v * reinterpret_cast<const float*>(ctl + 104)[t];
+        } else {
+          sc[i] = __ldcg(p.scores + (size_t)t * p.E + id);
+        }
       }
     }
   };
@@ -443,6 +483,24 @@ __global__ void __launch_bounds__(kThreads, NT <= 2 ? 2 : 1) expert_up_mma_kerne
   if (p.early == 2 && ngroups == 0) pdl_wait();   // every kernel waits before it ends
   // CTA 0 publishes the routing it derived (after the wait: earlier readers are done)
   if (blockIdx.x == 0) {
+    if (p.lg.a0 != nullptr && p.pub_scores != nullptr) {   // the scores and masks it computed
+      const int words = (p.E + 31) >> 5;
+      const float* rinv = reinterpret_cast<const float*>(ctl + 104);
+      for (int t = warp; t < L; t += kWarps) {
+        for (int w = 0; w < words; ++w) {
+          const int e = 32 * w + lane;
+          float sv = 0.0f;
+          if (e < p.E) {
+            float v = __ldcg(p.lg.a0 + (size_t)t * p.E + e);
+            v = v > 0.0f ? v : 0.0f;
+            sv = __ldg(p.lg.gain + e) * v * rinv[t];
+            p.pub_scores[(size_t)t * p.E + e] = sv;
+          }
+          const uint32_t m = __ballot_sync(0xffffffffu, sv != 0.0f);
+          if (p.pub_tok && lane == 0) p.pub_tok[(size_t)t * words + w] = m;
+        }
+      }
+    }
     if (p.ids_in == nullptr) {
       const int words = (p.E + 31) >> 5;
       const uint32_t* um = reinterpret_cast<const uint32_t*>(ctl + 8);
@@ -474,6 +532,7 @@ struct DownParams {
   const uint16_t* D;       // bf16 [E][d][d_e]
   const uint16_t* h;       // bf16 [q][L][d_e]
   const float* scores;
+  RouterLogits lg;
   const int32_t* ids_in;
   const int32_t* n_in;
   float* out;              // f32 [L][d]
@@ -499,7 +558,7 @@ __global__ void __launch_bounds__(kThreads, NT <= 2 ? 2 : 1) expert_down_mma_ker
   pdl_trigger();
   __syncthreads();
   // The routing inputs were final before the up kernel of this call passed its own wait.
-  const int nu = derive_union(p.scores, p.ids_in, p.n_in, L, p.E, ids_sm, ctl,
+  const int nu = derive_union(p.scores, p.lg, p.ids_in, p.n_in, L, p.E, ids_sm, ctl,
                               reinterpret_cast<uint32_t*>(red));
 
   // Column tiles: G * per tiles of at most max_cols (<= 16) columns, tile w -> CTA w % G,
@@ -741,7 +800,7 @@ cudaError_t expert_mma_setup(blockffn_ctx*) {
 cudaError_t launch_expert_mma(blockffn_ctx* c, const blockffn_weights* w, const void* x,
                               const float* scores, int L, const int32_t* union_ids,
                               const int32_t* n_union, float* out, void* x_next, int call_flags,
-                              const RoutingOut* pub, cudaStream_t st) {
+                              const RoutingOut* pub, const RouterLogits* logits, cudaStream_t st) {
   const MmaPlan pl = make_plan(c->cfg, L, c->num_sms);
   if (!pl.ok) return cudaErrorNotSupported;
   UpParams up{};
@@ -765,11 +824,15 @@ cudaError_t launch_expert_mma(blockffn_ctx* c, const blockffn_weights* w, const 
     up.pub_ids = pub->union_ids;
     up.pub_n = pub->n_union;
     up.stats = pub->stats;
+    up.pub_scores = pub->scores;
+    up.pub_tok = pub->tok_mask;
   }
+  if (logits) up.lg = *logits;
   DownParams dn{};
   dn.D = static_cast<const uint16_t*>(w->D);
   dn.h = up.h;
   dn.scores = scores;
+  if (logits) dn.lg = *logits;
   dn.ids_in = union_ids;
   dn.n_in = n_union;
   dn.out = out;

@@ -80,7 +80,7 @@ router_kernel(const uint16_t* __restrict__ x, const uint16_t* __restrict__ W_r,
               const float* __restrict__ gain, const float* __restrict__ bias, float* a0,
               float* scores, uint32_t* tok_mask, int L, int d, int E, float eps,
               unsigned int* ticket, int fuse_union, uint32_t* union_mask, int32_t* union_ids,
-              int32_t* n_union, blockffn_stats* stats) {
+              int32_t* n_union, blockffn_stats* stats, int raw) {
   __shared__ float red[kWarps][8];
   __shared__ int sm[3 * kMaxWords];
   __shared__ int is_last;
@@ -89,18 +89,25 @@ router_kernel(const uint16_t* __restrict__ x, const uint16_t* __restrict__ W_r,
   const int chunks = d >> 3;
   const uint4* wrow = reinterpret_cast<const uint4*>(W_r + (size_t)i * d);
   const float b = bias ? bias[i] : 0.0f;
+  // The kernel may have been started while the work before it on the stream still runs
+  // (programmatic dependent launch): the router weights are stable and are requested now,
+  // x and everything this kernel writes are touched only after the wait.
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  uint4 w_first = make_uint4(0u, 0u, 0u, 0u);
+  if ((int)threadIdx.x < chunks) w_first = __ldg(wrow + threadIdx.x);
+  asm volatile("griddepcontrol.wait;" ::: "memory");
 
   for (int t0 = 0; t0 < L; t0 += 8) {
     float acc[8];
 #pragma unroll
     for (int t = 0; t < 8; ++t) acc[t] = 0.0f;
     for (int c = threadIdx.x; c < chunks; c += kThreads) {
-      const uint4 wv = __ldg(wrow + c);
+      const uint4 wv = c == (int)threadIdx.x ? w_first : __ldg(wrow + c);
       const uint32_t wp[4] = {wv.x, wv.y, wv.z, wv.w};
 #pragma unroll
       for (int t = 0; t < 8; ++t) {
         if (t0 + t < L) {
-          const uint4 xv = __ldg(reinterpret_cast<const uint4*>(x + (size_t)(t0 + t) * d) + c);
+          const uint4 xv = __ldcg(reinterpret_cast<const uint4*>(x + (size_t)(t0 + t) * d) + c);
           const uint32_t xp[4] = {xv.x, xv.y, xv.z, xv.w};
 #pragma unroll
           for (int p = 0; p < 4; ++p) {
@@ -127,6 +134,9 @@ router_kernel(const uint16_t* __restrict__ x, const uint16_t* __restrict__ W_r,
     __syncthreads();
   }
 
+  // raw: the logits are all the caller wants (the tensor-core expert kernels normalise them
+  // themselves, which saves this kernel's serial tail)
+  if (raw) return;
   // last block done: normalise. The ticket is reset for the next call.
   __threadfence();
   if (threadIdx.x == 0) {
@@ -172,13 +182,22 @@ router_kernel(const uint16_t* __restrict__ x, const uint16_t* __restrict__ W_r,
 
 cudaError_t launch_router(blockffn_ctx* c, const blockffn_weights* w, const void* x, int L,
                           float* scores, uint32_t* tok_mask, bool fuse_union,
-                          blockffn_stats* stats, cudaStream_t st) {
-  router_kernel<<<c->cfg.E, kThreads, 0, st>>>(
-      static_cast<const uint16_t*>(x), static_cast<const uint16_t*>(w->W_r), w->gain, w->bias,
-      c->a0, scores, tok_mask, L, c->cfg.d, c->cfg.E, c->cfg.rms_eps, c->ticket,
-      fuse_union ? 1 : 0, c->union_mask, c->union_ids, c->n_union, stats);
-  c->launches += 1;
-  return cudaGetLastError();
+                          blockffn_stats* stats, bool raw, cudaStream_t st) {
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cudaLaunchConfig_t lc{};
+  lc.gridDim = dim3(c->cfg.E);
+  lc.blockDim = dim3(kThreads);
+  lc.stream = st;
+  lc.attrs = attr;
+  lc.numAttrs = (c->cfg.flags & BLOCKFFN_CFG_NO_CHAINING) ? 0 : 1;
+  const cudaError_t e = cudaLaunchKernelEx(
+      &lc, router_kernel, static_cast<const uint16_t*>(x), static_cast<const uint16_t*>(w->W_r),
+      w->gain, w->bias, c->a0, scores, tok_mask, L, c->cfg.d, c->cfg.E, c->cfg.rms_eps, c->ticket,
+      fuse_union ? 1 : 0, c->union_mask, c->union_ids, c->n_union, stats, raw ? 1 : 0);
+  if (e == cudaSuccess) c->launches += 1;
+  return e;
 }
 
 cudaError_t launch_chunk_union(blockffn_ctx* c, const float* scores, int L, uint32_t* union_mask,
