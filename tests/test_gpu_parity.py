@@ -362,3 +362,88 @@ def test_config4_stack_teacher_forced_and_free_running():
         drift = np.abs(res_gpu.cpu().numpy() - res_ref).max() / rms(res_ref)
         assert np.isfinite(drift) and drift <= 1e-1, (l, drift)
     assert layer.last_status() == 0
+
+
+# ----------------------------------------------------------------------------
+# the launch configuration the benchmark times: a CUDA graph of back-to-back calls with the
+# per-call promises set, weight copies rotated, full-size shapes; sampled chunks against the oracle
+# ----------------------------------------------------------------------------
+def graph_of(fn):
+    stream = torch.cuda.Stream()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(stream):
+        fn(stream)
+        stream.synchronize()
+        with torch.cuda.graph(g, stream=stream):
+            fn(stream)
+        g.replay()
+        g.replay()
+        stream.synchronize()
+
+
+@pytest.mark.parametrize("cfg,flag", [(1, B.CALL_INDEPENDENT_X), (2, B.CALL_INDEPENDENT_X),
+                                      (2, B.CALL_INDEPENDENT), (2, 0)])
+def test_bench_launch_configuration_scores_in(cfg, flag):
+    sh, seed = I.SHAPES[cfg], I.config_seed(cfg)
+    n_chunks, n_copies = 24, 3
+    w = I.make_layer(sh, seed, with_router=False)
+    layer = B.Layer(sh.d, sh.E, sh.d_e, L_max=sh.L)
+    dws = [layer.upload_weights(w) for _ in range(n_copies)]
+    xs = [I.make_x(sh.d, sh.L, seed, chunk=c) for c in range(n_chunks)]
+    ss = [I.make_scores(sh.E, sh.L, sh.u, seed, chunk=c) for c in range(n_chunks)]
+    xd = [B.to_device_bf16(x) for x in xs]
+    sd = [dev(s) for s in ss]
+    out = torch.full((n_chunks, sh.L, sh.d), float("nan"), device="cuda")
+
+    def enqueue(stream):
+        for c in range(n_chunks):
+            B.blockffn_layer_forward_scores(layer.h, dws[c % n_copies].struct, xd[c], sd[c], sh.L,
+                                            out[c], None, layer.stats, flag, stream)
+
+    graph_of(enqueue)
+    got = out.cpu().numpy()
+    assert np.isfinite(got).all()
+    for c in (0, 1, 7, n_chunks - 1):                      # sampled chunks, element by element
+        ref = oracle.layer_forward_scores(xs[c], ss[c], w["U"], w["D"], union_only=True)
+        assert_close(got[c], ref.out, f"config {cfg} flag {flag} chunk {c}")
+    # every chunk: what holds at any size (zero scores => untouched experts; finite; nonzero)
+    assert all(np.abs(got[c]).max() > 0 for c in range(n_chunks))
+    hs = layer.stats_host()
+    assert hs.n_chunks == 3 * n_chunks                     # one eager run + two replays
+    assert B.blockffn_cls(hs, sh.E) == pytest.approx(1 - sh.u / sh.E)
+    assert layer.last_status() == 0
+
+
+def test_bench_launch_configuration_stack():
+    """Config 4 as the benchmark runs it: residual accumulate, bf16 hand-over between layers,
+    CALL_INDEPENDENT on every layer call, one graph; compared with the oracle's stack."""
+    sh, seed = I.SHAPES[4], I.config_seed(4)
+    n_layers, L = 5, sh.L
+    layer = B.Layer(sh.d, sh.E, sh.d_e, L_max=L)
+    ws = [I.make_layer(sh, seed, layer=l, with_router=False) for l in range(n_layers)]
+    dws = [layer.upload_weights(w) for w in ws]
+    x0 = I.make_x(sh.d, L, seed, chunk=3)
+    ss = [I.make_scores(sh.E, L, sh.u, seed, layer=l, chunk=3) for l in range(n_layers)]
+    sd = [dev(s) for s in ss]
+    x0d = B.to_device_bf16(x0)
+    res = torch.zeros(L, sh.d, device="cuda")
+    xpp = torch.zeros(2, L, sh.d, dtype=torch.bfloat16, device="cuda")
+
+    def enqueue(stream):
+        res.copy_(x0d)
+        xpp[0].copy_(x0d)
+        for l in range(n_layers):
+            B.blockffn_layer_forward_scores(layer.h, dws[l].struct, xpp[l % 2], sd[l], L, res,
+                                            xpp[(l + 1) % 2], layer.stats,
+                                            B.CALL_ACCUMULATE | B.CALL_INDEPENDENT, stream)
+
+    graph_of(enqueue)
+    r = I.bf16_bits_to_f32(x0).astype(np.float64)
+    xr = x0
+    for l in range(n_layers):
+        ref = oracle.layer_forward_scores(xr, ss[l], ws[l]["U"], ws[l]["D"], union_only=True)
+        xr = oracle.residual_step(r, ref.out)
+    got = res.cpu().numpy()
+    drift = np.abs(got - r).max() / rms(r)
+    assert np.isfinite(got).all() and drift <= 1e-1, drift
+    assert layer.last_status() == 0
