@@ -59,12 +59,12 @@ constexpr int kOffIds = kOffCtl + kCtlBytes;
 struct UpLayout {
   int off_red, off_x, off_ring, total;
 };
-// red: per warp a 32 x (8 NT) tile; x: L rows of 2d bytes; ring: ring_rows rows of 2d bytes
-__host__ __device__ inline UpLayout up_layout(int d, int E, int NT, int L, int ring_rows) {
+// red: per warp a 32 x 8 tile; x: one tile of 8 tokens (2d bytes each); ring: ring_rows rows
+__host__ __device__ inline UpLayout up_layout(int d, int E, int ring_rows) {
   UpLayout s;
   s.off_red = kOffIds + align128(E * 4);
-  s.off_x = s.off_red + kWarps * 32 * 8 * NT * 4;
-  s.off_ring = s.off_x + align128(L * 2 * d);
+  s.off_x = s.off_red + kWarps * 32 * 8 * 4;
+  s.off_ring = s.off_x + align128(8 * 2 * d);
   s.total = s.off_ring + ring_rows * 2 * d;
   return s;
 }
@@ -72,13 +72,12 @@ __host__ __device__ inline UpLayout up_layout(int d, int E, int NT, int L, int r
 struct DownLayout {
   int off_red, off_h, off_d, slot_h, slot_d, total;
 };
-// h ring: ns slots of L rows of 2 d_e bytes; D ring: ns slots of max_cols rows of 2 d_e bytes
-__host__ __device__ inline DownLayout down_layout(int d_e, int E, int NT, int L, int ns,
-                                                  int max_cols) {
+// h ring: ns slots of 8 token rows of 2 d_e bytes; D ring: ns slots of max_cols rows of 2 d_e bytes
+__host__ __device__ inline DownLayout down_layout(int d_e, int E, int ns, int max_cols) {
   DownLayout s;
   s.off_red = kOffIds + align128(E * 4);
-  s.off_h = s.off_red + kWarps * 16 * 8 * NT * 4;
-  s.slot_h = L * 2 * d_e;
+  s.off_h = s.off_red + kWarps * 16 * 8 * 4;
+  s.slot_h = 8 * 2 * d_e;
   s.slot_d = max_cols * 2 * d_e;
   s.off_d = s.off_h + align128(ns * s.slot_h);
   s.total = s.off_d + ns * s.slot_d;
@@ -330,18 +329,23 @@ struct UpParams {
   uint32_t* pub_tok;
 };
 
-template <int NT>
-__global__ void __launch_bounds__(kThreads, NT <= 2 ? 2 : 1) expert_up_mma_kernel(const UpParams p) {
+// Chunks longer than 8 tokens go through the math in groups of 8 tokens (one mma n tile): the
+// weights stay in shared memory, the x tile of the next group replaces the current one. That
+// keeps the kernel within half an SM's shared memory for every L, which is what lets it run
+// next to the down kernel of the call before.
+__global__ void __launch_bounds__(kThreads, 2) expert_up_mma_kernel(const UpParams p) {
   extern __shared__ __align__(128) unsigned char smem[];
+  constexpr int NT = 1;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int d = p.d, d_e = p.d_e, L = p.L;
   constexpr int ns = kUpStages;
-  const UpLayout lay = up_layout(d, p.E, NT, L, p.ring_rows);
+  const UpLayout lay = up_layout(d, p.E, p.ring_rows);
   const uint32_t sbase = smem_u32(smem);
   int* ctl = reinterpret_cast<int*>(smem + kOffCtl);
   int* ids_sm = reinterpret_cast<int*>(smem + kOffIds);
   float* red = reinterpret_cast<float*>(smem + lay.off_red);
   const int row_bytes = 2 * d;
+  const int ntg = (L + 7) >> 3;            // token groups
 
   if (tid < 8) ctl[tid] = 0;
   if (p.early) {
@@ -383,51 +387,48 @@ __global__ void __launch_bounds__(kThreads, NT <= 2 ? 2 : 1) expert_up_mma_kerne
       j = 0;
     }
   };
-  // The router score, expert slot and neuron of each element this thread finishes in a stage
-  // (element e = t * 32 + m: token t, row m of the stage).
-  float sc[NT];
-  int hq[NT], hj[NT];
-  auto prepare = [&](int gi) {
+  // x tile of token group tgi: tokens [8 tgi, 8 tgi + 8) of the chunk
+  auto issue_x = [&](int tgi) {
+    const int nt = min(8, L - 8 * tgi);
+    copy_run(sbase + lay.off_x, p.x + (size_t)8 * tgi * d, nt * row_bytes);
+  };
+  // The router score, expert slot and neuron of the element this thread finishes in a pass
+  // (element e = t * 32 + m: token t of the group, row m of the stage).
+  float sc = 0.0f;
+  int hq = -1, hj = 0;
+  auto prepare = [&](int gi, int tgi) {
     const int ra = r0 + gi * rpg, rows = min(r1, ra + rpg) - ra;
-#pragma unroll
-    for (int i = 0; i < NT; ++i) {
-      const int e = tid + i * kThreads, t = e >> 5, m = e & 31;
-      sc[i] = 0.0f;
-      hq[i] = -1;
-      if (t < L && m < rows) {
-        hq[i] = row_q(ra + m);
-        hj[i] = ra + m - hq[i] * d_e;
-        const int id = ids_sm[hq[i]];
-        if (p.lg.a0 != nullptr) {      // gain * ReLU(logit) / rms, as in derive_union
-          float v = __ldcg(p.lg.a0 + (size_t)t * p.E + id);
-          v = v > 0.0f ? v : 0.0f;
-          sc[i] = __ldg(p.lg.gain + id) * v * reinterpret_cast<const float*>(ctl + 104)[t];
-        } else {
-          sc[i] = __ldcg(p.scores + (size_t)t * p.E + id);
-        }
+    const int t = 8 * tgi + (tid >> 5), m = tid & 31;
+    sc = 0.0f;
+    hq = -1;
+    if (t < L && m < rows) {
+      hq = row_q(ra + m);
+      hj = ra + m - hq * d_e;
+      const int id = ids_sm[hq];
+      if (p.lg.a0 != nullptr) {      // gain * ReLU(logit) / rms, as in derive_union
+        float v = __ldcg(p.lg.a0 + (size_t)t * p.E + id);
+        v = v > 0.0f ? v : 0.0f;
+        sc = __ldg(p.lg.gain + id) * v * reinterpret_cast<const float*>(ctl + 104)[t];
+      } else {
+        sc = __ldcg(p.scores + (size_t)t * p.E + id);
       }
     }
   };
   const int g = lane >> 2, tg = lane & 3, par = g & 1;
   const int npairs = d >> 6;   // 64-wide k blocks
-  const unsigned char* x_row[NT];
-#pragma unroll
-  for (int n = 0; n < NT; ++n) x_row[n] = smem + lay.off_x + min(8 * n + g, L - 1) * row_bytes;
 
   const int g_first = min(ngroups, ns);
   if (p.early) {
     for (int gi = 0; gi < g_first; ++gi) issue(gi);
-    if (ngroups > 0) prepare(0);
+    if (ngroups > 0) prepare(0, 0);
   }
   if (p.early < 2) pdl_wait();   // x may come from the kernel just before
-  if (ngroups > 0) copy_run(sbase + lay.off_x, p.x, L * row_bytes);
+  if (ngroups > 0) issue_x(0);
   if (!p.early) {
     for (int gi = 0; gi < g_first; ++gi) issue(gi);
-    if (ngroups > 0) prepare(0);
+    if (ngroups > 0) prepare(0, 0);
   }
   cp_async_commit();
-  cp_async_wait_group<0>();
-  __syncthreads();
 
   for (int gi = 0; gi < ngroups; ++gi) {
     const int rows = min(r1, r0 + (gi + 1) * rpg) - (r0 + gi * rpg);
@@ -437,48 +438,52 @@ __global__ void __launch_bounds__(kThreads, NT <= 2 ? 2 : 1) expert_up_mma_kerne
     const unsigned char* rb0 = slot + min(g + 8, rows - 1) * row_bytes;
     const unsigned char* ra1 = slot + min(g + 16, rows - 1) * row_bytes;
     const unsigned char* rb1 = slot + min(g + 24, rows - 1) * row_bytes;
-    float a00[NT][4], a01[NT][4], a10[NT][4], a11[NT][4];
-    zero_acc<NT>(a00);
-    zero_acc<NT>(a01);
-    zero_acc<NT>(a10);
-    zero_acc<NT>(a11);
+    for (int tgi = 0; tgi < ntg; ++tgi) {
+      const int nt = min(8, L - 8 * tgi);
+      const unsigned char* x_row = smem + lay.off_x + min(g, nt - 1) * row_bytes;
+      // the stage and the x tile of this pass have been requested: wait for all of it
+      cp_async_wait_group<0>();
+      __syncthreads();
+      float a00[NT][4], a01[NT][4], a10[NT][4], a11[NT][4];
+      zero_acc<NT>(a00);
+      zero_acc<NT>(a01);
+      zero_acc<NT>(a10);
+      zero_acc<NT>(a11);
 #pragma unroll 2
-    for (int pp = warp; pp < npairs; pp += kWarps) {
-      Frag64 fx[NT];
-#pragma unroll
-      for (int n = 0; n < NT; ++n) fx[n] = load_frag64(x_row[n] + 128 * pp, par, tg);
-      const Frag64 fa = load_frag64(ra0 + 128 * pp, par, tg);
-      const Frag64 fb = load_frag64(rb0 + 128 * pp, par, tg);
-      mma_block64<NT>(a00, a01, fa, fb, fx);
-      if (two) {
-        const Frag64 fc = load_frag64(ra1 + 128 * pp, par, tg);
-        const Frag64 fd = load_frag64(rb1 + 128 * pp, par, tg);
-        mma_block64<NT>(a10, a11, fc, fd, fx);
+      for (int pp = warp; pp < npairs; pp += kWarps) {
+        Frag64 fx[NT];
+        fx[0] = load_frag64(x_row + 128 * pp, par, tg);
+        const Frag64 fa = load_frag64(ra0 + 128 * pp, par, tg);
+        const Frag64 fb = load_frag64(rb0 + 128 * pp, par, tg);
+        mma_block64<NT>(a00, a01, fa, fb, fx);
+        if (two) {
+          const Frag64 fc = load_frag64(ra1 + 128 * pp, par, tg);
+          const Frag64 fd = load_frag64(rb1 + 128 * pp, par, tg);
+          mma_block64<NT>(a10, a11, fc, fd, fx);
+        }
       }
-    }
-    // cross-warp reduction of the K split, then Swish, score, store
-    float* mine = red + warp * (32 * 8 * NT);
-    store_partial<NT>(mine, 32, 0, a00, a01, g, tg);
-    if (two) store_partial<NT>(mine, 32, 16, a10, a11, g, tg);
-    __syncthreads();     // every warp is done with the slot: refill it
-    if (gi + ns < ngroups) issue(gi + ns);
-    cp_async_commit();   // one group per stage, empty or not, keeps the count below uniform
-    if (gi == 0 && p.early == 2) pdl_wait();   // h may still be read by the call before
-#pragma unroll
-    for (int i = 0; i < NT; ++i) {
-      if (hq[i] >= 0) {
-        const int e = tid + i * kThreads;
+      // cross-warp reduction of the K split, then Swish, score, store
+      float* mine = red + warp * (32 * 8);
+      store_partial<NT>(mine, 32, 0, a00, a01, g, tg);
+      if (two) store_partial<NT>(mine, 32, 16, a10, a11, g, tg);
+      __syncthreads();     // every warp is done with the x tile (and, after the last group, the slot)
+      const bool last_tg = tgi + 1 == ntg;
+      if (last_tg && gi + ns < ngroups) issue(gi + ns);
+      if (!last_tg) issue_x(tgi + 1);
+      else if (gi + 1 < ngroups && ntg > 1) issue_x(0);
+      cp_async_commit();
+      if (gi == 0 && tgi == 0 && p.early == 2) pdl_wait();   // h may still be read by the call before
+      if (hq >= 0) {
         float v = 0.0f;
 #pragma unroll
-        for (int w = 0; w < kWarps; ++w) v += red[w * (32 * 8 * NT) + e];
-        p.h[((size_t)hq[i] * L + (e >> 5)) * d_e + hj[i]] =
-            (uint16_t)f32_to_bf16_bits(sc[i] * swish_fast(v));
+        for (int w = 0; w < kWarps; ++w) v += red[w * (32 * 8) + tid];
+        p.h[((size_t)hq * L + 8 * tgi + (tid >> 5)) * d_e + hj] =
+            (uint16_t)f32_to_bf16_bits(sc * swish_fast(v));
       }
+      if (!last_tg) prepare(gi, tgi + 1);
+      else if (gi + 1 < ngroups) prepare(gi + 1, 0);
+      // the next pass starts with a wait and a barrier, which also protects red
     }
-    if (gi + 1 < ngroups) prepare(gi + 1);
-    // stage gi + 1, if it is a refill, was committed ns - 1 groups ago
-    if (gi + 1 >= ns) cp_async_wait_group<ns - 1>();
-    __syncthreads();
   }
   if (p.early == 2 && ngroups == 0) pdl_wait();   // every kernel waits before it ends
   // CTA 0 publishes the routing it derived (after the wait: earlier readers are done)
@@ -542,17 +547,21 @@ struct DownParams {
   uint32_t* status;
 };
 
-template <int NT>
-__global__ void __launch_bounds__(kThreads, NT <= 2 ? 2 : 1) expert_down_mma_kernel(const DownParams p) {
+// NTG: token groups of 8 in the chunk (1 .. 4), each with its own accumulators
+template <int NTG>
+__global__ void __launch_bounds__(kThreads, 2) expert_down_mma_kernel(const DownParams p) {
   extern __shared__ __align__(128) unsigned char smem[];
+  constexpr int NT = 1;
+  constexpr int kMaxTg = NTG;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int d = p.d, d_e = p.d_e, L = p.L, per = p.per;
-  const DownLayout lay = down_layout(d_e, p.E, NT, L, p.ns, p.max_cols);
+  const DownLayout lay = down_layout(d_e, p.E, p.ns, p.max_cols);
   const uint32_t sbase = smem_u32(smem);
   int* ctl = reinterpret_cast<int*>(smem + kOffCtl);
   int* ids_sm = reinterpret_cast<int*>(smem + kOffIds);
   float* red = reinterpret_cast<float*>(smem + lay.off_red);
   const int row_bytes = 2 * d_e;
+  constexpr int ntg = NTG;
 
   if (tid < 8) ctl[tid] = 0;
   pdl_trigger();
@@ -564,7 +573,8 @@ __global__ void __launch_bounds__(kThreads, NT <= 2 ? 2 : 1) expert_down_mma_ker
   // Column tiles: G * per tiles of at most max_cols (<= 16) columns, tile w -> CTA w % G,
   // tile w = columns [w cols_q + min(w, cols_rem), ...). Per tile, the experts go through
   // the ring in rounds: all of them at once when they fit (the usual case), else half a
-  // ring per round, the next round in flight during the math.
+  // ring per round, the next round in flight during the math. Within a round the chunk's
+  // tokens go through the math in groups of 8, each with its own h tile and accumulators.
   const int G = gridDim.x;
   const int rsz = (per == 1 && nu <= p.ns) ? max(nu, 1) : max(1, min(nu, p.ns / 2));
   const int rpt = (nu + rsz - 1) / rsz;                  // rounds per tile
@@ -577,106 +587,121 @@ __global__ void __launch_bounds__(kThreads, NT <= 2 ? 2 : 1) expert_down_mma_ker
     return w * p.cols_q + min(w, p.cols_rem);
   };
   auto tile_nc = [&](int ti) { return p.cols_q + ((int)blockIdx.x + ti * G < p.cols_rem ? 1 : 0); };
-  // (i_ti, i_rr): tile and round-in-tile of the next round to request; (c_ti, c_rr): to compute
-  int i_r = 0, i_ti = 0, i_rr = 0;
+  int i_r = 0, i_ti = 0, i_rr = 0;      // the next round to request: index, tile, round in tile
   auto issue_d = [&]() {
     const int q0 = i_rr * rsz, n = min(rsz, nu - q0);
     const char* base = dptr + (size_t)tile_c0(i_ti) * row_bytes;
     copy_pieces(sbase + lay.off_d + (i_r & 1) * rsz * lay.slot_d, lay.slot_d, n,
                 tile_nc(i_ti) * row_bytes,
                 [&](int i) { return base + (size_t)ids_sm[q0 + i] * estride; });
-  };
-  auto issue_h = [&](int r, int rr) {
-    const int q0 = rr * rsz, n = min(rsz, nu - q0);
-    copy_run(sbase + lay.off_h + (r & 1) * rsz * lay.slot_h, hptr + (size_t)q0 * lay.slot_h,
-             n * lay.slot_h);
-  };
-  auto advance = [&]() {
     ++i_r;
     if (++i_rr == rpt) {
       i_rr = 0;
       ++i_ti;
     }
   };
+  // h tile of (round-in-tile rr, token group tgi): tokens [8 tgi, ..) of the round's experts
+  // (a chunk of at most 8 tokens has one group, and its tiles are one run in memory: they are
+  // kept at the chunk's own stride so that all threads share one long copy)
+  const int hstride = ntg == 1 ? L * row_bytes : lay.slot_h;
+  auto issue_h = [&](int rr, int tgi) {
+    const int q0 = rr * rsz, n = min(rsz, nu - q0), nt = min(8, L - 8 * tgi);
+    const char* base = hptr + ((size_t)q0 * L + 8 * tgi) * row_bytes;
+    if (ntg == 1) {
+      copy_run(sbase + lay.off_h, base, n * hstride);
+    } else {
+      const size_t qstride = (size_t)L * row_bytes;
+      copy_pieces(sbase + lay.off_h, hstride, n, nt * row_bytes,
+                  [&](int i) { return base + (size_t)i * qstride; });
+    }
+  };
   const int g = lane >> 2, tg = lane & 3, par = g & 1;
   const int npairs = d_e >> 6;         // 64-wide k blocks per expert
   const int pshift = (npairs & (npairs - 1)) == 0 ? __ffs(npairs) - 1 : -1;
-  int h_off[NT];
-#pragma unroll
-  for (int n = 0; n < NT; ++n) h_off[n] = min(8 * n + g, L - 1) * row_bytes;
 
-  // before the wait: the weights of the first two rounds; after it: their h
+  // before the wait: the weights of the first two rounds
   const int npre = min(nrounds, 2);
-  const int rr1 = rpt > 1 ? 1 : 0;     // round-in-tile of round 1
   for (int r = 0; r < npre; ++r) {
     issue_d();
-    advance();
     cp_async_commit();
   }
   pdl_wait();            // h, out and x_next are safe to touch from here on
-  if (npre > 0) {
+  if (nrounds > 0) {
     issue_h(0, 0);
     cp_async_commit();
   }
-  if (npre > 1) {
-    issue_h(1, rr1);
-    cp_async_commit();
-  }
 
-  float acc0[NT][4], acc1[NT][4];
+  float acc0[kMaxTg][4], acc1[kMaxTg][4];
   int c_ti = 0, c_rr = 0;
   for (int r = 0; r < nrounds; ++r) {
     const int q0 = c_rr * rsz, n = min(rsz, nu - q0);
     const int c0 = tile_c0(c_ti), ncols = tile_nc(c_ti);
+    const int off_a = min(g, max(ncols, 1) - 1) * row_bytes;
+    const int off_b = min(g + 8, max(ncols, 1) - 1) * row_bytes;
+    const unsigned char* d_base = smem + lay.off_d + (r & 1) * rsz * lay.slot_d;
+    const unsigned char* h_base = smem + lay.off_h;
+    const int nblk = n * npairs;
     if (c_rr == 0) {
-      zero_acc<NT>(acc0);
-      zero_acc<NT>(acc1);
+      zero_acc<kMaxTg>(acc0);
+      zero_acc<kMaxTg>(acc1);
     }
-    // everything but the newest group has to have landed (the newest is the next round's)
-    if (r + 1 < nrounds) cp_async_wait_group<1>(); else cp_async_wait_group<0>();
-    __syncthreads();
-    if (ncols > 0) {
-      const int off_a = min(g, ncols - 1) * row_bytes, off_b = min(g + 8, ncols - 1) * row_bytes;
-      const unsigned char* d_base = smem + lay.off_d + (r & 1) * rsz * lay.slot_d;
-      const unsigned char* h_base = smem + lay.off_h + (r & 1) * rsz * lay.slot_h;
-      // the 64-wide k blocks of the round's experts are dealt round-robin to the warps
-      const int nblk = n * npairs;
+#pragma unroll
+    for (int tgi = 0; tgi < kMaxTg; ++tgi) {
+      if (tgi < ntg) {
+        const int nt = min(8, L - 8 * tgi);
+        const int h_off = min(g, nt - 1) * row_bytes;
+        // this round's slabs and this pass's h tile have been requested: wait for all of it
+        cp_async_wait_group<0>();
+        __syncthreads();
+        if (ncols > 0) {
+          // the 64-wide k blocks of the round's experts are dealt round-robin to the warps
 #pragma unroll 2
-      for (int b = warp; b < nblk; b += kWarps) {
-        const int i = pshift >= 0 ? b >> pshift : b / npairs, pp = b - i * npairs;
-        const unsigned char* da = d_base + i * lay.slot_d + 128 * pp;
-        const unsigned char* ha = h_base + i * lay.slot_h + 128 * pp;
-        const Frag64 fa = load_frag64(da + off_a, par, tg);
-        const Frag64 fb = load_frag64(da + off_b, par, tg);
-        Frag64 fx[NT];
-#pragma unroll
-        for (int nn = 0; nn < NT; ++nn) fx[nn] = load_frag64(ha + h_off[nn], par, tg);
-        mma_block64<NT>(acc0, acc1, fa, fb, fx);
-      }
-    }
-    if (r + 2 < nrounds) {       // refill this round's half of the ring
-      __syncthreads();
-      issue_d();
-      issue_h(i_r, i_rr);
-      advance();
-      cp_async_commit();
-    }
-    if (c_rr == rpt - 1) {       // the tile is complete: reduce across warps and store
-      store_partial<NT>(red + warp * (16 * 8 * NT), 16, 0, acc0, acc1, g, tg);
-      __syncthreads();
-      for (int e = tid; e < 16 * 8 * NT; e += kThreads) {
-        const int t = e >> 4, m = e & 15;
-        if (t < L && m < ncols) {
-          float v = 0.0f;
-#pragma unroll
-          for (int w = 0; w < kWarps; ++w) v += red[w * (16 * 8 * NT) + e];
-          const size_t o = (size_t)t * d + c0 + m;
-          if (p.accumulate) v += __ldcg(p.out + o);
-          p.out[o] = v;
-          if (p.x_next) p.x_next[o] = (uint16_t)f32_to_bf16_bits(v);
+          for (int b = warp; b < nblk; b += kWarps) {
+            const int i = pshift >= 0 ? b >> pshift : b / npairs, pp = b - i * npairs;
+            const unsigned char* da = d_base + i * lay.slot_d + 128 * pp;
+            const unsigned char* ha = h_base + i * hstride + 128 * pp;
+            const Frag64 fa = load_frag64(da + off_a, par, tg);
+            const Frag64 fb = load_frag64(da + off_b, par, tg);
+            Frag64 fx[NT];
+            fx[0] = load_frag64(ha + h_off, par, tg);
+            float (&b0)[1][4] = reinterpret_cast<float (&)[1][4]>(acc0[tgi]);
+            float (&b1)[1][4] = reinterpret_cast<float (&)[1][4]>(acc1[tgi]);
+            mma_block64<NT>(b0, b1, fa, fb, fx);
+          }
+        }
+        const bool last_tg = tgi + 1 == ntg;
+        if (!last_tg || r + 1 < nrounds) {   // more to fetch into what this pass has read
+          __syncthreads();   // every warp is done with the h tile (and, after the last group, the slabs)
+          if (last_tg && r + 2 < nrounds) issue_d();        // refill this round's half of the ring
+          if (!last_tg) issue_h(c_rr, tgi + 1);
+          else issue_h(c_rr + 1 == rpt ? 0 : c_rr + 1, 0);
+          cp_async_commit();
         }
       }
-      __syncthreads();
+    }
+    if (c_rr == rpt - 1) {       // the tile is complete: reduce across warps and store
+#pragma unroll
+      for (int tgi = 0; tgi < kMaxTg; ++tgi) {
+        if (tgi < ntg) {
+          float (&b0)[1][4] = reinterpret_cast<float (&)[1][4]>(acc0[tgi]);
+          float (&b1)[1][4] = reinterpret_cast<float (&)[1][4]>(acc1[tgi]);
+          store_partial<NT>(red + warp * 128, 16, 0, b0, b1, g, tg);
+          __syncthreads();
+          if (tid < 128) {
+            const int t = 8 * tgi + (tid >> 4), m = tid & 15;
+            if (t < L && m < ncols) {
+              float v = 0.0f;
+#pragma unroll
+              for (int w = 0; w < kWarps; ++w) v += red[w * 128 + tid];
+              const size_t o = (size_t)t * d + c0 + m;
+              if (p.accumulate) v += __ldcg(p.out + o);
+              p.out[o] = v;
+              if (p.x_next) p.x_next[o] = (uint16_t)f32_to_bf16_bits(v);
+            }
+          }
+          __syncthreads();
+        }
+      }
     }
     if (++c_rr == rpt) {
       c_rr = 0;
@@ -700,19 +725,19 @@ __global__ void __launch_bounds__(kThreads, NT <= 2 ? 2 : 1) expert_down_mma_ker
 
 // ---- host side -----------------------------------------------------------------------
 struct MmaPlan {
-  int NT, ring_rows, ns_down, max_cols, per, cols_q, cols_rem, smem_up, smem_down;
+  int ring_rows, ns_down, max_cols, per, cols_q, cols_rem, smem_up, smem_down;
   bool ok;
 };
 
 // Shapes the kernels take: d and d_e multiples of 64 (whole 64-wide k blocks, row strides
-// multiples of 128 bytes) and shared memory for x plus two stages of rows / two expert slabs.
+// multiples of 128 bytes) and, within half an SM's shared memory, an x tile plus a few rows
+// of U (up) and a few expert slabs with their h tiles (down).
 MmaPlan make_plan(const blockffn_config& cfg, int L, int grid) {
   MmaPlan pl{};
   pl.ok = false;
   const int d = cfg.d, d_e = cfg.d_e, E = cfg.E;
   if (L < 1 || L > 32 || grid < 1) return pl;
   if (d % 64 || d_e % 64 || E > 1024 || d > 32768 || d_e > 4096) return pl;
-  pl.NT = (L + 7) / 8;
   const int want_up = cfg.flags & 0xff, want_down = (cfg.flags >> 8) & 0xff;
   // down: column tiles
   pl.per = (d + 16 * grid - 1) / (16 * grid);
@@ -720,11 +745,10 @@ MmaPlan make_plan(const blockffn_config& cfg, int L, int grid) {
   pl.cols_q = d / W;
   pl.cols_rem = d % W;
   pl.max_cols = pl.cols_q + (pl.cols_rem ? 1 : 0);
-  // up: x resident, the rest of the budget is the ring
-  const int up_base = up_layout(d, E, pl.NT, L, 0).total;
-  const int down_base = down_layout(d_e, E, pl.NT, L, 0, pl.max_cols).total;
-  const int slot_dn = L * 2 * d_e + pl.max_cols * 2 * d_e;
-  // Paired: both kernels fit one SM together when x plus a modest ring fit half of it.
+  const int up_base = up_layout(d, E, 0).total;
+  const int down_base = down_layout(d_e, E, 0, pl.max_cols).total;
+  const int slot_dn = 8 * 2 * d_e + pl.max_cols * 2 * d_e;
+  // Paired: both kernels fit one SM together when the x tile plus a modest ring fit half of it.
   const bool paired = up_base + 12 * 2 * d <= kSmemHalf && down_base + 4 * slot_dn <= kSmemHalf;
   const int budget = paired ? kSmemHalf : kSmemMax;
   pl.ring_rows = (budget - up_base) / (2 * d);
@@ -736,8 +760,8 @@ MmaPlan make_plan(const blockffn_config& cfg, int L, int grid) {
   if (pl.ns_down > kMaxStages) pl.ns_down = kMaxStages;
   if (pl.ns_down > E) pl.ns_down = E < 2 ? 2 : E;
   if (pl.ns_down < 2) return pl;
-  pl.smem_up = up_layout(d, E, pl.NT, L, pl.ring_rows).total;
-  pl.smem_down = down_layout(d_e, E, pl.NT, L, pl.ns_down, pl.max_cols).total;
+  pl.smem_up = up_layout(d, E, pl.ring_rows).total;
+  pl.smem_down = down_layout(d_e, E, pl.ns_down, pl.max_cols).total;
   if (pl.smem_up > kSmemMax || pl.smem_down > kSmemMax) return pl;
   pl.ok = true;
   return pl;
@@ -746,10 +770,12 @@ MmaPlan make_plan(const blockffn_config& cfg, int L, int grid) {
 // Both kernels ask for the largest shared-memory carve-out: an SM keeps its carve-out while
 // any CTA runs on it, so a down CTA can only join an up CTA (and the next call's up CTA the
 // down CTA) if the first of them already configured the SM for both.
-template <int NT>
 cudaError_t set_attrs() {
-  const void* fns[2] = {reinterpret_cast<const void*>(&expert_up_mma_kernel<NT>),
-                        reinterpret_cast<const void*>(&expert_down_mma_kernel<NT>)};
+  const void* fns[5] = {reinterpret_cast<const void*>(&expert_up_mma_kernel),
+                        reinterpret_cast<const void*>(&expert_down_mma_kernel<1>),
+                        reinterpret_cast<const void*>(&expert_down_mma_kernel<2>),
+                        reinterpret_cast<const void*>(&expert_down_mma_kernel<3>),
+                        reinterpret_cast<const void*>(&expert_down_mma_kernel<4>)};
   for (const void* f : fns) {
     cudaError_t e = cudaFuncSetAttribute(f, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemMax);
     if (e != cudaSuccess) return e;
@@ -760,9 +786,8 @@ cudaError_t set_attrs() {
   return cudaSuccess;
 }
 
-template <int NT>
-cudaError_t launch_nt(const MmaPlan& pl, int grid, const UpParams& up, const DownParams& dn,
-                      bool chained, cudaStream_t st) {
+cudaError_t launch_pair(const MmaPlan& pl, int grid, const UpParams& up, const DownParams& dn,
+                        bool chained, cudaStream_t st) {
   cudaLaunchAttribute attr[1];
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[0].val.programmaticStreamSerializationAllowed = 1;
@@ -773,10 +798,15 @@ cudaError_t launch_nt(const MmaPlan& pl, int grid, const UpParams& up, const Dow
   lc.attrs = attr;
   lc.numAttrs = chained ? 1 : 0;
   lc.dynamicSmemBytes = pl.smem_up;
-  cudaError_t e = cudaLaunchKernelEx(&lc, expert_up_mma_kernel<NT>, up);
+  cudaError_t e = cudaLaunchKernelEx(&lc, expert_up_mma_kernel, up);
   if (e != cudaSuccess) return e;
   lc.dynamicSmemBytes = pl.smem_down;
-  return cudaLaunchKernelEx(&lc, expert_down_mma_kernel<NT>, dn);
+  switch ((dn.L + 7) / 8) {
+    case 1: return cudaLaunchKernelEx(&lc, expert_down_mma_kernel<1>, dn);
+    case 2: return cudaLaunchKernelEx(&lc, expert_down_mma_kernel<2>, dn);
+    case 3: return cudaLaunchKernelEx(&lc, expert_down_mma_kernel<3>, dn);
+    default: return cudaLaunchKernelEx(&lc, expert_down_mma_kernel<4>, dn);
+  }
 }
 
 }  // namespace
@@ -789,13 +819,7 @@ size_t expert_mma_h_bytes(const blockffn_config* cfg) {
   return sizeof(uint16_t) * (size_t)cfg->E * cfg->L_max * cfg->d_e + 256;
 }
 
-cudaError_t expert_mma_setup(blockffn_ctx*) {
-  cudaError_t e = set_attrs<1>();
-  if (e == cudaSuccess) e = set_attrs<2>();
-  if (e == cudaSuccess) e = set_attrs<3>();
-  if (e == cudaSuccess) e = set_attrs<4>();
-  return e;
-}
+cudaError_t expert_mma_setup(blockffn_ctx*) { return set_attrs(); }
 
 cudaError_t launch_expert_mma(blockffn_ctx* c, const blockffn_weights* w, const void* x,
                               const float* scores, int L, const int32_t* union_ids,
@@ -849,13 +873,7 @@ cudaError_t launch_expert_mma(blockffn_ctx* c, const blockffn_weights* w, const 
   dn.accumulate = (call_flags & BLOCKFFN_CALL_ACCUMULATE) ? 1 : 0;
   dn.status = c->status;
   const bool chained = !(c->cfg.flags & BLOCKFFN_CFG_NO_CHAINING);
-  cudaError_t e;
-  switch (pl.NT) {
-    case 1: e = launch_nt<1>(pl, c->num_sms, up, dn, chained, st); break;
-    case 2: e = launch_nt<2>(pl, c->num_sms, up, dn, chained, st); break;
-    case 3: e = launch_nt<3>(pl, c->num_sms, up, dn, chained, st); break;
-    default: e = launch_nt<4>(pl, c->num_sms, up, dn, chained, st); break;
-  }
+  const cudaError_t e = launch_pair(pl, c->num_sms, up, dn, chained, st);
   if (e == cudaSuccess) c->launches += 2;
   return e;
 }
