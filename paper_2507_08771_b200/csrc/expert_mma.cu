@@ -333,6 +333,8 @@ struct UpParams {
 // weights stay in shared memory, the x tile of the next group replaces the current one. That
 // keeps the kernel within half an SM's shared memory for every L, which is what lets it run
 // next to the down kernel of the call before.
+// MULTI: the chunk has more than one token group (L > 8)
+template <bool MULTI>
 __global__ void __launch_bounds__(kThreads, 2) expert_up_mma_kernel(const UpParams p) {
   extern __shared__ __align__(128) unsigned char smem[];
   constexpr int NT = 1;
@@ -345,7 +347,7 @@ __global__ void __launch_bounds__(kThreads, 2) expert_up_mma_kernel(const UpPara
   int* ids_sm = reinterpret_cast<int*>(smem + kOffIds);
   float* red = reinterpret_cast<float*>(smem + lay.off_red);
   const int row_bytes = 2 * d;
-  const int ntg = (L + 7) >> 3;            // token groups
+  const int ntg = MULTI ? (L + 7) >> 3 : 1;   // token groups
 
   if (tid < 8) ctl[tid] = 0;
   if (p.early) {
@@ -396,14 +398,17 @@ __global__ void __launch_bounds__(kThreads, 2) expert_up_mma_kernel(const UpPara
   // (element e = t * 32 + m: token t of the group, row m of the stage).
   float sc = 0.0f;
   int hq = -1, hj = 0;
+  uint16_t held[4] = {0, 0, 0, 0};
   auto prepare = [&](int gi, int tgi) {
     const int ra = r0 + gi * rpg, rows = min(r1, ra + rpg) - ra;
     const int t = 8 * tgi + (tid >> 5), m = tid & 31;
     sc = 0.0f;
     hq = -1;
-    if (t < L && m < rows) {
+    if (m < rows) {          // the row is this thread's for every token group of the stage
       hq = row_q(ra + m);
       hj = ra + m - hq * d_e;
+    }
+    if (t < L && m < rows) {
       const int id = ids_sm[hq];
       if (p.lg.a0 != nullptr) {      // gain * ReLU(logit) / rms, as in derive_union
         float v = __ldcg(p.lg.a0 + (size_t)t * p.E + id);
@@ -472,13 +477,35 @@ __global__ void __launch_bounds__(kThreads, 2) expert_up_mma_kernel(const UpPara
       if (!last_tg) issue_x(tgi + 1);
       else if (gi + 1 < ngroups && ntg > 1) issue_x(0);
       cp_async_commit();
-      if (gi == 0 && tgi == 0 && p.early == 2) pdl_wait();   // h may still be read by the call before
-      if (hq >= 0) {
+      // h may still be read by the down kernel of the call before: when this kernel runs ahead
+      // of it (early == 2), the first stage keeps its results in registers until all its token
+      // groups are done, so that all of that math happens before the wait.
+      const bool hold = MULTI && gi == 0 && p.early == 2;
+      if (!MULTI && gi == 0 && p.early == 2) pdl_wait();
+      uint16_t hval = 0;
+      const bool tok_ok = 8 * tgi + (tid >> 5) < L;
+      if (hq >= 0 && tok_ok) {
         float v = 0.0f;
 #pragma unroll
         for (int w = 0; w < kWarps; ++w) v += red[w * (32 * 8) + tid];
-        p.h[((size_t)hq * L + 8 * tgi + (tid >> 5)) * d_e + hj] =
-            (uint16_t)f32_to_bf16_bits(sc * swish_fast(v));
+        hval = (uint16_t)f32_to_bf16_bits(sc * swish_fast(v));
+      }
+      if (hold) {
+        if (tgi == 0) held[0] = hval;
+        else if (tgi == 1) held[1] = hval;
+        else if (tgi == 2) held[2] = hval;
+        else held[3] = hval;
+        if (last_tg) {
+          pdl_wait();
+          if (hq >= 0) {
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+              if (i < ntg && 8 * i + (tid >> 5) < L)
+                p.h[((size_t)hq * L + 8 * i + (tid >> 5)) * d_e + hj] = held[i];
+          }
+        }
+      } else if (hq >= 0 && tok_ok) {
+        p.h[((size_t)hq * L + 8 * tgi + (tid >> 5)) * d_e + hj] = hval;
       }
       if (!last_tg) prepare(gi, tgi + 1);
       else if (gi + 1 < ngroups) prepare(gi + 1, 0);
@@ -771,7 +798,8 @@ MmaPlan make_plan(const blockffn_config& cfg, int L, int grid) {
 // any CTA runs on it, so a down CTA can only join an up CTA (and the next call's up CTA the
 // down CTA) if the first of them already configured the SM for both.
 cudaError_t set_attrs() {
-  const void* fns[5] = {reinterpret_cast<const void*>(&expert_up_mma_kernel),
+  const void* fns[6] = {reinterpret_cast<const void*>(&expert_up_mma_kernel<false>),
+                        reinterpret_cast<const void*>(&expert_up_mma_kernel<true>),
                         reinterpret_cast<const void*>(&expert_down_mma_kernel<1>),
                         reinterpret_cast<const void*>(&expert_down_mma_kernel<2>),
                         reinterpret_cast<const void*>(&expert_down_mma_kernel<3>),
@@ -798,7 +826,8 @@ cudaError_t launch_pair(const MmaPlan& pl, int grid, const UpParams& up, const D
   lc.attrs = attr;
   lc.numAttrs = chained ? 1 : 0;
   lc.dynamicSmemBytes = pl.smem_up;
-  cudaError_t e = cudaLaunchKernelEx(&lc, expert_up_mma_kernel, up);
+  cudaError_t e = up.L > 8 ? cudaLaunchKernelEx(&lc, expert_up_mma_kernel<true>, up)
+                           : cudaLaunchKernelEx(&lc, expert_up_mma_kernel<false>, up);
   if (e != cudaSuccess) return e;
   lc.dynamicSmemBytes = pl.smem_down;
   switch ((dn.L + 7) / 8) {
