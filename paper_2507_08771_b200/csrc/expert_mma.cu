@@ -145,6 +145,8 @@ __device__ __forceinline__ float swish_fast(float z) { return __fdividef(z, 1.0f
 // ids_in != NULL: taken from the caller's list (E entries are readable); entries out of
 // range are dropped and reported, a count out of range is clamped and reported.
 // tm: scratch of at least L * ceil(E/32) words of shared memory.
+// MODE: 0 from scores, 1 from the caller's list, 2 from raw router logits
+template <int MODE>
 __device__ int derive_union(const float* scores, const RouterLogits& lg, const int32_t* ids_in,
                             const int32_t* n_in, int L, int E, int* ids_sm, int* ctl,
                             uint32_t* tm) {
@@ -155,7 +157,7 @@ __device__ int derive_union(const float* scores, const RouterLogits& lg, const i
   int* act = ctl + 72;
   uint32_t* um = reinterpret_cast<uint32_t*>(ctl + 8);
   float* rinv = reinterpret_cast<float*>(ctl + 104);
-  if (lg.a0 != nullptr) {
+  if constexpr (MODE == 2) {
     // Raw router logits: finish Eq. 3 here (ReLU, RMSNorm over all E entries, gain), with the
     // arithmetic of the router kernel's own normalisation, and take the nonzero pattern.
     for (int t = warp; t < L; t += nwarps) {
@@ -181,7 +183,7 @@ __device__ int derive_union(const float* scores, const RouterLogits& lg, const i
         if (lane == 0) tm[t * words + w] = m;
       }
     }
-  } else if (ids_in == nullptr) {
+  } else if constexpr (MODE == 0) {
     // warp -> tokens warp, warp + nwarps, ...; four mask words in flight per step
     for (int t = warp; t < L; t += nwarps) {
       for (int w0 = 0; w0 < words; w0 += 4) {
@@ -199,7 +201,7 @@ __device__ int derive_union(const float* scores, const RouterLogits& lg, const i
       }
     }
   }
-  if (lg.a0 != nullptr || ids_in == nullptr) {
+  if constexpr (MODE != 1) {
     __syncthreads();
     if (threadIdx.x < words) {
       uint32_t un = 0;
@@ -334,7 +336,7 @@ struct UpParams {
 // keeps the kernel within half an SM's shared memory for every L, which is what lets it run
 // next to the down kernel of the call before.
 // MULTI: the chunk has more than one token group (L > 8)
-template <bool MULTI>
+template <bool MULTI, int MODE>
 __global__ void __launch_bounds__(kThreads, 2) expert_up_mma_kernel(const UpParams p) {
   extern __shared__ __align__(128) unsigned char smem[];
   constexpr int NT = 1;
@@ -357,7 +359,7 @@ __global__ void __launch_bounds__(kThreads, 2) expert_up_mma_kernel(const UpPara
     pdl_trigger();
   }
   __syncthreads();
-  const int nu = derive_union(p.scores, p.lg, p.ids_in, p.n_in, L, p.E, ids_sm, ctl,
+  const int nu = derive_union<MODE>(p.scores, p.lg, p.ids_in, p.n_in, L, p.E, ids_sm, ctl,
                               reinterpret_cast<uint32_t*>(red));
 
   // This CTA's rows [r0, r1) of the u * d_e union rows (balanced: the first R % G CTAs take
@@ -410,7 +412,7 @@ __global__ void __launch_bounds__(kThreads, 2) expert_up_mma_kernel(const UpPara
     }
     if (t < L && m < rows) {
       const int id = ids_sm[hq];
-      if (p.lg.a0 != nullptr) {      // gain * ReLU(logit) / rms, as in derive_union
+      if constexpr (MODE == 2) {     // gain * ReLU(logit) / rms, as in derive_union
         float v = __ldcg(p.lg.a0 + (size_t)t * p.E + id);
         v = v > 0.0f ? v : 0.0f;
         sc = __ldg(p.lg.gain + id) * v * reinterpret_cast<const float*>(ctl + 104)[t];
@@ -575,7 +577,7 @@ struct DownParams {
 };
 
 // NTG: token groups of 8 in the chunk (1 .. 4), each with its own accumulators
-template <int NTG>
+template <int NTG, int MODE>
 __global__ void __launch_bounds__(kThreads, 2) expert_down_mma_kernel(const DownParams p) {
   extern __shared__ __align__(128) unsigned char smem[];
   constexpr int NT = 1;
@@ -594,7 +596,7 @@ __global__ void __launch_bounds__(kThreads, 2) expert_down_mma_kernel(const Down
   pdl_trigger();
   __syncthreads();
   // The routing inputs were final before the up kernel of this call passed its own wait.
-  const int nu = derive_union(p.scores, p.lg, p.ids_in, p.n_in, L, p.E, ids_sm, ctl,
+  const int nu = derive_union<MODE>(p.scores, p.lg, p.ids_in, p.n_in, L, p.E, ids_sm, ctl,
                               reinterpret_cast<uint32_t*>(red));
 
   // Column tiles: G * per tiles of at most max_cols (<= 16) columns, tile w -> CTA w % G,
@@ -797,23 +799,37 @@ MmaPlan make_plan(const blockffn_config& cfg, int L, int grid) {
 // Both kernels ask for the largest shared-memory carve-out: an SM keeps its carve-out while
 // any CTA runs on it, so a down CTA can only join an up CTA (and the next call's up CTA the
 // down CTA) if the first of them already configured the SM for both.
-cudaError_t set_attrs() {
-  const void* fns[6] = {reinterpret_cast<const void*>(&expert_up_mma_kernel<false>),
-                        reinterpret_cast<const void*>(&expert_up_mma_kernel<true>),
-                        reinterpret_cast<const void*>(&expert_down_mma_kernel<1>),
-                        reinterpret_cast<const void*>(&expert_down_mma_kernel<2>),
-                        reinterpret_cast<const void*>(&expert_down_mma_kernel<3>),
-                        reinterpret_cast<const void*>(&expert_down_mma_kernel<4>)};
+cudaError_t set_one(const void* f) {
+  cudaError_t e = cudaFuncSetAttribute(f, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemMax);
+  if (e != cudaSuccess) return e;
+  return cudaFuncSetAttribute(f, cudaFuncAttributePreferredSharedMemoryCarveout,
+                              cudaSharedmemCarveoutMaxShared);
+}
+
+template <int MODE>
+cudaError_t set_attrs_mode() {
+  const void* fns[6] = {reinterpret_cast<const void*>(&expert_up_mma_kernel<false, MODE>),
+                        reinterpret_cast<const void*>(&expert_up_mma_kernel<true, MODE>),
+                        reinterpret_cast<const void*>(&expert_down_mma_kernel<1, MODE>),
+                        reinterpret_cast<const void*>(&expert_down_mma_kernel<2, MODE>),
+                        reinterpret_cast<const void*>(&expert_down_mma_kernel<3, MODE>),
+                        reinterpret_cast<const void*>(&expert_down_mma_kernel<4, MODE>)};
   for (const void* f : fns) {
-    cudaError_t e = cudaFuncSetAttribute(f, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemMax);
-    if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(f, cudaFuncAttributePreferredSharedMemoryCarveout,
-                             cudaSharedmemCarveoutMaxShared);
+    const cudaError_t e = set_one(f);
     if (e != cudaSuccess) return e;
   }
   return cudaSuccess;
 }
 
+cudaError_t set_attrs() {
+  cudaError_t e = set_attrs_mode<0>();
+  if (e == cudaSuccess) e = set_attrs_mode<1>();
+  if (e == cudaSuccess) e = set_attrs_mode<2>();
+  return e;
+}
+
+// One call: the up kernel, then the down kernel, both with the routing mode compiled in.
+template <int MODE>
 cudaError_t launch_pair(const MmaPlan& pl, int grid, const UpParams& up, const DownParams& dn,
                         bool chained, cudaStream_t st) {
   cudaLaunchAttribute attr[1];
@@ -826,15 +842,15 @@ cudaError_t launch_pair(const MmaPlan& pl, int grid, const UpParams& up, const D
   lc.attrs = attr;
   lc.numAttrs = chained ? 1 : 0;
   lc.dynamicSmemBytes = pl.smem_up;
-  cudaError_t e = up.L > 8 ? cudaLaunchKernelEx(&lc, expert_up_mma_kernel<true>, up)
-                           : cudaLaunchKernelEx(&lc, expert_up_mma_kernel<false>, up);
+  cudaError_t e = up.L > 8 ? cudaLaunchKernelEx(&lc, expert_up_mma_kernel<true, MODE>, up)
+                           : cudaLaunchKernelEx(&lc, expert_up_mma_kernel<false, MODE>, up);
   if (e != cudaSuccess) return e;
   lc.dynamicSmemBytes = pl.smem_down;
   switch ((dn.L + 7) / 8) {
-    case 1: return cudaLaunchKernelEx(&lc, expert_down_mma_kernel<1>, dn);
-    case 2: return cudaLaunchKernelEx(&lc, expert_down_mma_kernel<2>, dn);
-    case 3: return cudaLaunchKernelEx(&lc, expert_down_mma_kernel<3>, dn);
-    default: return cudaLaunchKernelEx(&lc, expert_down_mma_kernel<4>, dn);
+    case 1: return cudaLaunchKernelEx(&lc, expert_down_mma_kernel<1, MODE>, dn);
+    case 2: return cudaLaunchKernelEx(&lc, expert_down_mma_kernel<2, MODE>, dn);
+    case 3: return cudaLaunchKernelEx(&lc, expert_down_mma_kernel<3, MODE>, dn);
+    default: return cudaLaunchKernelEx(&lc, expert_down_mma_kernel<4, MODE>, dn);
   }
 }
 
@@ -902,7 +918,9 @@ cudaError_t launch_expert_mma(blockffn_ctx* c, const blockffn_weights* w, const 
   dn.accumulate = (call_flags & BLOCKFFN_CALL_ACCUMULATE) ? 1 : 0;
   dn.status = c->status;
   const bool chained = !(c->cfg.flags & BLOCKFFN_CFG_NO_CHAINING);
-  const cudaError_t e = launch_pair(pl, c->num_sms, up, dn, chained, st);
+  const cudaError_t e = logits      ? launch_pair<2>(pl, c->num_sms, up, dn, chained, st)
+                        : union_ids ? launch_pair<1>(pl, c->num_sms, up, dn, chained, st)
+                                    : launch_pair<0>(pl, c->num_sms, up, dn, chained, st);
   if (e == cudaSuccess) c->launches += 2;
   return e;
 }
