@@ -448,15 +448,17 @@ __global__ void __launch_bounds__(kThreads, 2) expert_up_mma_kernel(const UpPara
     for (int tgi = 0; tgi < ntg; ++tgi) {
       const int nt = min(8, L - 8 * tgi);
       const unsigned char* x_row = smem + lay.off_x + min(g, nt - 1) * row_bytes;
-      // the stage and the x tile of this pass have been requested: wait for all of it
-      cp_async_wait_group<0>();
+      // Every pass ends with two commit groups: the next x tile, then the refill of a ring slot
+      // (either may be empty). The refill is only needed stages later, so all but the newest
+      // group have to have landed; the very first pass waits for everything requested so far.
+      if (gi == 0 && tgi == 0) cp_async_wait_group<0>(); else cp_async_wait_group<1>();
       __syncthreads();
       float a00[NT][4], a01[NT][4], a10[NT][4], a11[NT][4];
       zero_acc<NT>(a00);
       zero_acc<NT>(a01);
       zero_acc<NT>(a10);
       zero_acc<NT>(a11);
-#pragma unroll 2
+#pragma unroll 1
       for (int pp = warp; pp < npairs; pp += kWarps) {
         Frag64 fx[NT];
         fx[0] = load_frag64(x_row + 128 * pp, par, tg);
@@ -475,9 +477,10 @@ __global__ void __launch_bounds__(kThreads, 2) expert_up_mma_kernel(const UpPara
       if (two) store_partial<NT>(mine, 32, 16, a10, a11, g, tg);
       __syncthreads();     // every warp is done with the x tile (and, after the last group, the slot)
       const bool last_tg = tgi + 1 == ntg;
-      if (last_tg && gi + ns < ngroups) issue(gi + ns);
       if (!last_tg) issue_x(tgi + 1);
       else if (gi + 1 < ngroups && ntg > 1) issue_x(0);
+      cp_async_commit();
+      if (last_tg && gi + ns < ngroups) issue(gi + ns);
       cp_async_commit();
       // h may still be read by the down kernel of the call before: when this kernel runs ahead
       // of it (early == 2), the first stage keeps its results in registers until all its token
@@ -679,12 +682,14 @@ __global__ void __launch_bounds__(kThreads, 2) expert_down_mma_kernel(const Down
       if (tgi < ntg) {
         const int nt = min(8, L - 8 * tgi);
         const int h_off = min(g, nt - 1) * row_bytes;
-        // this round's slabs and this pass's h tile have been requested: wait for all of it
-        cp_async_wait_group<0>();
+        // Every pass ends with two commit groups: the next h tile, then the refill of half
+        // the D ring (either may be empty). The refill is only needed two rounds later, so all
+        // but the newest group have to have landed; the first pass waits for everything.
+        if (r == 0 && tgi == 0) cp_async_wait_group<0>(); else cp_async_wait_group<1>();
         __syncthreads();
         if (ncols > 0) {
           // the 64-wide k blocks of the round's experts are dealt round-robin to the warps
-#pragma unroll 2
+#pragma unroll 1
           for (int b = warp; b < nblk; b += kWarps) {
             const int i = pshift >= 0 ? b >> pshift : b / npairs, pp = b - i * npairs;
             const unsigned char* da = d_base + i * lay.slot_d + 128 * pp;
@@ -701,9 +706,10 @@ __global__ void __launch_bounds__(kThreads, 2) expert_down_mma_kernel(const Down
         const bool last_tg = tgi + 1 == ntg;
         if (!last_tg || r + 1 < nrounds) {   // more to fetch into what this pass has read
           __syncthreads();   // every warp is done with the h tile (and, after the last group, the slabs)
-          if (last_tg && r + 2 < nrounds) issue_d();        // refill this round's half of the ring
           if (!last_tg) issue_h(c_rr, tgi + 1);
           else issue_h(c_rr + 1 == rpt ? 0 : c_rr + 1, 0);
+          cp_async_commit();
+          if (last_tg && r + 2 < nrounds) issue_d();        // refill this round's half of the ring
           cp_async_commit();
         }
       }
