@@ -319,8 +319,7 @@ struct UpParams {
   const int32_t* ids_in;   // caller's union list, or NULL: derive from scores / logits
   const int32_t* n_in;
   uint16_t* h;             // bf16 [q][L][d_e] intermediate
-  int L, d, E, d_e, de_shift, ring_rows;   // de_shift: log2(d_e), or -1
-  int early;               // 0: wait first; 1: routing + weights before the wait; 2: x too
+  int L, d, E, d_e, de_shift, ring_rows;   // de_shift: log2(d_e)
   uint32_t* status;
   // what CTA 0 publishes when it derived the union itself (each may be NULL)
   uint32_t* pub_mask;
@@ -336,7 +335,8 @@ struct UpParams {
 // keeps the kernel within half an SM's shared memory for every L, which is what lets it run
 // next to the down kernel of the call before.
 // MULTI: the chunk has more than one token group (L > 8)
-template <bool MULTI, int MODE>
+// EARLY: 0 wait first; 1 routing inputs and weights before the wait; 2 x as well
+template <bool MULTI, int MODE, int EARLY>
 __global__ void __launch_bounds__(kThreads, 2) expert_up_mma_kernel(const UpParams p) {
   extern __shared__ __align__(128) unsigned char smem[];
   constexpr int NT = 1;
@@ -352,7 +352,7 @@ __global__ void __launch_bounds__(kThreads, 2) expert_up_mma_kernel(const UpPara
   const int ntg = MULTI ? (L + 7) >> 3 : 1;   // token groups
 
   if (tid < 8) ctl[tid] = 0;
-  if (p.early) {
+  if constexpr (EARLY != 0) {
     pdl_trigger();       // the next kernel may start fetching its weights right away
   } else {
     pdl_wait();          // scores / ids may come from the kernel just before
@@ -374,7 +374,7 @@ __global__ void __launch_bounds__(kThreads, 2) expert_up_mma_kernel(const UpPara
   const int rpg = ngroups ? (nrows + ngroups - 1) / ngroups : 0;
   const int slot_bytes = slot_rows * row_bytes;
   const int sh = p.de_shift;
-  auto row_q = [&](int r) { return sh >= 0 ? r >> sh : r / d_e; };
+  auto row_q = [&](int r) { return r >> sh; };   // d_e is a power of two
 
   // stage gi: rows [r0 + gi rpg, ...) -> slot gi % ns; one run per expert the rows fall in
   auto issue = [&](int gi) {
@@ -425,13 +425,13 @@ __global__ void __launch_bounds__(kThreads, 2) expert_up_mma_kernel(const UpPara
   const int npairs = d >> 6;   // 64-wide k blocks
 
   const int g_first = min(ngroups, ns);
-  if (p.early) {
+  if constexpr (EARLY != 0) {
     for (int gi = 0; gi < g_first; ++gi) issue(gi);
     if (ngroups > 0) prepare(0, 0);
   }
-  if (p.early < 2) pdl_wait();   // x may come from the kernel just before
+  if constexpr (EARLY < 2) pdl_wait();   // x may come from the kernel just before
   if (ngroups > 0) issue_x(0);
-  if (!p.early) {
+  if constexpr (EARLY == 0) {
     for (int gi = 0; gi < g_first; ++gi) issue(gi);
     if (ngroups > 0) prepare(0, 0);
   }
@@ -485,8 +485,8 @@ __global__ void __launch_bounds__(kThreads, 2) expert_up_mma_kernel(const UpPara
       // h may still be read by the down kernel of the call before: when this kernel runs ahead
       // of it (early == 2), the first stage keeps its results in registers until all its token
       // groups are done, so that all of that math happens before the wait.
-      const bool hold = MULTI && gi == 0 && p.early == 2;
-      if (!MULTI && gi == 0 && p.early == 2) pdl_wait();
+      const bool hold = MULTI && EARLY == 2 && gi == 0;
+      if (!MULTI && EARLY == 2 && gi == 0) pdl_wait();
       uint16_t hval = 0;
       const bool tok_ok = 8 * tgi + (tid >> 5) < L;
       if (hq >= 0 && tok_ok) {
@@ -517,7 +517,7 @@ __global__ void __launch_bounds__(kThreads, 2) expert_up_mma_kernel(const UpPara
       // the next pass starts with a wait and a barrier, which also protects red
     }
   }
-  if (p.early == 2 && ngroups == 0) pdl_wait();   // every kernel waits before it ends
+  if (EARLY == 2 && ngroups == 0) pdl_wait();   // every kernel waits before it ends
   // CTA 0 publishes the routing it derived (after the wait: earlier readers are done)
   if (blockIdx.x == 0) {
     if (p.lg.a0 != nullptr && p.pub_scores != nullptr) {   // the scores and masks it computed
@@ -649,7 +649,7 @@ __global__ void __launch_bounds__(kThreads, 2) expert_down_mma_kernel(const Down
   };
   const int g = lane >> 2, tg = lane & 3, par = g & 1;
   const int npairs = d_e >> 6;         // 64-wide k blocks per expert
-  const int pshift = (npairs & (npairs - 1)) == 0 ? __ffs(npairs) - 1 : -1;
+  const int pshift = __ffs(npairs) - 1;   // d_e, hence npairs, is a power of two
 
   // before the wait: the weights of the first two rounds
   const int npre = min(nrounds, 2);
@@ -691,7 +691,7 @@ __global__ void __launch_bounds__(kThreads, 2) expert_down_mma_kernel(const Down
           // the 64-wide k blocks of the round's experts are dealt round-robin to the warps
 #pragma unroll 1
           for (int b = warp; b < nblk; b += kWarps) {
-            const int i = pshift >= 0 ? b >> pshift : b / npairs, pp = b - i * npairs;
+            const int i = b >> pshift, pp = b - i * npairs;
             const unsigned char* da = d_base + i * lay.slot_d + 128 * pp;
             const unsigned char* ha = h_base + i * hstride + 128 * pp;
             const Frag64 fa = load_frag64(da + off_a, par, tg);
@@ -764,15 +764,15 @@ struct MmaPlan {
   bool ok;
 };
 
-// Shapes the kernels take: d and d_e multiples of 64 (whole 64-wide k blocks, row strides
-// multiples of 128 bytes) and, within half an SM's shared memory, an x tile plus a few rows
+// Shapes the kernels take: d a multiple of 64 and d_e a power of two >= 64 (whole 64-wide k
+// blocks, row strides multiples of 128 bytes, shifts instead of divisions) and, within half an SM's shared memory, an x tile plus a few rows
 // of U (up) and a few expert slabs with their h tiles (down).
 MmaPlan make_plan(const blockffn_config& cfg, int L, int grid) {
   MmaPlan pl{};
   pl.ok = false;
   const int d = cfg.d, d_e = cfg.d_e, E = cfg.E;
   if (L < 1 || L > 32 || grid < 1) return pl;
-  if (d % 64 || d_e % 64 || E > 1024 || d > 32768 || d_e > 4096) return pl;
+  if (d % 64 || d_e % 64 || (d_e & (d_e - 1)) || E > 1024 || d > 32768 || d_e > 4096) return pl;
   const int want_up = cfg.flags & 0xff, want_down = (cfg.flags >> 8) & 0xff;
   // down: column tiles
   pl.per = (d + 16 * grid - 1) / (16 * grid);
@@ -812,11 +812,16 @@ cudaError_t set_one(const void* f) {
                               cudaSharedmemCarveoutMaxShared);
 }
 
+template <int MODE, int EARLY>
+cudaError_t set_attrs_up() {
+  cudaError_t e = set_one(reinterpret_cast<const void*>(&expert_up_mma_kernel<false, MODE, EARLY>));
+  if (e != cudaSuccess) return e;
+  return set_one(reinterpret_cast<const void*>(&expert_up_mma_kernel<true, MODE, EARLY>));
+}
+
 template <int MODE>
-cudaError_t set_attrs_mode() {
-  const void* fns[6] = {reinterpret_cast<const void*>(&expert_up_mma_kernel<false, MODE>),
-                        reinterpret_cast<const void*>(&expert_up_mma_kernel<true, MODE>),
-                        reinterpret_cast<const void*>(&expert_down_mma_kernel<1, MODE>),
+cudaError_t set_attrs_down() {
+  const void* fns[4] = {reinterpret_cast<const void*>(&expert_down_mma_kernel<1, MODE>),
                         reinterpret_cast<const void*>(&expert_down_mma_kernel<2, MODE>),
                         reinterpret_cast<const void*>(&expert_down_mma_kernel<3, MODE>),
                         reinterpret_cast<const void*>(&expert_down_mma_kernel<4, MODE>)};
@@ -828,14 +833,21 @@ cudaError_t set_attrs_mode() {
 }
 
 cudaError_t set_attrs() {
-  cudaError_t e = set_attrs_mode<0>();
-  if (e == cudaSuccess) e = set_attrs_mode<1>();
-  if (e == cudaSuccess) e = set_attrs_mode<2>();
+  cudaError_t e = set_attrs_down<0>();
+  if (e == cudaSuccess) e = set_attrs_down<1>();
+  if (e == cudaSuccess) e = set_attrs_down<2>();
+  if (e == cudaSuccess) e = set_attrs_up<0, 0>();
+  if (e == cudaSuccess) e = set_attrs_up<0, 1>();
+  if (e == cudaSuccess) e = set_attrs_up<0, 2>();
+  if (e == cudaSuccess) e = set_attrs_up<1, 0>();
+  if (e == cudaSuccess) e = set_attrs_up<1, 1>();
+  if (e == cudaSuccess) e = set_attrs_up<1, 2>();
+  if (e == cudaSuccess) e = set_attrs_up<2, 0>();   // raw logits come from the kernel just before
   return e;
 }
 
 // One call: the up kernel, then the down kernel, both with the routing mode compiled in.
-template <int MODE>
+template <int MODE, int EARLY>
 cudaError_t launch_pair(const MmaPlan& pl, int grid, const UpParams& up, const DownParams& dn,
                         bool chained, cudaStream_t st) {
   cudaLaunchAttribute attr[1];
@@ -848,8 +860,8 @@ cudaError_t launch_pair(const MmaPlan& pl, int grid, const UpParams& up, const D
   lc.attrs = attr;
   lc.numAttrs = chained ? 1 : 0;
   lc.dynamicSmemBytes = pl.smem_up;
-  cudaError_t e = up.L > 8 ? cudaLaunchKernelEx(&lc, expert_up_mma_kernel<true, MODE>, up)
-                           : cudaLaunchKernelEx(&lc, expert_up_mma_kernel<false, MODE>, up);
+  cudaError_t e = up.L > 8 ? cudaLaunchKernelEx(&lc, expert_up_mma_kernel<true, MODE, EARLY>, up)
+                           : cudaLaunchKernelEx(&lc, expert_up_mma_kernel<false, MODE, EARLY>, up);
   if (e != cudaSuccess) return e;
   lc.dynamicSmemBytes = pl.smem_down;
   switch ((dn.L + 7) / 8) {
@@ -890,9 +902,7 @@ cudaError_t launch_expert_mma(blockffn_ctx* c, const blockffn_weights* w, const 
   up.E = c->cfg.E;
   up.d_e = c->cfg.d_e;
   up.ring_rows = pl.ring_rows;
-  up.de_shift = (c->cfg.d_e & (c->cfg.d_e - 1)) == 0 ? __builtin_ctz(c->cfg.d_e) : -1;
-  up.early = (call_flags & BLOCKFFN_CALL_INDEPENDENT_X) ? 2
-             : (call_flags & BLOCKFFN_CALL_INDEPENDENT) ? 1 : 0;
+  up.de_shift = __builtin_ctz(c->cfg.d_e);
   up.status = c->status;
   if (pub) {
     up.pub_mask = pub->union_mask;
@@ -924,9 +934,23 @@ cudaError_t launch_expert_mma(blockffn_ctx* c, const blockffn_weights* w, const 
   dn.accumulate = (call_flags & BLOCKFFN_CALL_ACCUMULATE) ? 1 : 0;
   dn.status = c->status;
   const bool chained = !(c->cfg.flags & BLOCKFFN_CFG_NO_CHAINING);
-  const cudaError_t e = logits      ? launch_pair<2>(pl, c->num_sms, up, dn, chained, st)
-                        : union_ids ? launch_pair<1>(pl, c->num_sms, up, dn, chained, st)
-                                    : launch_pair<0>(pl, c->num_sms, up, dn, chained, st);
+  const int early = logits ? 0
+                    : (call_flags & BLOCKFFN_CALL_INDEPENDENT_X) ? 2
+                    : (call_flags & BLOCKFFN_CALL_INDEPENDENT)   ? 1
+                                                                 : 0;
+  const int grid = c->num_sms;
+  cudaError_t e;
+  if (logits) {
+    e = launch_pair<2, 0>(pl, grid, up, dn, chained, st);
+  } else if (union_ids) {
+    e = early == 2   ? launch_pair<1, 2>(pl, grid, up, dn, chained, st)
+        : early == 1 ? launch_pair<1, 1>(pl, grid, up, dn, chained, st)
+                     : launch_pair<1, 0>(pl, grid, up, dn, chained, st);
+  } else {
+    e = early == 2   ? launch_pair<0, 2>(pl, grid, up, dn, chained, st)
+        : early == 1 ? launch_pair<0, 1>(pl, grid, up, dn, chained, st)
+                     : launch_pair<0, 0>(pl, grid, up, dn, chained, st);
+  }
   if (e == cudaSuccess) c->launches += 2;
   return e;
 }
