@@ -179,10 +179,12 @@ class Workload:
         self.d2h_bytes = self.out_host.numel() * 4
 
     # -- the hot path: union + expert FFN per chunk (and per layer for the stack) --
-    def enqueue_step(self, stream):
+    def enqueue_step(self, stream, lo=0, hi=None):
+        """Chunks [lo, hi) of the step."""
         B, lay = self.B, self.layer
+        hi = self.chunks if hi is None else hi
         if self.idx == 4:
-            for c in range(self.chunks):
+            for c in range(lo, hi):
                 # residual stream: out[c] starts as h0 = f32(x[c]); x ping-pongs in bf16
                 self.out[c].copy_(self.x[c])
                 self.x_pp[0].copy_(self.x[c])
@@ -192,7 +194,7 @@ class Workload:
                         self.out[c], self.x_pp[(l + 1) % 2], lay.stats,
                         B.CALL_ACCUMULATE | B.CALL_INDEPENDENT, stream)
         else:
-            for c in range(self.chunks):
+            for c in range(lo, hi):
                 B.blockffn_layer_forward_scores(
                     lay.h, self.dws[c % self.n_copies].struct, self.x[c], self.scores[c, 0], self.L,
                     self.out[c], None, lay.stats, self.call_flags, stream)
@@ -230,6 +232,60 @@ def max_over_ranks(values, world, device=None):
 def job_throughput(world, bytes_per_rank_step, ms_step):
     """Whole-job GB/s: every rank streams bytes_per_rank_step in ms_step (replicas, no collective)."""
     return world * bytes_per_rank_step / (ms_step * 1e-3) / 1e9
+
+
+def time_end_to_end(torch, wl, device, steps, warmup, segments=4):
+    """One step = every chunk's x and scores copied in from pinned host memory, the chunks run
+    through the library, every chunk's output copied back to pinned host memory. The step is cut
+    into segments that flow through three streams (copy in, compute, copy out), so the copies of
+    one segment run under the compute of another; events keep a segment's buffers from being
+    overwritten before they have been consumed. Returns ms per step (device time)."""
+    n = wl.chunks
+    segments = max(1, min(segments, n))
+    bounds = [(i * n // segments, (i + 1) * n // segments) for i in range(segments)]
+    s_in, s_run, s_out = (torch.cuda.Stream(device) for _ in range(3))
+    graphs = [capture(torch, s_run, lambda st, lo=lo, hi=hi: wl.enqueue_step(st, lo, hi))
+              for lo, hi in bounds]
+    x16 = wl.x.view(torch.int16)
+    ev_in = [torch.cuda.Event() for _ in bounds]
+    ev_run = [torch.cuda.Event() for _ in bounds]
+    ev_out = [torch.cuda.Event() for _ in bounds]
+    first = [True]
+
+    def step():
+        for j, (lo, hi) in enumerate(bounds):
+            with torch.cuda.stream(s_in):
+                if not first[0]:
+                    s_in.wait_event(ev_run[j])          # last step's compute has read x, scores
+                x16[lo:hi].copy_(wl.x_host[lo:hi], non_blocking=True)
+                wl.scores[lo:hi].copy_(wl.scores_host[lo:hi], non_blocking=True)
+                ev_in[j].record(s_in)
+            with torch.cuda.stream(s_run):
+                s_run.wait_event(ev_in[j])
+                if not first[0]:
+                    s_run.wait_event(ev_out[j])         # last step's out has been copied back
+                graphs[j].replay()
+                ev_run[j].record(s_run)
+            with torch.cuda.stream(s_out):
+                s_out.wait_event(ev_run[j])
+                wl.out_host[lo:hi].copy_(wl.out[lo:hi], non_blocking=True)
+                ev_out[j].record(s_out)
+        first[0] = False
+
+    for _ in range(warmup):
+        step()
+    torch.cuda.synchronize(device)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(s_in)
+    s_run.wait_event(e0)
+    s_out.wait_event(e0)
+    for _ in range(steps):
+        step()
+    s_in.wait_stream(s_run)
+    s_in.wait_stream(s_out)
+    e1.record(s_in)
+    torch.cuda.synchronize(device)
+    return e0.elapsed_time(e1) / steps
 
 
 def capture(torch, stream, fn):
@@ -378,15 +434,21 @@ def run_ours(args):
     clocks = sampler.stop() if rank == 0 else {}
 
     # end to end: host buffers in, host buffers out, copies inside the timed region
-    def pre():
-        wl.x.view(torch.int16).copy_(wl.x_host, non_blocking=True)
-        wl.scores.copy_(wl.scores_host, non_blocking=True)
-
-    def post():
-        wl.out_host.copy_(wl.out, non_blocking=True)
-
     barrier()
-    ms_e2e = time_replays(torch, stream, g_step, max(3, args.steps // 2), 3, pre, post)
+    ms_e2e = time_end_to_end(torch, wl, device, max(3, args.steps // 2), 3)
+    # one call on its own: enqueued on an idle device, events right around it (launch latency,
+    # cold routing inputs and weights, no overlap with a neighbour)
+    iso = []
+    with torch.cuda.stream(stream):
+        for c in range(min(32, wl.chunks)):
+            stream.synchronize()
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream)
+            wl.enqueue_step(stream, c, c + 1)
+            b.record(stream)
+            stream.synchronize()
+            iso.append(a.elapsed_time(b) * 1e3)
+    isolated_us = float(np.median(iso[4:])) if len(iso) > 4 else float(np.median(iso))
     barrier()
     ms_expert = time_replays(torch, stream, g_expert, args.steps, args.warmup)
     barrier()
@@ -419,6 +481,7 @@ def run_ours(args):
         "data": "synthetic",
         "latency_us_per_chunk": ms_step * 1e3 / wl.chunks,
         "latency_us_per_layer_call": ms_step * 1e3 / calls,
+        "latency_us_isolated_call": isolated_us,
         "pct_of_nominal_8TBs": 100.0 * value / world / NOMINAL_HBM_GBS,
         "config": {
             "workload": f"config {args.config}: {sh.name} (scores-in: chunk union + expert FFN)",
