@@ -160,27 +160,52 @@ __device__ int derive_union(const float* scores, const RouterLogits& lg, const i
   if constexpr (MODE == 2) {
     // Raw router logits: finish Eq. 3 here (ReLU, RMSNorm over all E entries, gain), with the
     // arithmetic of the router kernel's own normalisation, and take the nonzero pattern.
+    // (up to 128 experts a lane keeps its logits and gains in registers: one round trip)
+    const bool few = words <= 4;
     for (int t = warp; t < L; t += nwarps) {
-      float ss = 0.0f;
-      for (int e = lane; e < E; e += 32) {
-        float v = __ldcg(lg.a0 + (size_t)t * E + e);
-        v = v > 0.0f ? v : 0.0f;
-        ss = fmaf(v, v, ss);
+      float ss = 0.0f, v4[4], g4[4];
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const int e = 32 * u + lane;
+        const bool in = few && e < E;
+        v4[u] = in ? __ldcg(lg.a0 + (size_t)t * E + e) : 0.0f;
+        g4[u] = in ? __ldg(lg.gain + e) : 0.0f;
+      }
+      if (few) {
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          v4[u] = v4[u] > 0.0f ? v4[u] : 0.0f;
+          ss = fmaf(v4[u], v4[u], ss);
+        }
+      } else {
+        for (int e = lane; e < E; e += 32) {
+          float v = __ldcg(lg.a0 + (size_t)t * E + e);
+          v = v > 0.0f ? v : 0.0f;
+          ss = fmaf(v, v, ss);
+        }
       }
 #pragma unroll
       for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
       const float r = 1.0f / sqrtf(ss / (float)E + lg.eps);
       if (lane == 0) rinv[t] = r;
-      for (int w = 0; w < words; ++w) {
-        const int e = 32 * w + lane;
-        float s = 0.0f;
-        if (e < E) {
-          float v = __ldcg(lg.a0 + (size_t)t * E + e);
-          v = v > 0.0f ? v : 0.0f;
-          s = __ldg(lg.gain + e) * v * r;
+      if (few) {
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          const uint32_t m = __ballot_sync(0xffffffffu, g4[u] * v4[u] * r != 0.0f);
+          if (lane == 0 && u < words) tm[t * words + u] = m;
         }
-        const uint32_t m = __ballot_sync(0xffffffffu, s != 0.0f);
-        if (lane == 0) tm[t * words + w] = m;
+      } else {
+        for (int w = 0; w < words; ++w) {
+          const int e = 32 * w + lane;
+          float s = 0.0f;
+          if (e < E) {
+            float v = __ldcg(lg.a0 + (size_t)t * E + e);
+            v = v > 0.0f ? v : 0.0f;
+            s = __ldg(lg.gain + e) * v * r;
+          }
+          const uint32_t m = __ballot_sync(0xffffffffu, s != 0.0f);
+          if (lane == 0) tm[t * words + w] = m;
+        }
       }
     }
   } else if constexpr (MODE == 0) {
@@ -355,6 +380,9 @@ __global__ void __launch_bounds__(kThreads, 2) expert_up_mma_kernel(const UpPara
   if constexpr (EARLY != 0) {
     pdl_trigger();       // the next kernel may start fetching its weights right away
   } else {
+    if constexpr (MODE == 2) {   // the gains are weights: have them in L2 when the wait is over
+      if (tid * 32 < p.E) asm volatile("prefetch.global.L2 [%0];" ::"l"(p.lg.gain + tid * 32));
+    }
     pdl_wait();          // scores / ids may come from the kernel just before
     pdl_trigger();
   }
