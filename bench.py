@@ -42,7 +42,7 @@ def parse():
     p.add_argument("--impl", default="ours", choices=["ours", "reference"])
     p.add_argument("--config", type=int, default=1, choices=[1, 2, 3, 4])
     p.add_argument("--L", type=int, default=None, help="chunk length (default: the config's)")
-    p.add_argument("--chunks", type=int, default=256, help="chunks per step")
+    p.add_argument("--chunks", type=int, default=1024, help="chunks per step")
     p.add_argument("--variant", type=int, default=0, help="0 auto, 1 CUDA-core, 2 tensor-core")
     p.add_argument("--flags", type=lambda v: int(v, 0), default=0,
                    help="blockffn_config.flags (ring depths, BLOCKFFN_CFG_* bits)")
@@ -84,10 +84,17 @@ class ClockSampler:
             os.close(fd)
             self.proc = subprocess.Popen(
                 ["nvidia-smi", "-i", str(self.gpu), f"--query-gpu={self.Q}",
-                 "--format=csv,noheader,nounits", "-lms", "100"],
+                 "--format=csv,noheader,nounits", "-lms", "20"],
                 stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
         except Exception:
             self.proc = None
+
+    def mark(self):
+        """Samples taken so far are from before the load started: leave them out."""
+        try:
+            self.skip = sum(1 for _ in open(self.path))
+        except Exception:
+            self.skip = 0
 
     def stop(self):
         out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
@@ -100,7 +107,9 @@ class ClockSampler:
             self.proc.kill()
         sm, mx, reasons = [], [], set()
         try:
-            for line in open(self.path):
+            for k, line in enumerate(open(self.path)):
+                if k < getattr(self, "skip", 0):
+                    continue
                 f = [v.strip() for v in line.split(",")]
                 if len(f) < 9:
                     continue
@@ -425,13 +434,16 @@ def run_ours(args):
     g_expert = capture(torch, stream, wl.enqueue_expert_only)
     expert_launches = (lay.launch_count() - n0) // 2
 
+    # clocks and throttle reasons are sampled (every 20 ms) from before the warm-up replays until
+    # the last timed leg is over: the timed legs run the same kernels back to back
     sampler = ClockSampler(local)
     barrier()
     if rank == 0:
         sampler.start()
+        time.sleep(0.3)          # nvidia-smi needs a moment before its first sample
+        sampler.mark()
     ms_step = time_replays(torch, stream, g_step, args.steps, args.warmup)
     barrier()
-    clocks = sampler.stop() if rank == 0 else {}
 
     # end to end: host buffers in, host buffers out, copies inside the timed region
     barrier()
@@ -452,6 +464,7 @@ def run_ours(args):
     barrier()
     ms_expert = time_replays(torch, stream, g_expert, args.steps, args.warmup)
     barrier()
+    clocks = sampler.stop() if rank == 0 else {}
     status = lay.last_status()
     assert status == 0, f"device status word {status}"
     lay_is_mma = args.variant != 1 and expert_launches // max(wl.calls_per_step, 1) == 2 and sh.d % 64 == 0
@@ -505,7 +518,7 @@ def run_ours(args):
             "algorithmic_bytes_per_launch": alg_bytes, "launches_per_call": expert_launches // calls,
             # dram__bytes_read + write of one up + one down launch (ncu, config 1, see profiles/);
             # other configurations: not captured
-            "traffic": 11144192 if (args.config == 1 and wl.L == 8 and lay_is_mma) else None,
+            "traffic": 11128064 if (args.config == 1 and wl.L == 8 and lay_is_mma) else None,
         },
     }
     if not args.no_cpu_baseline and world == 1:
