@@ -144,7 +144,7 @@ __device__ __forceinline__ float swish_fast(float z) { return __fdividef(z, 1.0f
 // the number of active (token, expert) pairs and ctl[8 ..] the union mask words.
 // ids_in != NULL: taken from the caller's list (E entries are readable); entries out of
 // range are dropped and reported, a count out of range is clamped and reported.
-// tm: scratch of at least L * ceil(E/32) words of shared memory.
+// tm: scratch of at least 32 * ceil(E/32) words of shared memory (word-major, 32 tokens per word).
 // MODE: 0 from scores, 1 from the caller's list, 2 from raw router logits
 template <int MODE>
 __device__ int derive_union(const float* scores, const RouterLogits& lg, const int32_t* ids_in,
@@ -192,7 +192,7 @@ __device__ int derive_union(const float* scores, const RouterLogits& lg, const i
 #pragma unroll
         for (int u = 0; u < 4; ++u) {
           const uint32_t m = __ballot_sync(0xffffffffu, g4[u] * v4[u] * r != 0.0f);
-          if (lane == 0 && u < words) tm[t * words + u] = m;
+          if (lane == 0 && u < words) tm[u * 32 + t] = m;
         }
       } else {
         for (int w = 0; w < words; ++w) {
@@ -204,7 +204,7 @@ __device__ int derive_union(const float* scores, const RouterLogits& lg, const i
             s = __ldg(lg.gain + e) * v * r;
           }
           const uint32_t m = __ballot_sync(0xffffffffu, s != 0.0f);
-          if (lane == 0) tm[t * words + w] = m;
+          if (lane == 0) tm[w * 32 + t] = m;
         }
       }
     }
@@ -221,18 +221,53 @@ __device__ int derive_union(const float* scores, const RouterLogits& lg, const i
 #pragma unroll
         for (int u = 0; u < 4; ++u) {
           const uint32_t m = __ballot_sync(0xffffffffu, v[u] != 0.0f);
-          if (lane == 0 && w0 + u < words) tm[t * words + w0 + u] = m;
+          if (lane == 0 && w0 + u < words) tm[(w0 + u) * 32 + t] = m;
         }
       }
     }
   }
   if constexpr (MODE != 1) {
     __syncthreads();
+    if (words <= 4) {
+      // Up to 128 experts every warp folds the token masks itself (lane t holds token t's
+      // mask of a word; one warp-wide OR per word), so offsets and the union size need no
+      // second exchange through shared memory.
+      uint32_t un[4];
+      int nact = 0;
+#pragma unroll
+      for (int w = 0; w < 4; ++w) {
+        const uint32_t m = (w < words && lane < L) ? tm[w * 32 + lane] : 0u;
+        un[w] = __reduce_or_sync(0xffffffffu, m);
+        nact += __popc(m);
+      }
+      int off = 0, total = 0;
+#pragma unroll
+      for (int w = 0; w < 4; ++w) {
+        if (w < warp) off += __popc(un[w]);
+        total += __popc(un[w]);
+      }
+      if (warp < words) {
+        uint32_t mine = un[0];
+#pragma unroll
+        for (int w = 1; w < 4; ++w) mine = warp == w ? un[w] : mine;
+        if ((mine >> lane) & 1u) ids_sm[off + __popc(mine & ((1u << lane) - 1u))] = 32 * warp + lane;
+      }
+      if (warp == 4) {    // a warp without a word of its own leaves the summary
+        nact = __reduce_add_sync(0xffffffffu, nact);
+        if (lane < 4) um[lane] = lane == 0 ? un[0] : lane == 1 ? un[1] : lane == 2 ? un[2] : un[3];
+        if (lane == 0) {
+          ctl[0] = total;
+          ctl[2] = nact;
+        }
+      }
+      __syncthreads();
+      return total;
+    }
     if (threadIdx.x < words) {
       uint32_t un = 0;
       int nact = 0;
       for (int t = 0; t < L; ++t) {
-        const uint32_t m = tm[t * words + threadIdx.x];
+        const uint32_t m = tm[threadIdx.x * 32 + t];
         un |= m;
         nact += __popc(m);
       }
