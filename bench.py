@@ -559,12 +559,14 @@ class RouterWorkload:
             xs = np.stack([I.make_correlated_x(sh.d, sh.L, rho, seed, chunk=c) for c in range(chunks)])
         self.x = torch.from_numpy(xs.view(np.int16)).to(device).view(torch.bfloat16)
         self.out = torch.zeros(chunks, sh.L, sh.d, dtype=torch.float32, device=device)
+        # the chunks are independent of one another: x never comes from the call before
+        self.call_flags = B.CALL_INDEPENDENT_X
 
     def enqueue_step(self, stream):
         B, lay = self.B, self.layer
         for c in range(self.chunks):
             B.blockffn_layer_forward(lay.h, self.dws[c % len(self.dws)].struct, self.x[c], self.sh.L,
-                                     self.out[c], None, lay.stats, 0, stream)
+                                     self.out[c], None, lay.stats, self.call_flags, stream)
 
     def sparsity(self):
         hs = self.layer.stats_host()

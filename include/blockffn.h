@@ -113,8 +113,10 @@ typedef struct {
 #define BLOCKFFN_CALL_INDEPENDENT_X 4 /* in addition x is stable in the same sense (the chunk does
                                        not consume the previous call's output); implies
                                        BLOCKFFN_CALL_INDEPENDENT. The up projection then runs in full
-                                       under the previous call and only its store waits. Ignored by
-                                       blockffn_layer_forward (its router writes the scores).       */
+                                       under the previous call and only its store waits. In
+                                       blockffn_layer_forward (whose router writes the scores the
+                                       expert stage consumes) the router alone runs ahead: it
+                                       computes the logits under the previous call.                 */
 
 typedef struct blockffn_ctx* blockffn_handle;
 

@@ -69,6 +69,8 @@ blockffn_status blockffn_create(const blockffn_config* cfg, blockffn_handle* out
     return o;
   };
   const size_t o_a0 = take(sizeof(float) * L * E);
+  const size_t o_a0b = take(sizeof(float) * L * E);
+  const size_t o_a0c = take(sizeof(float) * L * E);
   const size_t o_sc = take(sizeof(float) * L * E);
   const size_t o_tm = take(sizeof(uint32_t) * L * W);
   const size_t o_um = take(sizeof(uint32_t) * W);
@@ -92,6 +94,9 @@ blockffn_status blockffn_create(const blockffn_config* cfg, blockffn_handle* out
   char* b = static_cast<char*>(base);
   c->ws_base = base;
   c->a0 = reinterpret_cast<float*>(b + o_a0);
+  c->a0_pair[0] = reinterpret_cast<float*>(b + o_a0b);
+  c->a0_pair[1] = reinterpret_cast<float*>(b + o_a0c);
+  c->a0_phase = 0;
   c->scores = reinterpret_cast<float*>(b + o_sc);
   c->tok_mask = reinterpret_cast<uint32_t*>(b + o_tm);
   c->union_mask = reinterpret_cast<uint32_t*>(b + o_um);
@@ -127,7 +132,7 @@ blockffn_status blockffn_router(blockffn_handle h, const blockffn_weights* w, co
       (reinterpret_cast<uintptr_t>(tok_mask) & 3u))
     return BLOCKFFN_ERR_INVALID_ARG;
   cudaError_t e =
-      launch_router(h, w, x, L, scores, tok_mask, false, nullptr, false,
+      launch_router(h, w, x, L, scores, tok_mask, false, nullptr, false, h->a0, false,
                     static_cast<cudaStream_t>(stream));
   return e == cudaSuccess ? BLOCKFFN_OK : BLOCKFFN_ERR_CUDA;
 }
@@ -180,22 +185,31 @@ blockffn_status blockffn_layer_forward(blockffn_handle h, const blockffn_weights
   if (call_flags & ~kCallFlags)
     return BLOCKFFN_ERR_INVALID_ARG;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  // The router writes the scores this very call consumes: never "independent".
+  // The router writes the scores this very call consumes: the expert kernels are never
+  // "independent". The router itself may run ahead when x is stable.
   const int flags = call_flags & ~(BLOCKFFN_CALL_INDEPENDENT | BLOCKFFN_CALL_INDEPENDENT_X);
   if (use_mma(h, L)) {
     // The router kernel leaves the raw logits; the expert kernels (every CTA needs the union
     // before it can fetch a weight byte) apply ReLU, RMSNorm and gain themselves and CTA 0
     // publishes scores, masks, union and counters.
-    if (launch_router(h, w, x, L, h->scores, h->tok_mask, false, nullptr, true, st) != cudaSuccess)
+    // Successive calls alternate between two logit buffers: a router that runs under the call
+    // before never writes what that call's kernels still read. (Whatever read the other
+    // buffer finished before the previous call's up kernel let anything start behind it:
+    // that kernel waits first, and the router before it waited before it ended.)
+    float* logits = h->a0_pair[h->a0_phase];
+    h->a0_phase ^= 1;
+    const bool x_stable = (call_flags & BLOCKFFN_CALL_INDEPENDENT_X) != 0;
+    if (launch_router(h, w, x, L, h->scores, h->tok_mask, false, nullptr, true, logits, x_stable,
+                      st) != cudaSuccess)
       return BLOCKFFN_ERR_CUDA;
     const RoutingOut pub{h->union_mask, h->union_ids, h->n_union, stats, h->scores, h->tok_mask};
-    const RouterLogits lg{h->a0, w->gain, h->cfg.rms_eps};
+    const RouterLogits lg{logits, w->gain, h->cfg.rms_eps};
     return launch_expert_mma(h, w, x, h->scores, L, nullptr, nullptr, out, x_next, flags, &pub, &lg,
                              st) == cudaSuccess
                ? BLOCKFFN_OK
                : BLOCKFFN_ERR_CUDA;
   }
-  if (launch_router(h, w, x, L, h->scores, h->tok_mask, true, stats, false, st) != cudaSuccess)
+  if (launch_router(h, w, x, L, h->scores, h->tok_mask, true, stats, false, h->a0, false, st) != cudaSuccess)
     return BLOCKFFN_ERR_CUDA;
   return expert_dispatch(h, w, x, h->scores, L, h->union_ids, h->n_union, out, x_next, flags, st);
 }

@@ -15,6 +15,8 @@ struct blockffn_ctx {
   // ---- workspace (device) ----
   void* ws_base;
   float* a0;            // [L_max][E] router logits
+  float* a0_pair[2];    // the two logit buffers blockffn_layer_forward alternates between
+  int a0_phase;         // which of them its next call writes
   float* scores;        // [L_max][E]
   uint32_t* tok_mask;   // [L_max][words]
   uint32_t* union_mask; // [words]
@@ -42,7 +44,8 @@ __device__ __forceinline__ float swish(float z) { return z / (1.0f + __expf(-z))
 // ---- launchers (each returns the cudaError_t of its launch) ----------------
 cudaError_t launch_router(blockffn_ctx* c, const blockffn_weights* w, const void* x, int L,
                           float* scores, uint32_t* tok_mask, bool fuse_union,
-                          blockffn_stats* stats, bool raw, cudaStream_t st);
+                          blockffn_stats* stats, bool raw, float* logits, bool x_stable,
+                          cudaStream_t st);
 cudaError_t launch_chunk_union(blockffn_ctx* c, const float* scores, int L, uint32_t* union_mask,
                                int32_t* union_ids, int32_t* n_union, blockffn_stats* stats,
                                cudaStream_t st);

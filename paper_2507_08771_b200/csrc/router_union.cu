@@ -80,7 +80,7 @@ router_kernel(const uint16_t* __restrict__ x, const uint16_t* __restrict__ W_r,
               const float* __restrict__ gain, const float* __restrict__ bias, float* a0,
               float* scores, uint32_t* tok_mask, int L, int d, int E, float eps,
               unsigned int* ticket, int fuse_union, uint32_t* union_mask, int32_t* union_ids,
-              int32_t* n_union, blockffn_stats* stats, int raw) {
+              int32_t* n_union, blockffn_stats* stats, int raw, int x_stable) {
   __shared__ float red[kWarps][8];
   __shared__ int sm[3 * kMaxWords];
   __shared__ int is_last;
@@ -95,7 +95,15 @@ router_kernel(const uint16_t* __restrict__ x, const uint16_t* __restrict__ W_r,
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   uint4 w_first = make_uint4(0u, 0u, 0u, 0u);
   if ((int)threadIdx.x < chunks) w_first = __ldg(wrow + threadIdx.x);
-  asm volatile("griddepcontrol.wait;" ::: "memory");
+  {  // x may still change until the wait is over, but asking L2 for its lines now is harmless
+    // (L2 is where writes land too); the blocks share the lines out between them
+    const int lines = (L * d * 2 + 127) >> 7;
+    for (int ln = i + (int)gridDim.x * (int)threadIdx.x; ln < lines; ln += gridDim.x * kThreads)
+      asm volatile("prefetch.global.L2 [%0];" ::"l"(reinterpret_cast<const char*>(x) + (size_t)ln * 128));
+  }
+  // x_stable (raw only): x does not come from the work before and a0 is a buffer that work
+  // does not read, so the logits are computed under it; the wait moves to the end.
+  if (!x_stable) asm volatile("griddepcontrol.wait;" ::: "memory");
 
   for (int t0 = 0; t0 < L; t0 += 8) {
     float acc[8];
@@ -104,16 +112,19 @@ router_kernel(const uint16_t* __restrict__ x, const uint16_t* __restrict__ W_r,
     for (int c = threadIdx.x; c < chunks; c += kThreads) {
       const uint4 wv = c == (int)threadIdx.x ? w_first : __ldg(wrow + c);
       const uint32_t wp[4] = {wv.x, wv.y, wv.z, wv.w};
+      // all eight token vectors are requested before the first is used: one memory latency
+      uint4 xv[8];
+#pragma unroll
+      for (int t = 0; t < 8; ++t)
+        xv[t] = t0 + t < L ? __ldcg(reinterpret_cast<const uint4*>(x + (size_t)(t0 + t) * d) + c)
+                           : make_uint4(0u, 0u, 0u, 0u);
 #pragma unroll
       for (int t = 0; t < 8; ++t) {
-        if (t0 + t < L) {
-          const uint4 xv = __ldcg(reinterpret_cast<const uint4*>(x + (size_t)(t0 + t) * d) + c);
-          const uint32_t xp[4] = {xv.x, xv.y, xv.z, xv.w};
+        const uint32_t xp[4] = {xv[t].x, xv[t].y, xv[t].z, xv[t].w};
 #pragma unroll
-          for (int p = 0; p < 4; ++p) {
-            acc[t] = fmaf(bf16_lo(wp[p]), bf16_lo(xp[p]), acc[t]);
-            acc[t] = fmaf(bf16_hi(wp[p]), bf16_hi(xp[p]), acc[t]);
-          }
+        for (int p = 0; p < 4; ++p) {
+          acc[t] = fmaf(bf16_lo(wp[p]), bf16_lo(xp[p]), acc[t]);
+          acc[t] = fmaf(bf16_hi(wp[p]), bf16_hi(xp[p]), acc[t]);
         }
       }
     }
@@ -136,7 +147,11 @@ router_kernel(const uint16_t* __restrict__ x, const uint16_t* __restrict__ W_r,
 
   // raw: the logits are all the caller wants (the tensor-core expert kernels normalise them
   // themselves, which saves this kernel's serial tail)
-  if (raw) return;
+  if (raw) {
+    // every kernel of a chain waits before it ends: completion of one implies all before it
+    if (x_stable) asm volatile("griddepcontrol.wait;" ::: "memory");
+    return;
+  }
   // last block done: normalise. The ticket is reset for the next call.
   __threadfence();
   if (threadIdx.x == 0) {
@@ -182,7 +197,8 @@ router_kernel(const uint16_t* __restrict__ x, const uint16_t* __restrict__ W_r,
 
 cudaError_t launch_router(blockffn_ctx* c, const blockffn_weights* w, const void* x, int L,
                           float* scores, uint32_t* tok_mask, bool fuse_union,
-                          blockffn_stats* stats, bool raw, cudaStream_t st) {
+                          blockffn_stats* stats, bool raw, float* logits, bool x_stable,
+                          cudaStream_t st) {
   cudaLaunchAttribute attr[1];
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[0].val.programmaticStreamSerializationAllowed = 1;
@@ -194,8 +210,9 @@ cudaError_t launch_router(blockffn_ctx* c, const blockffn_weights* w, const void
   lc.numAttrs = (c->cfg.flags & BLOCKFFN_CFG_NO_CHAINING) ? 0 : 1;
   const cudaError_t e = cudaLaunchKernelEx(
       &lc, router_kernel, static_cast<const uint16_t*>(x), static_cast<const uint16_t*>(w->W_r),
-      w->gain, w->bias, c->a0, scores, tok_mask, L, c->cfg.d, c->cfg.E, c->cfg.rms_eps, c->ticket,
-      fuse_union ? 1 : 0, c->union_mask, c->union_ids, c->n_union, stats, raw ? 1 : 0);
+      w->gain, w->bias, logits, scores, tok_mask, L, c->cfg.d, c->cfg.E, c->cfg.rms_eps, c->ticket,
+      fuse_union ? 1 : 0, c->union_mask, c->union_ids, c->n_union, stats, raw ? 1 : 0,
+      (raw && x_stable) ? 1 : 0);
   if (e == cudaSuccess) c->launches += 1;
   return e;
 }

@@ -239,6 +239,42 @@ def test_host_side_argument_errors():
         B.blockffn_layer_forward_scores(layer.h, dw.struct, x, s, 4, out, call_flags=64)
 
 
+@pytest.mark.parametrize("flag", [0, B.CALL_INDEPENDENT_X])
+def test_bench_launch_configuration_router_on(flag):
+    """Back-to-back blockffn_layer_forward calls in a graph; with the promise set the router of a
+    call runs under the expert kernels of the call before it (alternating logit buffers)."""
+    sh, seed = I.SHAPES[3], I.config_seed(3)
+    n_chunks, n_copies = 13, 3                             # odd: replays meet on the same buffer
+    w = I.make_layer(sh, seed, bias_shift=I.ROUTER_BIAS_SHIFT)
+    layer = B.Layer(sh.d, sh.E, sh.d_e, L_max=sh.L)
+    dws = [layer.upload_weights(w) for _ in range(n_copies)]
+    xs = [I.make_x(sh.d, sh.L, seed, chunk=c) for c in range(n_chunks)]
+    xd = [B.to_device_bf16(x) for x in xs]
+    out = torch.full((n_chunks, sh.L, sh.d), float("nan"), device="cuda")
+
+    def enqueue(stream):
+        for c in range(n_chunks):
+            B.blockffn_layer_forward(layer.h, dws[c % n_copies].struct, xd[c], sh.L, out[c], None,
+                                     layer.stats, flag, stream)
+
+    graph_of(enqueue)
+    got = out.cpu().numpy()
+    assert np.isfinite(got).all()
+    checked = 0
+    for c in range(n_chunks):
+        ref = oracle.layer_forward(xs[c], w["W_r"], w["gain"], w["U"], w["D"],
+                                   bias=w.get("bias"), union_only=True)
+        borderline = (np.abs(ref.a0) < FLIP_BAND).any()    # a sign the two sides may disagree on
+        if borderline:
+            continue
+        assert_close(got[c], ref.out, f"router on, flag {flag}, chunk {c}")
+        checked += 1
+    assert checked >= n_chunks // 2
+    hs = layer.stats_host()
+    assert hs.n_chunks == 3 * n_chunks and hs.n_tokens == 3 * n_chunks * sh.L
+    assert layer.last_status() == 0
+
+
 # ----------------------------------------------------------------------------
 # whole layer: the benchmark configurations
 # ----------------------------------------------------------------------------
