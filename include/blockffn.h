@@ -121,7 +121,9 @@ typedef struct {
 typedef struct blockffn_ctx* blockffn_handle;
 
 /* Creates a handle on the current CUDA device and allocates its workspace there
- * (the only allocation the library ever makes). Returns WORKSPACE if that fails. */
+ * (the only allocation the library ever makes), plus one non-blocking stream and a few events
+ * of its own for the router of blockffn_layer_forward (the handle works without them if they
+ * cannot be created). Returns WORKSPACE if the allocation fails.                          */
 BLOCKFFN_API blockffn_status blockffn_create(const blockffn_config* cfg, blockffn_handle* out);
 /* Frees the workspace. The caller synchronises outstanding work first. */
 BLOCKFFN_API blockffn_status blockffn_destroy(blockffn_handle h);
@@ -154,7 +156,14 @@ BLOCKFFN_API blockffn_status blockffn_expert_ffn(blockffn_handle h, const blockf
 
 /* Whole layer, router on: Eq. 3 -> Union(x) -> Eq. 1/2, everything device side.
  * The scores, masks, ids and count land in the handle's workspace
- * (blockffn_read_routing). stats may be NULL.                                            */
+ * (blockffn_read_routing). stats may be NULL.
+ * call_flags: ACCUMULATE as above. With INDEPENDENT_X (x and the weights are stable, see the
+ * flag) the router is launched on the handle's own stream, ordered behind layer calls made a
+ * few calls earlier on `stream` and in front of this call's expert kernels (event record /
+ * wait, also inside a stream capture), so that it runs under the calls before it; the expert
+ * kernels then fetch their weights under the previous call as a scores-in call does. The
+ * first such calls on a stream, or after the stream or its capture changed, keep the router
+ * on `stream`. All work of the call is complete when `stream` has reached its end.        */
 BLOCKFFN_API blockffn_status blockffn_layer_forward(blockffn_handle h, const blockffn_weights* w,
                                                     const void* x, int32_t L, float* out,
                                                     void* x_next, blockffn_stats* stats,

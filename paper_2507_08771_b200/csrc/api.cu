@@ -29,7 +29,7 @@ blockffn_status expert_dispatch(blockffn_ctx* c, const blockffn_weights* w, cons
   cudaError_t e;
   if (use_mma(c, L))
     e = launch_expert_mma(c, w, x, scores, L, union_ids, n_union, out, x_next, call_flags, nullptr,
-                          nullptr, st);
+                          nullptr, false, st);
   else
     e = launch_expert_simt(c, w, x, scores, L, union_ids, n_union, out, x_next, call_flags, st);
   return e == cudaSuccess ? BLOCKFFN_OK : BLOCKFFN_ERR_CUDA;
@@ -38,6 +38,31 @@ blockffn_status expert_dispatch(blockffn_ctx* c, const blockffn_weights* w, cons
 }  // namespace
 
 extern "C" {
+
+// Frees the side stream and its events (those that exist).
+static void release_side(blockffn_ctx* c) {
+  for (int i = 0; i < kLogitRing; ++i) {
+    if (c->ev_call[i]) cudaEventDestroy(c->ev_call[i]);
+    if (c->ev_router[i]) cudaEventDestroy(c->ev_router[i]);
+    c->ev_call[i] = c->ev_router[i] = nullptr;
+  }
+  if (c->side) cudaStreamDestroy(c->side);
+  c->side = nullptr;
+}
+
+// Whether `st` is being captured, and under which capture id. False when that cannot be told.
+static bool capture_state(cudaStream_t st, bool* capturing, unsigned long long* id) {
+  cudaStreamCaptureStatus cs = cudaStreamCaptureStatusNone;
+  unsigned long long cid = 0;
+  if (cudaStreamGetCaptureInfo(st, &cs, &cid) != cudaSuccess) {
+    cudaGetLastError();
+    return false;
+  }
+  if (cs == cudaStreamCaptureStatusInvalidated) return false;
+  *capturing = cs == cudaStreamCaptureStatusActive;
+  *id = *capturing ? cid : 0;
+  return true;
+}
 
 blockffn_status blockffn_create(const blockffn_config* cfg, blockffn_handle* out) {
   if (!cfg || !out) return BLOCKFFN_ERR_INVALID_ARG;
@@ -69,8 +94,8 @@ blockffn_status blockffn_create(const blockffn_config* cfg, blockffn_handle* out
     return o;
   };
   const size_t o_a0 = take(sizeof(float) * L * E);
-  const size_t o_a0b = take(sizeof(float) * L * E);
-  const size_t o_a0c = take(sizeof(float) * L * E);
+  size_t o_ring[kLogitRing];
+  for (int i = 0; i < kLogitRing; ++i) o_ring[i] = take(sizeof(float) * L * E);
   const size_t o_sc = take(sizeof(float) * L * E);
   const size_t o_tm = take(sizeof(uint32_t) * L * W);
   const size_t o_um = take(sizeof(uint32_t) * W);
@@ -94,8 +119,7 @@ blockffn_status blockffn_create(const blockffn_config* cfg, blockffn_handle* out
   char* b = static_cast<char*>(base);
   c->ws_base = base;
   c->a0 = reinterpret_cast<float*>(b + o_a0);
-  c->a0_pair[0] = reinterpret_cast<float*>(b + o_a0b);
-  c->a0_pair[1] = reinterpret_cast<float*>(b + o_a0c);
+  for (int i = 0; i < kLogitRing; ++i) c->a0_ring[i] = reinterpret_cast<float*>(b + o_ring[i]);
   c->a0_phase = 0;
   c->scores = reinterpret_cast<float*>(b + o_sc);
   c->tok_mask = reinterpret_cast<uint32_t*>(b + o_tm);
@@ -111,12 +135,29 @@ blockffn_status blockffn_create(const blockffn_config* cfg, blockffn_handle* out
     delete c;
     return BLOCKFFN_ERR_CUDA;
   }
+  // The stream and events the router of blockffn_layer_forward may run on; without them that
+  // call keeps its router on the caller's stream.
+  c->side = nullptr;
+  c->last_layer_waited_first = false;
+  for (int i = 0; i < kLogitRing; ++i) {
+    c->ev_call[i] = c->ev_router[i] = nullptr;
+    c->call_mark[i].set = false;
+  }
+  bool side_ok = cudaStreamCreateWithFlags(&c->side, cudaStreamNonBlocking) == cudaSuccess;
+  for (int i = 0; i < kLogitRing && side_ok; ++i)
+    side_ok = cudaEventCreateWithFlags(&c->ev_call[i], cudaEventDisableTiming) == cudaSuccess &&
+              cudaEventCreateWithFlags(&c->ev_router[i], cudaEventDisableTiming) == cudaSuccess;
+  if (!side_ok) {
+    cudaGetLastError();
+    release_side(c);
+  }
   *out = c;
   return BLOCKFFN_OK;
 }
 
 blockffn_status blockffn_destroy(blockffn_handle h) {
   if (!h) return BLOCKFFN_ERR_INVALID_ARG;
+  release_side(h);
   cudaError_t e = cudaFree(h->ws_base);
   delete h;
   return e == cudaSuccess ? BLOCKFFN_OK : BLOCKFFN_ERR_CUDA;
@@ -132,7 +173,7 @@ blockffn_status blockffn_router(blockffn_handle h, const blockffn_weights* w, co
       (reinterpret_cast<uintptr_t>(tok_mask) & 3u))
     return BLOCKFFN_ERR_INVALID_ARG;
   cudaError_t e =
-      launch_router(h, w, x, L, scores, tok_mask, false, nullptr, false, h->a0, false,
+      launch_router(h, w, x, L, scores, tok_mask, false, nullptr, false, h->a0, false, true,
                     static_cast<cudaStream_t>(stream));
   return e == cudaSuccess ? BLOCKFFN_OK : BLOCKFFN_ERR_CUDA;
 }
@@ -192,24 +233,65 @@ blockffn_status blockffn_layer_forward(blockffn_handle h, const blockffn_weights
     // The router kernel leaves the raw logits; the expert kernels (every CTA needs the union
     // before it can fetch a weight byte) apply ReLU, RMSNorm and gain themselves and CTA 0
     // publishes scores, masks, union and counters.
-    // Successive calls alternate between two logit buffers: a router that runs under the call
-    // before never writes what that call's kernels still read. (Whatever read the other
-    // buffer finished before the previous call's up kernel let anything start behind it:
-    // that kernel waits first, and the router before it waited before it ended.)
-    float* logits = h->a0_pair[h->a0_phase];
-    h->a0_phase ^= 1;
+    // Successive calls cycle through kLogitRing logit buffers: a router that runs under earlier
+    // calls never writes what their kernels still read.
+    const int b = h->a0_phase;
+    const int oldest = (b + 1) % kLogitRing;   // the call kLogitRing - 1 calls back
+    h->a0_phase = oldest;
+    float* logits = h->a0_ring[b];
     const bool x_stable = (call_flags & BLOCKFFN_CALL_INDEPENDENT_X) != 0;
-    if (launch_router(h, w, x, L, h->scores, h->tok_mask, false, nullptr, true, logits, x_stable,
-                      st) != cudaSuccess)
-      return BLOCKFFN_ERR_CUDA;
+    const bool chained = !(h->cfg.flags & BLOCKFFN_CFG_NO_CHAINING);
     const RoutingOut pub{h->union_mask, h->union_ids, h->n_union, stats, h->scores, h->tok_mask};
     const RouterLogits lg{logits, w->gain, h->cfg.rms_eps};
+    // With x stable the router needs nothing from the caller's stream except that the readers
+    // of its logit buffer (the layer call kLogitRing calls back) are done. It then runs on the
+    // handle's own stream behind the mark that the call kLogitRing - 1 calls back left at its
+    // start, and the expert kernels, which start behind the finished router, fetch their
+    // weights under the previous call like a scores-in call does. The mark must come from the
+    // same stream and the same capture (or both from none); otherwise the router stays on the
+    // caller's stream.
+    bool capturing = false;
+    unsigned long long cap_id = 0;
+    const bool marks = x_stable && chained && h->side && capture_state(st, &capturing, &cap_id);
+    const auto& prev = h->call_mark[oldest];
+    const bool aside = marks && prev.set && prev.stream == st && prev.capturing == capturing &&
+                       prev.id == cap_id;
+    h->call_mark[b].set = false;
+    if (marks && cudaEventRecord(h->ev_call[b], st) == cudaSuccess) {
+      h->call_mark[b].set = true;
+      h->call_mark[b].stream = st;
+      h->call_mark[b].capturing = capturing;
+      h->call_mark[b].id = cap_id;
+    }
+    if (aside) {
+      if (cudaStreamWaitEvent(h->side, h->ev_call[oldest], 0) != cudaSuccess ||
+          launch_router(h, w, x, L, h->scores, h->tok_mask, false, nullptr, true, logits, false,
+                        false, h->side) != cudaSuccess ||
+          cudaEventRecord(h->ev_router[b], h->side) != cudaSuccess ||
+          cudaStreamWaitEvent(st, h->ev_router[b], 0) != cudaSuccess)
+        return BLOCKFFN_ERR_CUDA;
+      h->last_layer_waited_first = false;
+      return launch_expert_mma(h, w, x, h->scores, L, nullptr, nullptr, out, x_next, flags, &pub,
+                               &lg, true, st) == cudaSuccess
+                 ? BLOCKFFN_OK
+                 : BLOCKFFN_ERR_CUDA;
+    }
+    // Router on the caller's stream. It may still compute under the previous call when x is
+    // stable, as long as that call's up kernel waited first: what read this logit buffer then
+    // finished before anything behind that kernel could start (the router before it waited
+    // before it ended, and so does every kernel).
+    const bool ahead = x_stable && h->last_layer_waited_first;
+    h->last_layer_waited_first = true;
+    if (launch_router(h, w, x, L, h->scores, h->tok_mask, false, nullptr, true, logits, ahead,
+                      true, st) != cudaSuccess)
+      return BLOCKFFN_ERR_CUDA;
     return launch_expert_mma(h, w, x, h->scores, L, nullptr, nullptr, out, x_next, flags, &pub, &lg,
-                             st) == cudaSuccess
+                             false, st) == cudaSuccess
                ? BLOCKFFN_OK
                : BLOCKFFN_ERR_CUDA;
   }
-  if (launch_router(h, w, x, L, h->scores, h->tok_mask, true, stats, false, h->a0, false, st) != cudaSuccess)
+  h->last_layer_waited_first = false;
+  if (launch_router(h, w, x, L, h->scores, h->tok_mask, true, stats, false, h->a0, false, true, st) != cudaSuccess)
     return BLOCKFFN_ERR_CUDA;
   return expert_dispatch(h, w, x, h->scores, L, h->union_ids, h->n_union, out, x_next, flags, st);
 }
@@ -233,7 +315,7 @@ blockffn_status blockffn_layer_forward_scores(blockffn_handle h, const blockffn_
     // list before it can fetch a weight byte) and CTA 0 publishes it: no separate launch.
     const RoutingOut pub{h->union_mask, h->union_ids, h->n_union, stats, nullptr, nullptr};
     return launch_expert_mma(h, w, x, scores, L, nullptr, nullptr, out, x_next, call_flags, &pub,
-                             nullptr, st) == cudaSuccess
+                             nullptr, false, st) == cudaSuccess
                ? BLOCKFFN_OK
                : BLOCKFFN_ERR_CUDA;
   }

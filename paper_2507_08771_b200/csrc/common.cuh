@@ -6,6 +6,10 @@
 
 #include "blockffn.h"
 
+// Logit buffers a handle cycles through: the router of a layer call may start as soon as the
+// call kLogitRing - 1 calls earlier has started, i.e. once the readers of its buffer are done.
+constexpr int kLogitRing = 4;
+
 struct blockffn_ctx {
   blockffn_config cfg;
   int device;
@@ -15,8 +19,19 @@ struct blockffn_ctx {
   // ---- workspace (device) ----
   void* ws_base;
   float* a0;            // [L_max][E] router logits
-  float* a0_pair[2];    // the two logit buffers blockffn_layer_forward alternates between
+  float* a0_ring[kLogitRing];   // the logit buffers blockffn_layer_forward cycles through
   int a0_phase;         // which of them its next call writes
+  // ---- router on a stream of its own (blockffn_layer_forward with x stable) ----
+  cudaStream_t side;          // non-blocking; NULL when it could not be created
+  cudaEvent_t ev_call[kLogitRing];     // recorded on the caller's stream at the start of a layer call
+  cudaEvent_t ev_router[kLogitRing];   // recorded on `side` behind the router of a layer call
+  struct {
+    bool set;                 // ev_call[i] holds a record that may be waited for
+    cudaStream_t stream;      // ... made on this stream
+    bool capturing;           // ... inside a stream capture
+    unsigned long long id;    // ... with this capture id
+  } call_mark[kLogitRing];
+  bool last_layer_waited_first;   // the previous layer call's up kernel waited before anything
   float* scores;        // [L_max][E]
   uint32_t* tok_mask;   // [L_max][words]
   uint32_t* union_mask; // [words]
@@ -45,7 +60,7 @@ __device__ __forceinline__ float swish(float z) { return z / (1.0f + __expf(-z))
 cudaError_t launch_router(blockffn_ctx* c, const blockffn_weights* w, const void* x, int L,
                           float* scores, uint32_t* tok_mask, bool fuse_union,
                           blockffn_stats* stats, bool raw, float* logits, bool x_stable,
-                          cudaStream_t st);
+                          bool chained, cudaStream_t st);
 cudaError_t launch_chunk_union(blockffn_ctx* c, const float* scores, int L, uint32_t* union_mask,
                                int32_t* union_ids, int32_t* n_union, blockffn_stats* stats,
                                cudaStream_t st);
@@ -79,4 +94,5 @@ cudaError_t expert_mma_setup(blockffn_ctx* c);
 cudaError_t launch_expert_mma(blockffn_ctx* c, const blockffn_weights* w, const void* x,
                               const float* scores, int L, const int32_t* union_ids,
                               const int32_t* n_union, float* out, void* x_next, int call_flags,
-                              const RoutingOut* pub, const RouterLogits* logits, cudaStream_t st);
+                              const RoutingOut* pub, const RouterLogits* logits, bool logits_final,
+                              cudaStream_t st);

@@ -906,6 +906,7 @@ cudaError_t set_attrs() {
   if (e == cudaSuccess) e = set_attrs_up<1, 1>();
   if (e == cudaSuccess) e = set_attrs_up<1, 2>();
   if (e == cudaSuccess) e = set_attrs_up<2, 0>();   // raw logits come from the kernel just before
+  if (e == cudaSuccess) e = set_attrs_up<2, 2>();   // ... or from a router that has finished
   return e;
 }
 
@@ -950,7 +951,8 @@ cudaError_t expert_mma_setup(blockffn_ctx*) { return set_attrs(); }
 cudaError_t launch_expert_mma(blockffn_ctx* c, const blockffn_weights* w, const void* x,
                               const float* scores, int L, const int32_t* union_ids,
                               const int32_t* n_union, float* out, void* x_next, int call_flags,
-                              const RoutingOut* pub, const RouterLogits* logits, cudaStream_t st) {
+                              const RoutingOut* pub, const RouterLogits* logits, bool logits_final,
+                              cudaStream_t st) {
   const MmaPlan pl = make_plan(c->cfg, L, c->num_sms);
   if (!pl.ok) return cudaErrorNotSupported;
   UpParams up{};
@@ -997,14 +999,16 @@ cudaError_t launch_expert_mma(blockffn_ctx* c, const blockffn_weights* w, const 
   dn.accumulate = (call_flags & BLOCKFFN_CALL_ACCUMULATE) ? 1 : 0;
   dn.status = c->status;
   const bool chained = !(c->cfg.flags & BLOCKFFN_CFG_NO_CHAINING);
-  const int early = logits ? 0
+  // logits_final: the router finished before these kernels could start and x is stable
+  const int early = logits ? (logits_final ? 2 : 0)
                     : (call_flags & BLOCKFFN_CALL_INDEPENDENT_X) ? 2
                     : (call_flags & BLOCKFFN_CALL_INDEPENDENT)   ? 1
                                                                  : 0;
   const int grid = c->num_sms;
   cudaError_t e;
   if (logits) {
-    e = launch_pair<2, 0>(pl, grid, up, dn, chained, st);
+    e = early == 2 ? launch_pair<2, 2>(pl, grid, up, dn, chained, st)
+                   : launch_pair<2, 0>(pl, grid, up, dn, chained, st);
   } else if (union_ids) {
     e = early == 2   ? launch_pair<1, 2>(pl, grid, up, dn, chained, st)
         : early == 1 ? launch_pair<1, 1>(pl, grid, up, dn, chained, st)

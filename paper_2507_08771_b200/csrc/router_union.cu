@@ -198,7 +198,7 @@ router_kernel(const uint16_t* __restrict__ x, const uint16_t* __restrict__ W_r,
 cudaError_t launch_router(blockffn_ctx* c, const blockffn_weights* w, const void* x, int L,
                           float* scores, uint32_t* tok_mask, bool fuse_union,
                           blockffn_stats* stats, bool raw, float* logits, bool x_stable,
-                          cudaStream_t st) {
+                          bool chained, cudaStream_t st) {
   cudaLaunchAttribute attr[1];
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[0].val.programmaticStreamSerializationAllowed = 1;
@@ -207,7 +207,7 @@ cudaError_t launch_router(blockffn_ctx* c, const blockffn_weights* w, const void
   lc.blockDim = dim3(kThreads);
   lc.stream = st;
   lc.attrs = attr;
-  lc.numAttrs = (c->cfg.flags & BLOCKFFN_CFG_NO_CHAINING) ? 0 : 1;
+  lc.numAttrs = (!chained || (c->cfg.flags & BLOCKFFN_CFG_NO_CHAINING)) ? 0 : 1;
   const cudaError_t e = cudaLaunchKernelEx(
       &lc, router_kernel, static_cast<const uint16_t*>(x), static_cast<const uint16_t*>(w->W_r),
       w->gain, w->bias, logits, scores, tok_mask, L, c->cfg.d, c->cfg.E, c->cfg.rms_eps, c->ticket,

@@ -275,6 +275,48 @@ def test_bench_launch_configuration_router_on(flag):
     assert layer.last_status() == 0
 
 
+def test_router_ahead_mixed_sequence():
+    """Layer calls with and without the x-stable promise, a scores-in call in between, eager on one
+    stream: every transition between the router's three launch forms, each result checked."""
+    sh, seed = I.SHAPES[3], I.config_seed(3)
+    w = I.make_layer(sh, seed, bias_shift=I.ROUTER_BIAS_SHIFT)
+    layer = B.Layer(sh.d, sh.E, sh.d_e, L_max=sh.L)
+    dw = layer.upload_weights(w)
+    X = B.CALL_INDEPENDENT_X
+    plan = [X, X, X, X, X, 0, X, X, "scores", X, X, X, X, X, 0, 0, X]
+    xs = [I.make_x(sh.d, sh.L, seed, chunk=100 + c) for c in range(len(plan))]
+    xd = [B.to_device_bf16(x) for x in xs]
+    s_in = I.make_scores(sh.E, sh.L, sh.u, seed, chunk=7)
+    s_dev = dev(s_in)
+    out = torch.full((len(plan), sh.L, sh.d), float("nan"), device="cuda")
+    stream = torch.cuda.Stream()
+    with torch.cuda.stream(stream):
+        for rep in range(2):                               # the second pass starts mid-ring
+            for c, f in enumerate(plan):
+                if f == "scores":
+                    B.blockffn_layer_forward_scores(layer.h, dw.struct, xd[c], s_dev, sh.L, out[c],
+                                                    None, layer.stats, X, stream.cuda_stream)
+                else:
+                    B.blockffn_layer_forward(layer.h, dw.struct, xd[c], sh.L, out[c], None,
+                                             layer.stats, f, stream.cuda_stream)
+        stream.synchronize()
+    got = out.cpu().numpy()
+    assert np.isfinite(got).all()
+    checked = 0
+    for c, f in enumerate(plan):
+        if f == "scores":
+            ref = oracle.layer_forward_scores(xs[c], s_in, w["U"], w["D"], union_only=True)
+        else:
+            ref = oracle.layer_forward(xs[c], w["W_r"], w["gain"], w["U"], w["D"], bias=w["bias"],
+                                       union_only=True)
+            if (np.abs(ref.a0) < FLIP_BAND).any():
+                continue
+        assert_close(got[c], ref.out, f"mixed sequence, call {c} ({f})")
+        checked += 1
+    assert checked >= len(plan) // 2
+    assert layer.last_status() == 0
+
+
 # ----------------------------------------------------------------------------
 # whole layer: the benchmark configurations
 # ----------------------------------------------------------------------------
