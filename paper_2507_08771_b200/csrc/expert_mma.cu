@@ -725,6 +725,13 @@ __global__ void __launch_bounds__(kThreads, 2) expert_down_mma_kernel(const Down
     issue_h(0, 0);
     cp_async_commit();
   }
+  // the residual the first tile's first token group is added to: asked for now, used in the
+  // epilogue (one memory round trip off the tail of the kernel)
+  float resid = 0.0f;
+  if (p.accumulate && tid < 128) {
+    const int t = tid >> 4, m = tid & 15;
+    if (t < L && m < tile_nc(0)) resid = __ldcg(p.out + (size_t)t * d + tile_c0(0) + m);
+  }
 
   float acc0[kMaxTg][4], acc1[kMaxTg][4];
   int c_ti = 0, c_rr = 0;
@@ -792,7 +799,7 @@ __global__ void __launch_bounds__(kThreads, 2) expert_down_mma_kernel(const Down
 #pragma unroll
               for (int w = 0; w < kWarps; ++w) v += red[w * 128 + tid];
               const size_t o = (size_t)t * d + c0 + m;
-              if (p.accumulate) v += __ldcg(p.out + o);
+              if (p.accumulate) v += (c_ti == 0 && tgi == 0) ? resid : __ldcg(p.out + o);
               p.out[o] = v;
               if (p.x_next) p.x_next[o] = (uint16_t)f32_to_bf16_bits(v);
             }
