@@ -173,7 +173,7 @@ blockffn_status blockffn_router(blockffn_handle h, const blockffn_weights* w, co
       (reinterpret_cast<uintptr_t>(tok_mask) & 3u))
     return BLOCKFFN_ERR_INVALID_ARG;
   cudaError_t e =
-      launch_router(h, w, x, L, scores, tok_mask, false, nullptr, false, h->a0, false, true,
+      launch_router(h, w, x, L, scores, tok_mask, false, nullptr, false, h->a0, 0,
                     static_cast<cudaStream_t>(stream));
   return e == cudaSuccess ? BLOCKFFN_OK : BLOCKFFN_ERR_CUDA;
 }
@@ -265,8 +265,8 @@ blockffn_status blockffn_layer_forward(blockffn_handle h, const blockffn_weights
     }
     if (aside) {
       if (cudaStreamWaitEvent(h->side, h->ev_call[oldest], 0) != cudaSuccess ||
-          launch_router(h, w, x, L, h->scores, h->tok_mask, false, nullptr, true, logits, false,
-                        false, h->side) != cudaSuccess ||
+          launch_router(h, w, x, L, h->scores, h->tok_mask, false, nullptr, true, logits, 2,
+                        h->side) != cudaSuccess ||
           cudaEventRecord(h->ev_router[b], h->side) != cudaSuccess ||
           cudaStreamWaitEvent(st, h->ev_router[b], 0) != cudaSuccess)
         return BLOCKFFN_ERR_CUDA;
@@ -282,8 +282,8 @@ blockffn_status blockffn_layer_forward(blockffn_handle h, const blockffn_weights
     // before it ended, and so does every kernel).
     const bool ahead = x_stable && h->last_layer_waited_first;
     h->last_layer_waited_first = true;
-    if (launch_router(h, w, x, L, h->scores, h->tok_mask, false, nullptr, true, logits, ahead,
-                      true, st) != cudaSuccess)
+    if (launch_router(h, w, x, L, h->scores, h->tok_mask, false, nullptr, true, logits,
+                      ahead ? 1 : 0, st) != cudaSuccess)
       return BLOCKFFN_ERR_CUDA;
     return launch_expert_mma(h, w, x, h->scores, L, nullptr, nullptr, out, x_next, flags, &pub, &lg,
                              false, st) == cudaSuccess
@@ -291,7 +291,7 @@ blockffn_status blockffn_layer_forward(blockffn_handle h, const blockffn_weights
                : BLOCKFFN_ERR_CUDA;
   }
   h->last_layer_waited_first = false;
-  if (launch_router(h, w, x, L, h->scores, h->tok_mask, true, stats, false, h->a0, false, true, st) != cudaSuccess)
+  if (launch_router(h, w, x, L, h->scores, h->tok_mask, true, stats, false, h->a0, 0, st) != cudaSuccess)
     return BLOCKFFN_ERR_CUDA;
   return expert_dispatch(h, w, x, h->scores, L, h->union_ids, h->n_union, out, x_next, flags, st);
 }

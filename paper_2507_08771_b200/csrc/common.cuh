@@ -59,8 +59,11 @@ __device__ __forceinline__ float swish(float z) { return z / (1.0f + __expf(-z))
 // ---- launchers (each returns the cudaError_t of its launch) ----------------
 cudaError_t launch_router(blockffn_ctx* c, const blockffn_weights* w, const void* x, int L,
                           float* scores, uint32_t* tok_mask, bool fuse_union,
-                          blockffn_stats* stats, bool raw, float* logits, bool x_stable,
-                          bool chained, cudaStream_t st);
+                          blockffn_stats* stats, bool raw, float* logits, int mode,
+                          cudaStream_t st);
+// mode: 0 the kernel waits for the work before it first; 1 (raw only) it computes under that
+// work and waits at its end; 2 (raw only) it is launched without programmatic chaining on a
+// stream of its own and lets its dependents go only by exiting, behind a fence.
 cudaError_t launch_chunk_union(blockffn_ctx* c, const float* scores, int L, uint32_t* union_mask,
                                int32_t* union_ids, int32_t* n_union, blockffn_stats* stats,
                                cudaStream_t st);

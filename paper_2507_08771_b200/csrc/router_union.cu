@@ -80,7 +80,7 @@ router_kernel(const uint16_t* __restrict__ x, const uint16_t* __restrict__ W_r,
               const float* __restrict__ gain, const float* __restrict__ bias, float* a0,
               float* scores, uint32_t* tok_mask, int L, int d, int E, float eps,
               unsigned int* ticket, int fuse_union, uint32_t* union_mask, int32_t* union_ids,
-              int32_t* n_union, blockffn_stats* stats, int raw, int x_stable) {
+              int32_t* n_union, blockffn_stats* stats, int raw, int mode) {
   __shared__ float red[kWarps][8];
   __shared__ int sm[3 * kMaxWords];
   __shared__ int is_last;
@@ -92,7 +92,9 @@ router_kernel(const uint16_t* __restrict__ x, const uint16_t* __restrict__ W_r,
   // The kernel may have been started while the work before it on the stream still runs
   // (programmatic dependent launch): the router weights are stable and are requested now,
   // x and everything this kernel writes are touched only after the wait.
-  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  // mode 2 (raw, launched on a stream of its own): dependents are let go only by the exit of
+  // the blocks, behind a fence, because they read the logits without waiting (see the end).
+  if (mode != 2) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   uint4 w_first = make_uint4(0u, 0u, 0u, 0u);
   if ((int)threadIdx.x < chunks) w_first = __ldg(wrow + threadIdx.x);
   {  // x may still change until the wait is over, but asking L2 for its lines now is harmless
@@ -101,9 +103,9 @@ router_kernel(const uint16_t* __restrict__ x, const uint16_t* __restrict__ W_r,
     for (int ln = i + (int)gridDim.x * (int)threadIdx.x; ln < lines; ln += gridDim.x * kThreads)
       asm volatile("prefetch.global.L2 [%0];" ::"l"(reinterpret_cast<const char*>(x) + (size_t)ln * 128));
   }
-  // x_stable (raw only): x does not come from the work before and a0 is a buffer that work
+  // mode 1 (raw only): x does not come from the work before and a0 is a buffer that work
   // does not read, so the logits are computed under it; the wait moves to the end.
-  if (!x_stable) asm volatile("griddepcontrol.wait;" ::: "memory");
+  if (mode == 0) asm volatile("griddepcontrol.wait;" ::: "memory");
 
   for (int t0 = 0; t0 < L; t0 += 8) {
     float acc[8];
@@ -149,7 +151,12 @@ router_kernel(const uint16_t* __restrict__ x, const uint16_t* __restrict__ W_r,
   // themselves, which saves this kernel's serial tail)
   if (raw) {
     // every kernel of a chain waits before it ends: completion of one implies all before it
-    if (x_stable) asm volatile("griddepcontrol.wait;" ::: "memory");
+    if (mode == 1) asm volatile("griddepcontrol.wait;" ::: "memory");
+    // mode 2: a kernel launched with the programmatic attribute treats every kernel it depends
+    // on as a programmatic prerequisite, event edges from other streams included, so the expert
+    // kernels may start as soon as this grid's blocks have exited. The fence makes each block's
+    // logits visible device-wide before that exit.
+    if (mode == 2) __threadfence();
     return;
   }
   // last block done: normalise. The ticket is reset for the next call.
@@ -197,8 +204,8 @@ router_kernel(const uint16_t* __restrict__ x, const uint16_t* __restrict__ W_r,
 
 cudaError_t launch_router(blockffn_ctx* c, const blockffn_weights* w, const void* x, int L,
                           float* scores, uint32_t* tok_mask, bool fuse_union,
-                          blockffn_stats* stats, bool raw, float* logits, bool x_stable,
-                          bool chained, cudaStream_t st) {
+                          blockffn_stats* stats, bool raw, float* logits, int mode,
+                          cudaStream_t st) {
   cudaLaunchAttribute attr[1];
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[0].val.programmaticStreamSerializationAllowed = 1;
@@ -207,12 +214,12 @@ cudaError_t launch_router(blockffn_ctx* c, const blockffn_weights* w, const void
   lc.blockDim = dim3(kThreads);
   lc.stream = st;
   lc.attrs = attr;
-  lc.numAttrs = (!chained || (c->cfg.flags & BLOCKFFN_CFG_NO_CHAINING)) ? 0 : 1;
+  lc.numAttrs = (mode == 2 || (c->cfg.flags & BLOCKFFN_CFG_NO_CHAINING)) ? 0 : 1;
   const cudaError_t e = cudaLaunchKernelEx(
       &lc, router_kernel, static_cast<const uint16_t*>(x), static_cast<const uint16_t*>(w->W_r),
       w->gain, w->bias, logits, scores, tok_mask, L, c->cfg.d, c->cfg.E, c->cfg.rms_eps, c->ticket,
       fuse_union ? 1 : 0, c->union_mask, c->union_ids, c->n_union, stats, raw ? 1 : 0,
-      (raw && x_stable) ? 1 : 0);
+      raw ? mode : 0);
   if (e == cudaSuccess) c->launches += 1;
   return e;
 }
