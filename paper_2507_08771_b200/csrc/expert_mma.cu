@@ -488,17 +488,36 @@ __global__ void __launch_bounds__(kThreads, 2) expert_up_mma_kernel(const UpPara
   const int npairs = d >> 6;   // 64-wide k blocks
 
   const int g_first = min(ngroups, ns);
-  if constexpr (EARLY != 0) {
-    for (int gi = 0; gi < g_first; ++gi) issue(gi);
+  // DEEP (one token group, x not later than the weights): every stage is a commit group of its
+  // own, x rides with the first, and a pass waits for its own stage only, so that up to
+  // ns - 1 later stages stay in flight under its math. Otherwise the first pass waits for
+  // everything requested so far and later passes for all but the newest group.
+  constexpr bool DEEP = !MULTI && EARLY != 1;
+  if constexpr (DEEP) {
+    if constexpr (EARLY == 0) pdl_wait();   // x may come from the kernel just before
+    if (ngroups > 0) {
+      issue_x(0);
+      issue(0);
+    }
+    cp_async_commit();
+    for (int gi = 1; gi < g_first; ++gi) {
+      issue(gi);
+      cp_async_commit();
+    }
     if (ngroups > 0) prepare(0, 0);
+  } else {
+    if constexpr (EARLY != 0) {
+      for (int gi = 0; gi < g_first; ++gi) issue(gi);
+      if (ngroups > 0) prepare(0, 0);
+    }
+    if constexpr (EARLY < 2) pdl_wait();   // x may come from the kernel just before
+    if (ngroups > 0) issue_x(0);
+    if constexpr (EARLY == 0) {
+      for (int gi = 0; gi < g_first; ++gi) issue(gi);
+      if (ngroups > 0) prepare(0, 0);
+    }
+    cp_async_commit();
   }
-  if constexpr (EARLY < 2) pdl_wait();   // x may come from the kernel just before
-  if (ngroups > 0) issue_x(0);
-  if constexpr (EARLY == 0) {
-    for (int gi = 0; gi < g_first; ++gi) issue(gi);
-    if (ngroups > 0) prepare(0, 0);
-  }
-  cp_async_commit();
 
   for (int gi = 0; gi < ngroups; ++gi) {
     const int rows = min(r1, r0 + (gi + 1) * rpg) - (r0 + gi * rpg);
@@ -514,7 +533,14 @@ __global__ void __launch_bounds__(kThreads, 2) expert_up_mma_kernel(const UpPara
       // Every pass ends with two commit groups: the next x tile, then the refill of a ring slot
       // (either may be empty). The refill is only needed stages later, so all but the newest
       // group have to have landed; the very first pass waits for everything requested so far.
-      if (gi == 0 && tgi == 0) cp_async_wait_group<0>(); else cp_async_wait_group<1>();
+      if constexpr (DEEP) {
+        // one group per stage and per pass: all but the g_first - 1 newest have to have landed
+        if (g_first >= 3) cp_async_wait_group<2>();
+        else if (g_first == 2) cp_async_wait_group<1>();
+        else cp_async_wait_group<0>();
+      } else {
+        if (gi == 0 && tgi == 0) cp_async_wait_group<0>(); else cp_async_wait_group<1>();
+      }
       __syncthreads();
       float a00[NT][4], a01[NT][4], a10[NT][4], a11[NT][4];
       zero_acc<NT>(a00);
@@ -540,9 +566,11 @@ __global__ void __launch_bounds__(kThreads, 2) expert_up_mma_kernel(const UpPara
       if (two) store_partial<NT>(mine, 32, 16, a10, a11, g, tg);
       __syncthreads();     // every warp is done with the x tile (and, after the last group, the slot)
       const bool last_tg = tgi + 1 == ntg;
-      if (!last_tg) issue_x(tgi + 1);
-      else if (gi + 1 < ngroups && ntg > 1) issue_x(0);
-      cp_async_commit();
+      if constexpr (!DEEP) {
+        if (!last_tg) issue_x(tgi + 1);
+        else if (gi + 1 < ngroups && ntg > 1) issue_x(0);
+        cp_async_commit();
+      }
       if (last_tg && gi + ns < ngroups) issue(gi + ns);
       cp_async_commit();
       // h may still be read by the down kernel of the call before: when this kernel runs ahead
