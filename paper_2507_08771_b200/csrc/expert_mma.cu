@@ -506,12 +506,19 @@ __global__ void __launch_bounds__(kThreads, 2) expert_up_mma_kernel(const UpPara
     }
     if (ngroups > 0) prepare(0, 0);
   } else {
+    // (x, when it is stable, goes first: its short round trip then runs under the long issue
+    // of the weights instead of behind it)
+    if constexpr (EARLY == 2) {
+      if (ngroups > 0) issue_x(0);
+    }
     if constexpr (EARLY != 0) {
       for (int gi = 0; gi < g_first; ++gi) issue(gi);
       if (ngroups > 0) prepare(0, 0);
     }
     if constexpr (EARLY < 2) pdl_wait();   // x may come from the kernel just before
-    if (ngroups > 0) issue_x(0);
+    if constexpr (EARLY < 2) {
+      if (ngroups > 0) issue_x(0);
+    }
     if constexpr (EARLY == 0) {
       for (int gi = 0; gi < g_first; ++gi) issue(gi);
       if (ngroups > 0) prepare(0, 0);
