@@ -518,7 +518,7 @@ def run_ours(args):
             "algorithmic_bytes_per_launch": alg_bytes, "launches_per_call": expert_launches // calls,
             # dram__bytes_read + write of one up + one down launch (ncu, config 1, see profiles/);
             # other configurations: not captured
-            "traffic": 11128320 if (args.config == 1 and wl.L == 8 and lay_is_mma) else None,
+            "traffic": 11130112 if (args.config == 1 and wl.L == 8 and lay_is_mma) else None,
         },
     }
     if not args.no_cpu_baseline and world == 1:
