@@ -573,9 +573,49 @@ class RouterWorkload:
         return (self.B.blockffn_tls(hs, self.sh.E), 1.0 - self.B.blockffn_cls(hs, self.sh.E))
 
 
+def read_ceilings(args, torch, device, B):
+    """What a plain read reaches on this device (blockffn_probe_read: 128-bit loads, four CTAs per
+    SM, data discarded): streaming over 2 GiB, and single launches the size of one call's active
+    weights, back to back over memory that is not in L2, launched plainly and chained like the
+    library's own kernels."""
+    nbytes = 2 << 30
+    buf = torch.empty(nbytes, dtype=torch.uint8, device=device)
+    buf.fill_(1)
+    stream = torch.cuda.Stream(device)
+    steps = max(3, args.steps // 2)
+
+    def enqueue_stream(st):
+        for _ in range(4):
+            B.blockffn_probe_read(buf, nbytes, False, st)
+
+    g = capture(torch, stream, enqueue_stream)
+    ms = time_replays(torch, stream, g, steps, 2)
+    out = {"streaming_read_GBps": 4 * nbytes / ms / 1e6, "streaming_bytes": nbytes}
+    rows = []
+    for cfg_index in (1, 2):
+        sh = I.SHAPES[cfg_index]
+        size = sh.u * 2 * sh.d_e * sh.d * 2            # the active weights of one call
+        n = min(128, nbytes // size)
+        base = buf.data_ptr()
+        row = {"config": cfg_index, "bytes_per_launch": size, "launches": n}
+        for name, chained in (("plain", False), ("chained", True)):
+            def enqueue(st, chained=chained):
+                for i in range(n):
+                    B.blockffn_probe_read(base + i * size, size, chained, st)
+            g = capture(torch, stream, enqueue)
+            us = time_replays(torch, stream, g, steps, 2) * 1e3 / n
+            row[name] = {"us_per_launch": us, "GBps": size / us / 1e3}
+        rows.append(row)
+    out["size_matched"] = rows
+    del buf
+    torch.cuda.empty_cache()
+    return out
+
+
 def extras(args, torch, device, peak):
     """The other configurations, each as us per call and GB/s of active expert bytes."""
-    out = {}
+    from paper_2507_08771_b200 import binding as B
+    out = {"read_ceilings": read_ceilings(args, torch, device, B)}
     chunks = min(args.chunks, 64)
 
     def timed(wl):

@@ -33,6 +33,7 @@
 #ifndef BLOCKFFN_H_
 #define BLOCKFFN_H_
 
+#include <stddef.h>
 #include <stdint.h>
 
 #ifdef __cplusplus
@@ -229,6 +230,18 @@ BLOCKFFN_API blockffn_status blockffn_expert_ffn_noalloc(
     const blockffn_config* cfg, const blockffn_weights* w, const void* x, const float* scores,
     int32_t L, const int32_t* union_ids, const int32_t* n_union, float* out, void* x_next,
     int32_t call_flags, void* stream);
+
+/* Measurement aid; the paper has no counterpart. Enqueues one kernel that reads `bytes` bytes at
+ * `src` (device memory, 16-byte aligned, a multiple of 16 bytes) once, with 128-bit loads from
+ * four CTAs per SM, and discards them: what a plain read of that many bytes costs on the
+ * device it runs on. The benchmark uses it for its read-only ceilings (streaming over
+ * gigabytes; one launch the size of a call's active weights, back to back over cold memory).
+ * chained != 0 launches it with programmatic dependent launch like the library's own kernels
+ * (it starts under the launch before it and waits for it before it ends). Needs no handle,
+ * allocates nothing. INVALID_ARG for a NULL or misaligned src or a size that is 0 or not a
+ * multiple of 16.                                                                          */
+BLOCKFFN_API blockffn_status blockffn_probe_read(const void* src, size_t bytes, int32_t chained,
+                                                 void* stream);
 
 /* Human-readable name of a status code (static storage). */
 BLOCKFFN_API const char* blockffn_status_string(blockffn_status s);

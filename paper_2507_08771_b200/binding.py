@@ -30,6 +30,7 @@ EXPORTS = [
     "blockffn_expert_ffn", "blockffn_layer_forward", "blockffn_layer_forward_scores",
     "blockffn_read_routing", "blockffn_last_status", "blockffn_tls", "blockffn_cls",
     "blockffn_launch_count", "blockffn_status_string", "blockffn_expert_ffn_noalloc",
+    "blockffn_probe_read",
 ]
 NOALLOC_SCRATCH_BYTES = 1 << 20
 
@@ -78,6 +79,7 @@ def load():
     lib.blockffn_read_routing.argtypes = [vp, i32, vp, vp, vp, vp, vp, vp]
     lib.blockffn_expert_ffn_noalloc.argtypes = [ctypes.POINTER(Config), ctypes.POINTER(Weights), vp,
                                                 vp, i32, vp, vp, vp, vp, i32, vp]
+    lib.blockffn_probe_read.argtypes = [vp, ctypes.c_size_t, i32, vp]
     lib.blockffn_last_status.argtypes = [vp, ctypes.POINTER(ctypes.c_uint32), i32, vp]
     lib.blockffn_tls.argtypes = [ctypes.POINTER(Stats), i32]
     lib.blockffn_tls.restype = ctypes.c_double
@@ -160,6 +162,12 @@ def blockffn_expert_ffn_noalloc(cfg: Config, w: Weights, x, scores, L, union_ids
                                               _ptr(scores), L, _ptr(union_ids), _ptr(n_union),
                                               _ptr(out), _ptr(x_next), call_flags,
                                               _stream(stream)), "blockffn_expert_ffn_noalloc")
+
+
+def blockffn_probe_read(src, nbytes, chained=False, stream=None):
+    """Measurement aid: one kernel that reads nbytes at src (device) once and discards them."""
+    _check(load().blockffn_probe_read(_ptr(src), int(nbytes), 1 if chained else 0, _stream(stream)),
+           "blockffn_probe_read")
 
 
 def blockffn_layer_forward(h, w: Weights, x, L, out, x_next=None, stats=None, call_flags=0,

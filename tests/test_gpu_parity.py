@@ -525,3 +525,13 @@ def test_bench_launch_configuration_stack():
     drift = np.abs(got - r).max() / rms(r)
     assert np.isfinite(got).all() and drift <= 1e-1, drift
     assert layer.last_status() == 0
+
+
+def test_probe_read_runs_and_checks_its_arguments():
+    buf = torch.zeros(1 << 22, dtype=torch.uint8, device="cuda")
+    B.blockffn_probe_read(buf, buf.numel())
+    B.blockffn_probe_read(buf, 4096, chained=True)
+    torch.cuda.synchronize()
+    for src, n in ((buf.data_ptr() + 8, 4096), (buf, 100), (buf, 0), (None, 4096)):
+        with pytest.raises(B.BlockFFNError):
+            B.blockffn_probe_read(src, n)
