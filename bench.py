@@ -670,15 +670,40 @@ def extras(args, torch, device, peak):
     sweep_rows, dense_us = [], None
     for frac in (1.0, 0.9, 0.8, 0.7, 0.6, 0.5, 0.4, 0.3, 0.2, 0.1):
         u = int(round(frac * sh.E))
-        wl = Workload(3, sh.L, chunks, 0, device, args.flags, u=u)
-        us = timed(wl) * 1e3 / wl.calls_per_step
+        # each point is timed twice: with the library's default assumption about the union
+        # (30 % of the experts) and with the point's own union size given as the handle's hint
+        row = {"union_frac": frac, "u": u}
+        for key, hint in (("default", 0), ("hinted", B.cfg_expected_union(u))):
+            wl = Workload(3, sh.L, chunks, 0, device, args.flags | hint, u=u)
+            row[key] = {"us_per_call": timed(wl) * 1e3 / wl.calls_per_step}
+            row[key]["GBps"] = wl.active_bytes / row[key]["us_per_call"] / 1e3
+            del wl
+            torch.cuda.empty_cache()
+        us = min(row["default"]["us_per_call"], row["hinted"]["us_per_call"])
         dense_us = us if dense_us is None else dense_us
-        sweep_rows.append({"union_frac": frac, "u": u, "us_per_call": us,
-                           "GBps": wl.active_bytes / us / 1e3, "time_vs_dense": us / dense_us})
-        del wl
-        torch.cuda.empty_cache()
+        row.update({"us_per_call": us, "GBps": u * sh.expert_bytes / us / 1e3,
+                    "time_vs_dense": us / dense_us})
+        sweep_rows.append(row)
     full["union_sweep"] = sweep_rows
     out["config3_full_layer"] = full
+
+    # beyond the benchmark's list: the paper's largest FFN shape at its kernel table's operating
+    # points (32 tree tokens over a 30.86 % union, one token with 12.45 % active), against the
+    # dense layer of the same shape
+    sh5 = I.SHAPES[5]
+    u1 = int(round(I.PAPER_ONE_TOKEN_ACTIVE * sh5.E))
+    rows = {}
+    for name, L, u in (("tree_32_tokens", 32, sh5.u), ("dense_32_tokens", 32, sh5.E),
+                       ("one_token", 1, u1), ("dense_one_token", 1, sh5.E)):
+        wl = Workload(5, L, min(chunks, 16), 0, device, args.flags | B.cfg_expected_union(u), u=u)
+        us = timed(wl) * 1e3 / wl.calls_per_step
+        rows[name] = {"L": L, "u": u, "E": sh5.E, "us_per_call": us,
+                      "GBps": wl.active_bytes / us / 1e3}
+        del wl
+        torch.cuda.empty_cache()
+    rows["tree_time_vs_dense"] = rows["tree_32_tokens"]["us_per_call"] / rows["dense_32_tokens"]["us_per_call"]
+    rows["one_token_time_vs_dense"] = rows["one_token"]["us_per_call"] / rows["dense_one_token"]["us_per_call"]
+    out["paper_2p8b_shape"] = rows
 
     # config 4: 24-layer stack, residual between layers
     wl = Workload(4, None, min(args.chunks, I.STACK_CHUNKS), 0, device, args.flags)

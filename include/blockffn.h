@@ -81,6 +81,14 @@ typedef struct {
  * weights while the kernel enqueued before it on the stream is still finishing
  * (programmatic dependent launch); this bit launches them fully serialised instead. */
 #define BLOCKFFN_CFG_NO_CHAINING 0x10000
+/* How many experts the caller expects in a chunk's union (1 .. E), bits 17-27 of flags. The
+ * tensor-core kernels size their shared memory before the union is known: when the expected
+ * union's share fits half an SM, two kernels share an SM and consecutive launches overlap
+ * (best for the paper's operating points); a larger expected union gives each kernel a whole
+ * SM and fewer, larger stages instead. 0 = assume the paper's sparsity: 30 % of the experts
+ * for a chunk (CLS of Table "moe-ppl"), 12.5 % for a single token (Sec. 4.4). The hint only
+ * changes speed; any union size gives the same results under any hint.                     */
+#define BLOCKFFN_CFG_EXPECTED_UNION(u) (((u) & 0x7ff) << 17)
 
 /* Layer parameters: device pointers, caller-owned, read-only to the library. */
 typedef struct {

@@ -25,6 +25,11 @@ VARIANT_AUTO, VARIANT_SIMT, VARIANT_MMA = 0, 1, 2
 CALL_ACCUMULATE, CALL_INDEPENDENT, CALL_INDEPENDENT_X = 1, 2, 4
 CFG_NO_CHAINING = 0x10000
 
+
+def cfg_expected_union(u: int) -> int:
+    """flags bits that tell the tensor-core kernels how large a union to size their stages for."""
+    return (int(u) & 0x7ff) << 17
+
 EXPORTS = [
     "blockffn_create", "blockffn_destroy", "blockffn_router", "blockffn_chunk_union",
     "blockffn_expert_ffn", "blockffn_layer_forward", "blockffn_layer_forward_scores",

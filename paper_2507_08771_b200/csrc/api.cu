@@ -74,7 +74,8 @@ blockffn_status blockffn_create(const blockffn_config* cfg, blockffn_handle* out
   if (!(cfg->rms_eps >= 0.0f)) return BLOCKFFN_ERR_INVALID_ARG;
   if (cfg->variant < BLOCKFFN_VARIANT_AUTO || cfg->variant > BLOCKFFN_VARIANT_MMA)
     return BLOCKFFN_ERR_INVALID_ARG;
-  if (cfg->flags & ~0x1ffff) return BLOCKFFN_ERR_INVALID_ARG;
+  if (cfg->flags & ~0x0fffffff) return BLOCKFFN_ERR_INVALID_ARG;
+  if (((cfg->flags >> 17) & 0x7ff) > cfg->E) return BLOCKFFN_ERR_INVALID_ARG;
   blockffn_ctx* c = new (std::nothrow) blockffn_ctx();
   if (!c) return BLOCKFFN_ERR_WORKSPACE;
   c->cfg = *cfg;

@@ -888,8 +888,21 @@ MmaPlan make_plan(const blockffn_config& cfg, int L, int grid) {
   const int up_base = up_layout(d, E, 0).total;
   const int down_base = down_layout(d_e, E, 0, pl.max_cols).total;
   const int slot_dn = 8 * 2 * d_e + pl.max_cols * 2 * d_e;
-  // Paired: both kernels fit one SM together when the x tile plus a modest ring fit half of it.
-  const bool paired = up_base + 12 * 2 * d <= kSmemHalf && down_base + 4 * slot_dn <= kSmemHalf;
+  // Paired: an up and a down CTA share an SM (half its shared memory each), so that consecutive
+  // launches overlap. That pays as long as the share of the union a CTA works on fits the half:
+  // otherwise each kernel goes through many short stages, and a whole SM per kernel (fewer,
+  // larger stages, no overlap) is faster. The union is not known at launch time, so the choice
+  // follows the caller's hint, or else the paper's sparsity: 30 % of the experts for a chunk,
+  // 12.5 % for a single token.
+  int u_exp = (cfg.flags >> 17) & 0x7ff;
+  if (u_exp == 0) u_exp = (L == 1 ? E + 4 : 3 * E + 5) / (L == 1 ? 8 : 10);
+  if (u_exp < 1) u_exp = 1;
+  if (u_exp > E) u_exp = E;
+  const int rows_exp = (u_exp * d_e + grid - 1) / grid;
+  const int half_rows = (kSmemHalf - up_base) / (2 * d);
+  const int half_slots = (kSmemHalf - down_base - 128) / slot_dn;
+  const bool fits_half = up_base + 12 * 2 * d <= kSmemHalf && down_base + 4 * slot_dn <= kSmemHalf;
+  const bool paired = fits_half && rows_exp <= half_rows && u_exp <= half_slots;
   const int budget = paired ? kSmemHalf : kSmemMax;
   pl.ring_rows = (budget - up_base) / (2 * d);
   if (want_up && want_up < pl.ring_rows) pl.ring_rows = want_up;

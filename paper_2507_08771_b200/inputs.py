@@ -78,7 +78,12 @@ SHAPES = {
     2: Shape("l_sweep", d=2048, E=64, d_e=128, L=8, union_frac=0.3),
     3: Shape("full_layer", d=2048, E=64, d_e=128, L=8, union_frac=0.3),
     4: Shape("stack24", d=2048, E=64, d_e=128, L=8, union_frac=0.3),
+    # not in the benchmark's list: the FFN of the paper's largest model (App. "model-setting") at the
+    # operating points of its kernel table (Sec. 4.4): a draft tree of 32 tokens whose union is
+    # 30.86 % of the experts, and a single token with 12.45 % of them active
+    5: Shape("paper_2p8b_tree", d=2048, E=128, d_e=128, L=32, union_frac=0.3086),
 }
+PAPER_ONE_TOKEN_ACTIVE = 0.1245   # fraction of experts active for one token (Sec. 4.4)
 STACK_LAYERS = 24
 STACK_CHUNKS = 256
 L_SWEEP = (1, 2, 4, 8, 16, 32)

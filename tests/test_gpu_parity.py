@@ -415,6 +415,36 @@ def test_config3_full_layer_and_union_sweep():
                         u=int(round(frac * sh.E)))
 
 
+@pytest.mark.parametrize("hint", [1, 64])
+def test_expected_union_hint_changes_only_speed(hint):
+    """The hint decides whether a kernel gets half an SM or a whole one; results do not depend on it."""
+    sh, seed = I.SHAPES[2], I.config_seed(2)
+    w = I.make_layer(sh, seed, with_router=False)
+    layer = B.Layer(sh.d, sh.E, sh.d_e, L_max=32, flags=B.cfg_expected_union(hint))
+    dw = layer.upload_weights(w)
+    for L, u in ((1, 19), (8, 19), (8, 64), (32, 45), (5, 3)):
+        check_scores_in(layer, dw, w, sh, L, seed, chunk=L + u, u=u)
+    assert layer.last_status() == 0
+    with pytest.raises(B.BlockFFNError):
+        B.Layer(sh.d, sh.E, sh.d_e, L_max=8, flags=B.cfg_expected_union(sh.E + 1))
+
+
+def test_paper_2p8b_operating_points():
+    """The FFN shape of the paper's largest model at its kernel table's two operating points:
+    32 tree tokens over a 30.86 % union (several stages, four token groups) and one token with
+    12.45 % of the experts active."""
+    sh, seed = I.SHAPES[5], I.config_seed(5)
+    w = I.make_layer(sh, seed, with_router=False)
+    layer = B.Layer(sh.d, sh.E, sh.d_e, L_max=sh.L)
+    dw = layer.upload_weights(w)
+    assert sh.u == 40
+    check_scores_in(layer, dw, w, sh, sh.L, seed, chunk=0)
+    check_scores_in(layer, dw, w, sh, 1, seed, chunk=1,
+                    u=int(round(I.PAPER_ONE_TOKEN_ACTIVE * sh.E)))
+    check_scores_in(layer, dw, w, sh, 8, seed, chunk=2)
+    assert layer.last_status() == 0
+
+
 def test_config4_stack_teacher_forced_and_free_running():
     sh, seed = I.SHAPES[4], I.config_seed(4)
     n_layers = 6                       # distinct layers; the 24-layer run is the benchmark's
