@@ -434,7 +434,7 @@ def test_paper_2p8b_operating_points():
     32 tree tokens over a 30.86 % union (several stages, four token groups) and one token with
     12.45 % of the experts active."""
     sh, seed = I.SHAPES[5], I.config_seed(5)
-    w = I.make_layer(sh, seed, with_router=False)
+    w = I.make_layer(sh, seed, bias_shift=I.ROUTER_BIAS_SHIFT)
     layer = B.Layer(sh.d, sh.E, sh.d_e, L_max=sh.L)
     dw = layer.upload_weights(w)
     assert sh.u == 40
@@ -442,6 +442,9 @@ def test_paper_2p8b_operating_points():
     check_scores_in(layer, dw, w, sh, 1, seed, chunk=1,
                     u=int(round(I.PAPER_ONE_TOKEN_ACTIVE * sh.E)))
     check_scores_in(layer, dw, w, sh, 8, seed, chunk=2)
+    # router on: 128 experts are the most the kernels normalise in one round trip (four mask words)
+    xc = I.make_correlated_x(sh.d, 8, 0.9, seed, chunk=3)
+    check_layer_router_on(layer, dw, w, xc, 8, bias=w["bias"])
     assert layer.last_status() == 0
 
 
