@@ -573,8 +573,28 @@ class RouterWorkload:
         return (self.B.blockffn_tls(hs, self.sh.E), 1.0 - self.B.blockffn_cls(hs, self.sh.E))
 
 
+_probe_lib = None
+
+
+def probe_read(src, nbytes, chained, stream):
+    """bench_probe.cu's benchprobe_read (a library of its own, built by __graft_entry__.build())."""
+    global _probe_lib
+    import ctypes
+    if _probe_lib is None:
+        path = os.path.join(ROOT, "libbenchprobe.so")
+        if not os.path.exists(path):
+            raise ImportError(f"{path} not found: build it with `python __graft_entry__.py`")
+        _probe_lib = ctypes.CDLL(path)
+        _probe_lib.benchprobe_read.argtypes = [ctypes.c_void_p, ctypes.c_size_t, ctypes.c_int,
+                                               ctypes.c_void_p]
+    ptr = src if isinstance(src, int) else src.data_ptr()
+    rc = _probe_lib.benchprobe_read(ptr, int(nbytes), 1 if chained else 0, stream.cuda_stream)
+    if rc != 0:
+        raise RuntimeError(f"benchprobe_read returned {rc}")
+
+
 def read_ceilings(args, torch, device, B):
-    """What a plain read reaches on this device (blockffn_probe_read: 128-bit loads, four CTAs per
+    """What a plain read reaches on this device (bench_probe.cu: 128-bit loads, four CTAs per
     SM, data discarded): streaming over 2 GiB, and single launches the size of one call's active
     weights, back to back over memory that is not in L2, launched plainly and chained like the
     library's own kernels."""
@@ -586,7 +606,7 @@ def read_ceilings(args, torch, device, B):
 
     def enqueue_stream(st):
         for _ in range(4):
-            B.blockffn_probe_read(buf, nbytes, False, st)
+            probe_read(buf, nbytes, False, st)
 
     g = capture(torch, stream, enqueue_stream)
     ms = time_replays(torch, stream, g, steps, 2)
@@ -601,7 +621,7 @@ def read_ceilings(args, torch, device, B):
         for name, chained in (("plain", False), ("chained", True)):
             def enqueue(st, chained=chained):
                 for i in range(n):
-                    B.blockffn_probe_read(base + i * size, size, chained, st)
+                    probe_read(base + i * size, size, chained, st)
             g = capture(torch, stream, enqueue)
             us = time_replays(torch, stream, g, steps, 2) * 1e3 / n
             row[name] = {"us_per_launch": us, "GBps": size / us / 1e3}

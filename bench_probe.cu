@@ -1,7 +1,18 @@
-// Measurement aid (no counterpart in the paper): a read-only pass over a buffer, so that the
-// benchmark can state what a plain read reaches on the device it runs on -- streaming over
-// gigabytes, and in one launch the size of a call's active weights.
-#include "common.cuh"
+// Measurement aid of bench.py, built into a small library of its own (not part of the BlockFFN
+// library, no counterpart in the paper): a read-only pass over a buffer, so that the benchmark
+// can state what a plain read reaches on the device it runs on -- streaming over gigabytes, and
+// in one launch the size of a call's active weights.
+//
+//   int benchprobe_read(const void* src, size_t bytes, int chained, void* stream)
+//
+// Enqueues one kernel that reads `bytes` bytes at `src` (device memory, 16-byte aligned, a
+// multiple of 16 bytes) once, with 128-bit loads from four CTAs per SM, and discards them.
+// chained != 0 launches it with programmatic dependent launch (it starts under the launch before
+// it and waits for that launch before it ends). Returns 0, 1 for a bad argument, 4 for a CUDA
+// error. Allocates nothing.
+#include <cuda_runtime.h>
+#include <stddef.h>
+#include <stdint.h>
 
 namespace {
 
@@ -34,14 +45,13 @@ __global__ void __launch_bounds__(kThreads) read_probe_kernel(const uint4* __res
 
 }  // namespace
 
-extern "C" blockffn_status blockffn_probe_read(const void* src, size_t bytes, int32_t chained,
-                                               void* stream) {
-  if (!src || bytes == 0 || (bytes & 15u) || (reinterpret_cast<uintptr_t>(src) & 15u))
-    return BLOCKFFN_ERR_INVALID_ARG;
+extern "C" __attribute__((visibility("default"))) int benchprobe_read(const void* src, size_t bytes,
+                                                                      int chained, void* stream) {
+  if (!src || bytes == 0 || (bytes & 15u) || (reinterpret_cast<uintptr_t>(src) & 15u)) return 1;
   int device = 0, sms = 0;
   if (cudaGetDevice(&device) != cudaSuccess ||
       cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device) != cudaSuccess)
-    return BLOCKFFN_ERR_CUDA;
+    return 4;
   cudaLaunchAttribute attr[1];
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[0].val.programmaticStreamSerializationAllowed = 1;
@@ -53,5 +63,5 @@ extern "C" blockffn_status blockffn_probe_read(const void* src, size_t bytes, in
   lc.numAttrs = chained ? 1 : 0;
   const cudaError_t e = cudaLaunchKernelEx(&lc, read_probe_kernel,
                                            static_cast<const uint4*>(src), bytes >> 4);
-  return e == cudaSuccess ? BLOCKFFN_OK : BLOCKFFN_ERR_CUDA;
+  return e == cudaSuccess ? 0 : 4;
 }

@@ -58,12 +58,15 @@ typedef enum {
 /* Bits of the device status word (blockffn_last_status). */
 #define BLOCKFFN_DEV_BAD_UNION_ID 1u    /* a union id was < 0 or >= E: that entry was skipped   */
 #define BLOCKFFN_DEV_BAD_UNION_COUNT 2u /* n_union was < 0 or > E: it was clamped               */
-#define BLOCKFFN_DEV_WAIT_EXPIRED 4u    /* a bounded on-chip wait ran out: the call's out is invalid */
+#define BLOCKFFN_DEV_WAIT_EXPIRED 4u    /* a bounded wait inside a kernel ran out: the call's out is invalid */
 
 /* Kernel family used by the expert stage. AUTO picks by L and shape. */
 #define BLOCKFFN_VARIANT_AUTO 0
 #define BLOCKFFN_VARIANT_SIMT 1   /* CUDA-core dot products, fp32 intermediate             */
-#define BLOCKFFN_VARIANT_MMA 2    /* bulk-copy staged, tensor-core tiles, bf16 intermediate */
+#define BLOCKFFN_VARIANT_MMA 2    /* asynchronously staged, tensor-core tiles, bf16 intermediate;
+                                     blockffn_create returns UNSUPPORTED for a shape or ring
+                                     depth these kernels do not take (d % 64, d_e a power of
+                                     two >= 64, ring depths >= 3 / 2)                        */
 
 typedef struct {
   int32_t d;       /* hidden size d_h                                          */
@@ -81,6 +84,14 @@ typedef struct {
  * weights while the kernel enqueued before it on the stream is still finishing
  * (programmatic dependent launch); this bit launches them fully serialised instead. */
 #define BLOCKFFN_CFG_NO_CHAINING 0x10000
+/* Chunks of at most 8 tokens normally run as one kernel per call, several calls in flight per
+ * SM; this bit selects the older two-kernel form (up projection, down projection) for them
+ * too. Same results within the tolerance; kept for comparison and as the path of longer chunks. */
+#define BLOCKFFN_CFG_TWO_KERNELS 0x20000000
+/* Test aid: the one-kernel form's hand-over waits for an arrival that never comes, gives up
+ * after two milliseconds, sets BLOCKFFN_DEV_WAIT_EXPIRED and leaves out untouched. Exercises
+ * the bounded wait without any fault.                                                      */
+#define BLOCKFFN_CFG_TEST_EXPIRE_WAIT 0x10000000
 /* How many experts the caller expects in a chunk's union (1 .. E), bits 17-27 of flags. The
  * tensor-core kernels size their shared memory before the union is known: when the expected
  * union's share fits half an SM, two kernels share an SM and consecutive launches overlap
@@ -154,6 +165,8 @@ BLOCKFFN_API blockffn_status blockffn_chunk_union(blockffn_handle h, const float
 
 /* Eq. 1 + Eq. 2 restricted to the listed experts: reads U_i, D_i only for
  * i in union_ids[0 .. *n_union). out = (out +) sum_i scores[t][i] * D_i Swish(U_i x_t).
+ * union_ids must be a readable i32 [E] array (what blockffn_chunk_union writes); only its
+ * first *n_union entries count, the rest may hold anything and are ignored.
  * x_next (bf16 [L][d], may be NULL, must not alias x) receives the bf16 rounding of the
  * final out: the next layer's input when out is a running fp32 residual.
  * An expert missing from the list contributes nothing, whatever its score.              */
@@ -227,7 +240,10 @@ BLOCKFFN_API uint64_t blockffn_launch_count(blockffn_handle h);
  *     256-byte header. A call whose E * L * d_e * 4 exceeds that size returns
  *     BLOCKFFN_ERR_WORKSPACE and enqueues nothing.
  *   - The first call on a device looks up the array's device address (with that device
- *     current) and caches it; make that first call outside any stream capture.
+ *     current) and caches it; make that first call at start-up, outside any stream capture.
+ *     That first call is also where the driver may load the library's image onto the device,
+ *     array included. Later calls find the address under a lock and may come from any host
+ *     thread.
  *   - All calls on a device share the one array. Calls enqueued on the same stream are safe;
  *     two calls that may run on the GPU at the same time (different streams, or graph
  *     branches) race on it and give wrong results. Nothing in the array carries over from
@@ -238,18 +254,6 @@ BLOCKFFN_API blockffn_status blockffn_expert_ffn_noalloc(
     const blockffn_config* cfg, const blockffn_weights* w, const void* x, const float* scores,
     int32_t L, const int32_t* union_ids, const int32_t* n_union, float* out, void* x_next,
     int32_t call_flags, void* stream);
-
-/* Measurement aid; the paper has no counterpart. Enqueues one kernel that reads `bytes` bytes at
- * `src` (device memory, 16-byte aligned, a multiple of 16 bytes) once, with 128-bit loads from
- * four CTAs per SM, and discards them: what a plain read of that many bytes costs on the
- * device it runs on. The benchmark uses it for its read-only ceilings (streaming over
- * gigabytes; one launch the size of a call's active weights, back to back over cold memory).
- * chained != 0 launches it with programmatic dependent launch like the library's own kernels
- * (it starts under the launch before it and waits for it before it ends). Needs no handle,
- * allocates nothing. INVALID_ARG for a NULL or misaligned src or a size that is 0 or not a
- * multiple of 16.                                                                          */
-BLOCKFFN_API blockffn_status blockffn_probe_read(const void* src, size_t bytes, int32_t chained,
-                                                 void* stream);
 
 /* Human-readable name of a status code (static storage). */
 BLOCKFFN_API const char* blockffn_status_string(blockffn_status s);

@@ -24,6 +24,8 @@ DEV_BAD_UNION_ID, DEV_BAD_UNION_COUNT, DEV_WAIT_EXPIRED = 1, 2, 4
 VARIANT_AUTO, VARIANT_SIMT, VARIANT_MMA = 0, 1, 2
 CALL_ACCUMULATE, CALL_INDEPENDENT, CALL_INDEPENDENT_X = 1, 2, 4
 CFG_NO_CHAINING = 0x10000
+CFG_TWO_KERNELS = 0x20000000
+CFG_TEST_EXPIRE_WAIT = 0x10000000
 
 
 def cfg_expected_union(u: int) -> int:
@@ -35,7 +37,6 @@ EXPORTS = [
     "blockffn_expert_ffn", "blockffn_layer_forward", "blockffn_layer_forward_scores",
     "blockffn_read_routing", "blockffn_last_status", "blockffn_tls", "blockffn_cls",
     "blockffn_launch_count", "blockffn_status_string", "blockffn_expert_ffn_noalloc",
-    "blockffn_probe_read",
 ]
 NOALLOC_SCRATCH_BYTES = 1 << 20
 
@@ -84,7 +85,6 @@ def load():
     lib.blockffn_read_routing.argtypes = [vp, i32, vp, vp, vp, vp, vp, vp]
     lib.blockffn_expert_ffn_noalloc.argtypes = [ctypes.POINTER(Config), ctypes.POINTER(Weights), vp,
                                                 vp, i32, vp, vp, vp, vp, i32, vp]
-    lib.blockffn_probe_read.argtypes = [vp, ctypes.c_size_t, i32, vp]
     lib.blockffn_last_status.argtypes = [vp, ctypes.POINTER(ctypes.c_uint32), i32, vp]
     lib.blockffn_tls.argtypes = [ctypes.POINTER(Stats), i32]
     lib.blockffn_tls.restype = ctypes.c_double
@@ -167,12 +167,6 @@ def blockffn_expert_ffn_noalloc(cfg: Config, w: Weights, x, scores, L, union_ids
                                               _ptr(scores), L, _ptr(union_ids), _ptr(n_union),
                                               _ptr(out), _ptr(x_next), call_flags,
                                               _stream(stream)), "blockffn_expert_ffn_noalloc")
-
-
-def blockffn_probe_read(src, nbytes, chained=False, stream=None):
-    """Measurement aid: one kernel that reads nbytes at src (device) once and discards them."""
-    _check(load().blockffn_probe_read(_ptr(src), int(nbytes), 1 if chained else 0, _stream(stream)),
-           "blockffn_probe_read")
 
 
 def blockffn_layer_forward(h, w: Weights, x, L, out, x_next=None, stats=None, call_flags=0,

@@ -21,6 +21,19 @@ bool use_mma(const blockffn_ctx* c, int L) {
   return c->cfg.variant != BLOCKFFN_VARIANT_SIMT && expert_mma_supported(c, L);
 }
 
+// Tensor-core expert stage: one kernel per call where the shape allows it, else the pair.
+cudaError_t launch_tensor_core(blockffn_ctx* c, const blockffn_weights* w, const void* x,
+                               const float* scores, int L, const int32_t* union_ids,
+                               const int32_t* n_union, float* out, void* x_next, int call_flags,
+                               const RoutingOut* pub, const RouterLogits* logits, bool logits_final,
+                               cudaStream_t st) {
+  if (expert_lean_supported(c, L))
+    return launch_expert_lean(c, w, x, scores, L, union_ids, n_union, out, x_next, call_flags, pub,
+                              logits, logits_final, st);
+  return launch_expert_mma(c, w, x, scores, L, union_ids, n_union, out, x_next, call_flags, pub,
+                           logits, logits_final, st);
+}
+
 // Expert stage from a given union list.
 blockffn_status expert_dispatch(blockffn_ctx* c, const blockffn_weights* w, const void* x,
                                 const float* scores, int L, const int32_t* union_ids,
@@ -28,8 +41,8 @@ blockffn_status expert_dispatch(blockffn_ctx* c, const blockffn_weights* w, cons
                                 cudaStream_t st) {
   cudaError_t e;
   if (use_mma(c, L))
-    e = launch_expert_mma(c, w, x, scores, L, union_ids, n_union, out, x_next, call_flags, nullptr,
-                          nullptr, false, st);
+    e = launch_tensor_core(c, w, x, scores, L, union_ids, n_union, out, x_next, call_flags, nullptr,
+                           nullptr, false, st);
   else
     e = launch_expert_simt(c, w, x, scores, L, union_ids, n_union, out, x_next, call_flags, st);
   return e == cudaSuccess ? BLOCKFFN_OK : BLOCKFFN_ERR_CUDA;
@@ -74,7 +87,7 @@ blockffn_status blockffn_create(const blockffn_config* cfg, blockffn_handle* out
   if (!(cfg->rms_eps >= 0.0f)) return BLOCKFFN_ERR_INVALID_ARG;
   if (cfg->variant < BLOCKFFN_VARIANT_AUTO || cfg->variant > BLOCKFFN_VARIANT_MMA)
     return BLOCKFFN_ERR_INVALID_ARG;
-  if (cfg->flags & ~0x0fffffff) return BLOCKFFN_ERR_INVALID_ARG;
+  if (cfg->flags & ~0x3fffffff) return BLOCKFFN_ERR_INVALID_ARG;
   if (((cfg->flags >> 17) & 0x7ff) > cfg->E) return BLOCKFFN_ERR_INVALID_ARG;
   blockffn_ctx* c = new (std::nothrow) blockffn_ctx();
   if (!c) return BLOCKFFN_ERR_WORKSPACE;
@@ -104,6 +117,9 @@ blockffn_status blockffn_create(const blockffn_config* cfg, blockffn_handle* out
   const size_t o_nu = take(sizeof(int32_t));
   const size_t o_h32 = take(sizeof(float) * E * L * d_e);
   const size_t o_h16 = take(expert_mma_h_bytes(cfg));
+  const size_t lean_bytes = expert_lean_ws_bytes(cfg, c->num_sms);
+  const size_t o_lean = take(lean_bytes);
+  const size_t o_seq = take(sizeof(unsigned long long) * 16);
   const size_t o_tk = take(sizeof(unsigned int) * 8);
   const size_t o_st = take(sizeof(uint32_t));
   void* base = nullptr;
@@ -129,12 +145,22 @@ blockffn_status blockffn_create(const blockffn_config* cfg, blockffn_handle* out
   c->n_union = reinterpret_cast<int32_t*>(b + o_nu);
   c->h32 = reinterpret_cast<float*>(b + o_h32);
   c->h16 = b + o_h16;
+  c->lean_ring = lean_bytes ? b + o_lean : nullptr;
+  c->lean_seq = reinterpret_cast<unsigned long long*>(b + o_seq);
   c->ticket = reinterpret_cast<unsigned int*>(b + o_tk);
   c->status = reinterpret_cast<uint32_t*>(b + o_st);
-  if (expert_mma_setup(c) != cudaSuccess) {
+  if (expert_mma_setup(c) != cudaSuccess || expert_lean_setup(c) != cudaSuccess) {
     cudaFree(base);
     delete c;
     return BLOCKFFN_ERR_CUDA;
+  }
+  // A caller that names the tensor-core kernels gets them or an error, never a silent switch
+  // to the other family (AUTO keeps choosing per call).
+  if (cfg->variant == BLOCKFFN_VARIANT_MMA &&
+      !(expert_mma_supported(c, 1) && expert_mma_supported(c, cfg->L_max))) {
+    cudaFree(base);
+    delete c;
+    return BLOCKFFN_ERR_UNSUPPORTED;
   }
   // The stream and events the router of blockffn_layer_forward may run on; without them that
   // call keeps its router on the caller's stream.
@@ -272,8 +298,8 @@ blockffn_status blockffn_layer_forward(blockffn_handle h, const blockffn_weights
           cudaStreamWaitEvent(st, h->ev_router[b], 0) != cudaSuccess)
         return BLOCKFFN_ERR_CUDA;
       h->last_layer_waited_first = false;
-      return launch_expert_mma(h, w, x, h->scores, L, nullptr, nullptr, out, x_next, flags, &pub,
-                               &lg, true, st) == cudaSuccess
+      return launch_tensor_core(h, w, x, h->scores, L, nullptr, nullptr, out, x_next, flags, &pub,
+                                &lg, true, st) == cudaSuccess
                  ? BLOCKFFN_OK
                  : BLOCKFFN_ERR_CUDA;
     }
@@ -286,8 +312,8 @@ blockffn_status blockffn_layer_forward(blockffn_handle h, const blockffn_weights
     if (launch_router(h, w, x, L, h->scores, h->tok_mask, false, nullptr, true, logits,
                       ahead ? 1 : 0, st) != cudaSuccess)
       return BLOCKFFN_ERR_CUDA;
-    return launch_expert_mma(h, w, x, h->scores, L, nullptr, nullptr, out, x_next, flags, &pub, &lg,
-                             false, st) == cudaSuccess
+    return launch_tensor_core(h, w, x, h->scores, L, nullptr, nullptr, out, x_next, flags, &pub, &lg,
+                              false, st) == cudaSuccess
                ? BLOCKFFN_OK
                : BLOCKFFN_ERR_CUDA;
   }
@@ -315,8 +341,8 @@ blockffn_status blockffn_layer_forward_scores(blockffn_handle h, const blockffn_
     // The expert kernels derive Union(x) from the scores themselves (every CTA needs the
     // list before it can fetch a weight byte) and CTA 0 publishes it: no separate launch.
     const RoutingOut pub{h->union_mask, h->union_ids, h->n_union, stats, nullptr, nullptr};
-    return launch_expert_mma(h, w, x, scores, L, nullptr, nullptr, out, x_next, call_flags, &pub,
-                             nullptr, false, st) == cudaSuccess
+    return launch_tensor_core(h, w, x, scores, L, nullptr, nullptr, out, x_next, call_flags, &pub,
+                              nullptr, false, st) == cudaSuccess
                ? BLOCKFFN_OK
                : BLOCKFFN_ERR_CUDA;
   }

@@ -39,6 +39,8 @@ struct blockffn_ctx {
   int32_t* n_union;     // [1]
   float* h32;           // [E][L_max][d_e] fp32 intermediate (SIMT variant)
   void* h16;            // bf16 intermediate (MMA variant), slot-major padded rows
+  void* lean_ring;      // ring of bf16 intermediates of the one-kernel form (NULL: not used)
+  unsigned long long* lean_seq;   // [0] call tickets, [1 .. 8] arrival counters of the ring slots
   unsigned int* ticket; // last-block-done counters [8]
   uint32_t* status;     // sticky device status word
 };
@@ -87,6 +89,17 @@ struct RouterLogits {
   const float* gain;    // [E]
   float eps;
 };
+
+// One-kernel form of the tensor-core expert stage for chunks of at most 8 tokens (same
+// arguments as launch_expert_mma below).
+bool expert_lean_supported(const blockffn_ctx* c, int L);
+size_t expert_lean_ws_bytes(const blockffn_config* cfg, int grid);
+cudaError_t expert_lean_setup(blockffn_ctx* c);
+cudaError_t launch_expert_lean(blockffn_ctx* c, const blockffn_weights* w, const void* x,
+                               const float* scores, int L, const int32_t* union_ids,
+                               const int32_t* n_union, float* out, void* x_next, int call_flags,
+                               const RoutingOut* pub, const RouterLogits* logits, bool logits_final,
+                               cudaStream_t st);
 
 // Tensor-core / bulk-copy variant of the expert stage. union_ids == NULL: the kernels derive
 // the union from the nonzero pattern of scores and publish it through pub; with logits != NULL

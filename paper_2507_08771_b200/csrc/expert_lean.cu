@@ -1,0 +1,721 @@
+// Expert stage (Eq. 1, Eq. 2 restricted to Union(x), Sec. 3.3) for chunks of at most 8 tokens:
+// one kernel per call, several calls in flight per SM.
+//
+// A call lasts a few microseconds, most of which is memory latency: the routing inputs, then
+// the weights they select, then the intermediate every CTA needs from every other. What the
+// device sustains is therefore set by how many calls are in flight per SM, i.e. by how little
+// shared memory and how few registers one CTA holds. This kernel keeps only the weights in
+// shared memory; the small operands (x for the up projection, the intermediate h for the
+// down projection) go from L2 straight into the registers of the one warp that uses them:
+// with K split over the warps no two warps read the same element, so a shared tile would
+// only be a detour. Three CTAs (three successive calls) then fit one SM at d = 2048.
+//
+//   CTA b, call n:
+//     ticket           one atomic per CTA on the handle's call counter; ticket / grid is the
+//                      call's index n (all CTAs of a call take theirs before any CTA of the next
+//                      call exists, see below), n mod 8 its slot in the ring of h buffers
+//     Union(x)         derived by every CTA from the scores, the caller's list or raw logits
+//     up projection    the CTA's share of the union's neuron rows -> shared memory (16-byte
+//                      asynchronous copies), K split over the 8 warps, mma.sync m16n8k16 with
+//                      the weights as the M operand and the tokens as N, cross-warp sum, Swish,
+//                      router score, bf16 -> h ring slot (global, L2)
+//     hand-over        one arrival per CTA on the slot's counter (after a fence); the D slabs of
+//                      the CTA's output columns are requested into the same shared memory; then
+//                      one thread polls the counter until all CTAs of the call have arrived
+//                      (bounded: BLOCKFFN_DEV_WAIT_EXPIRED) and the warps fetch their h fragments
+//     down projection  out[t][c] over all union experts for the CTA's <= 16 columns, one writer
+//                      per element, fixed summation order
+//     griddepcontrol.wait before out is touched (and before the kernel ends)
+//
+// Ordering between calls. Kernels are chained by programmatic dependent launch and trigger
+// their dependents only once the CTA holds its ticket, so tickets of successive calls never
+// interleave. Every kernel waits for its predecessor before it ends; a CTA of call n + R can
+// therefore exist only if fewer than R calls are incomplete, R - 1 being the number of CTAs
+// that fit one SM. With R = 8 ring slots (at most 7 CTAs of 256 threads... fit the 2048-thread
+// SM together with the CTA that replaces them) a slot is never reused while a CTA of its earlier
+// call is alive, and its arrival counter is an exact multiple of the grid size when a call
+// starts: the counters only ever grow, nothing is reset, graph replays need no host state.
+// The polling thread issues no asynchronous copies: a fence or an acquire by a thread waits
+// for that thread's own copies in flight.
+#include "mma_tiles.cuh"
+
+namespace {
+
+constexpr int kHRing = 8;            // h buffers and arrival counters per handle
+constexpr int kSyncThread = kThreads - 1;
+constexpr int kCopyThreads = kThreads - 32;   // the last warp (the polling thread's) issues no D copies
+constexpr int kMaxKB = 4;            // 64-wide k blocks of x per warp: d <= 8 * 64 * kMaxKB
+constexpr int kHB = 5;               // h fragments a warp keeps in registers per batch
+
+struct LeanLayout {
+  int off_red, off_w, total;
+};
+// red: cross-warp partials, up [8 warps][8 tokens][red_rows] f32, down [8 warps][8][16] f32
+__host__ __device__ inline LeanLayout lean_layout(int E, int red_rows, int cap_bytes) {
+  LeanLayout s;
+  s.off_red = kOffIds + align128(E * 4);
+  const int red = kWarps * 8 * 4 * (red_rows > 16 ? red_rows : 16);
+  s.off_w = s.off_red + align128(red);
+  s.total = s.off_w + cap_bytes;
+  return s;
+}
+
+struct LeanParams {
+  const uint16_t* x;       // bf16 [L][d]
+  const uint16_t* U;       // bf16 [E][d_e][d]
+  const uint16_t* D;       // bf16 [E][d][d_e]
+  const float* scores;
+  RouterLogits lg;
+  const int32_t* ids_in;
+  const int32_t* n_in;
+  uint16_t* h_ring;        // kHRing buffers of h_slot elements, each bf16 [q][L][d_e]
+  size_t h_slot;
+  unsigned long long* seq;     // tickets: one per CTA per call
+  unsigned long long* ready;   // [kHRing] arrivals, never reset
+  float* out;
+  uint16_t* x_next;
+  int L, d, E, d_e, de_shift;
+  int cap_bytes, red_rows;     // weight region; rows the up partial tile is sized for
+  int max_cols, cols_q, cols_rem;
+  int accumulate;
+  int hold;                    // test aid: wait for an arrival that never comes
+  unsigned long long wait_ns;  // bound of the hand-over wait
+  uint32_t* status;
+  uint32_t* pub_mask;
+  int32_t* pub_ids;
+  int32_t* pub_n;
+  blockffn_stats* stats;
+  float* pub_scores;
+  uint32_t* pub_tok;
+};
+
+__device__ __forceinline__ unsigned long long global_ns() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+__device__ __forceinline__ unsigned long long ld_acquire_u64(const unsigned long long* p) {
+  unsigned long long v;
+  asm volatile("ld.acquire.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(p) : "memory");
+  return v;
+}
+// A 64-wide k block of a small operand row straight from global memory (L2): this lane's 8
+// consecutive k of each 32-wide half, the same k permutation load_frag64 applies to the
+// shared-memory operand.
+// (volatile: the loads are issued where they are written, long before their first use, and must
+// not be sunk to it)
+__device__ __forceinline__ uint4 ld_cg_v4(const uint4* p) {
+  uint4 v;
+  asm volatile("ld.global.cg.v4.u32 {%0, %1, %2, %3}, [%4];"
+               : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+               : "l"(p)
+               : "memory");
+  return v;
+}
+// ---- instruction-lean building blocks ----------------------------------------------------
+// A call's 2000-odd warp instructions per warp were what limited three resident CTAs, not the
+// memory system: four schedulers issue for 24 warps. Everything below is written to spend few
+// instructions: 32-bit shared-memory addresses with constant offsets, 32-bit element indices
+// into global memory (one mad.wide per address), no select in the fragment path.
+//
+// Rows of an operand tile are stored even rows first, then 64 bytes of padding, then the odd
+// rows: the two rows a quarter-warp reads together (g and g + 1) then sit 64 bytes apart modulo
+// 128, i.e. on disjoint halves of the 32 banks, and a fragment is two plain 128-bit loads.
+__device__ __forceinline__ uint4 lds128(uint32_t a) {
+  uint4 v;
+  asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];"
+               : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+               : "r"(a));
+  return v;
+}
+// global address = base + 16 * idx16 (idx16 < 2^32)
+__device__ __forceinline__ const void* at16(const void* base, uint32_t idx16) {
+  unsigned long long a;
+  asm("mad.wide.u32 %0, %1, 16, %2;" : "=l"(a) : "r"(idx16), "l"(base));
+  return reinterpret_cast<const void*>(a);
+}
+// the four mma of one 64-wide k block: a = rows g (lo/hi half), b = rows g + 8, x = the tokens
+__device__ __forceinline__ void mma64(float (&c0)[4], float (&c1)[4], const uint4& alo,
+                                      const uint4& ahi, const uint4& blo, const uint4& bhi,
+                                      const Frag64& x) {
+  mma_bf16(c0, alo.x, blo.x, alo.y, blo.y, x.lo.x, x.lo.y);
+  mma_bf16(c1, ahi.x, bhi.x, ahi.y, bhi.y, x.hi.x, x.hi.y);
+  mma_bf16(c0, alo.z, blo.z, alo.w, blo.w, x.lo.z, x.lo.w);
+  mma_bf16(c1, ahi.z, bhi.z, ahi.w, bhi.w, x.hi.z, x.hi.w);
+}
+
+// KB: 64-wide k blocks of x per warp (ceil(d / 512)); MODE as derive_union; EARLY: 0 wait first,
+// 1 routing inputs and weights before the wait, 2 x as well (the wait then comes before out).
+template <int KB, int MODE, int EARLY>
+__global__ void __launch_bounds__(kThreads, 3) expert_lean_kernel(const LeanParams p) {
+  extern __shared__ __align__(128) unsigned char smem[];
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int d = p.d, d_e = p.d_e, L = p.L;
+  const LeanLayout lay = lean_layout(p.E, p.red_rows, p.cap_bytes);
+  const uint32_t sbase = smem_u32(smem);
+  const uint32_t wbase = sbase + lay.off_w;
+  int* ctl = reinterpret_cast<int*>(smem + kOffCtl);
+  int* ids_sm = reinterpret_cast<int*>(smem + kOffIds);
+  float* red = reinterpret_cast<float*>(smem + lay.off_red);
+  const int g = lane >> 2, tg = lane & 3;
+  const int G = gridDim.x, bx = blockIdx.x;
+
+  if (tid < 8) ctl[tid] = 0;
+  if constexpr (EARLY == 0) {
+    if constexpr (MODE == 2) {
+      if (tid * 32 < p.E) asm volatile("prefetch.global.L2 [%0];" ::"l"(p.lg.gain + tid * 32));
+    }
+    pdl_wait();
+  }
+  unsigned long long ticket = 0;
+  if (tid == 0) ticket = atomicAdd(p.seq, 1ull);
+  __syncthreads();
+  // Thread 0 turns its ticket into the call's ring slot and lets the dependents go while the
+  // routing loads are in flight: every CTA of this call then holds its ticket before a CTA of
+  // the next call exists, and the next call starts as early as that allows.
+  auto on_ticket = [&]() {
+    const unsigned long long n = ticket / (unsigned)G;
+    ctl[6] = (int)(n & (kHRing - 1));
+    *reinterpret_cast<unsigned long long*>(ctl + 138) =
+        p.hold ? ~0ull : ((n >> 3) + 1ull) * (unsigned)G;
+    pdl_trigger();
+  };
+  const int nu = derive_union<MODE>(p.scores, p.lg, p.ids_in, p.n_in, L, p.E, ids_sm, ctl,
+                                    reinterpret_cast<uint32_t*>(red), on_ticket);
+
+  // ---- up projection ---------------------------------------------------------------------
+  const int R = nu * d_e;
+  const int rq = R / G, rrem = R - rq * G;
+  const int r0 = bx * rq + min(bx, rrem), nrows = rq + (bx < rrem ? 1 : 0), r1 = r0 + nrows;
+  const int row_bytes = 2 * d;
+  const int cap_rows = min((p.cap_bytes - 128) / row_bytes, 2 * p.red_rows);
+  const bool single = nrows <= min(p.red_rows, cap_rows);
+  const int slot_rows = single ? max(nrows, 1) : min(p.red_rows, cap_rows / 2);
+  const int ngroups = (nrows + slot_rows - 1) / slot_rows;
+  const int rpg = ngroups ? (nrows + ngroups - 1) / ngroups : 0;
+  const int half_u = ((slot_rows + 1) >> 1) * row_bytes + 64;   // where the odd rows start
+  const int slot_bytes = slot_rows * row_bytes + 64;
+  const int sh = p.de_shift;
+  const int ldr = p.red_rows;
+  // This thread's part of a row copy: 16-byte chunk my_c of the rows my_sub, my_sub + rpi, ...
+  const int cpr = d >> 3;                       // chunks per row (<= 256)
+  const int rpi = kThreads / cpr;               // rows the CTA copies per step
+  const int my_sub = tid / cpr, my_c = tid - my_sub * cpr;
+  const bool copies_u = my_sub < rpi;
+  // stage gi: rows [r0 + gi rpg, ...) -> slot gi & 1, row m of the stage at
+  // (m >> 1) row_bytes + (m & 1) half_u
+  auto issue_u = [&](int gi) {
+    const int ra = r0 + gi * rpg;
+    const int rows = min(r1, ra + rpg) - ra;
+    const uint32_t slot0 = wbase + (gi & 1) * slot_bytes + my_c * 16;
+    if (copies_u) {
+      int m = my_sub;
+      while (m < rows) {
+        const int r = ra + m, q = r >> sh;
+        const int seg_end = min(rows, ((q + 1) << sh) - ra);     // rows of this expert end here
+        uint32_t idx = (uint32_t)(ids_sm[q] * d_e + (r - (q << sh))) * (uint32_t)cpr + my_c;
+        const uint32_t step = (uint32_t)rpi * cpr;
+#pragma unroll 4
+        for (; m < seg_end; m += rpi, idx += step)
+          cp_async16(slot0 + (m >> 1) * row_bytes + (m & 1) * half_u, at16(p.U, idx));
+      }
+    }
+  };
+  // score, expert slot and neuron of the h element this thread finishes in a stage
+  // (token tid / 32, row tid % 32 of the stage)
+  float sc = 0.0f;
+  int hidx = -1;        // element index into the h buffer, -1: nothing to finish
+  auto prepare = [&](int gi) {
+    const int ra = r0 + gi * rpg, rows = min(r1, ra + rpg) - ra;
+    const int t = tid >> 5, m = tid & 31;
+    sc = 0.0f;
+    hidx = -1;
+    if (t < L && m < rows) {
+      const int hq = (ra + m) >> sh;
+      hidx = (hq * L + t) * d_e + (ra + m - (hq << sh));
+      const int id = ids_sm[hq];
+      if constexpr (MODE == 2) {
+        float v = __ldcg(p.lg.a0 + t * p.E + id);
+        v = v > 0.0f ? v : 0.0f;
+        sc = __ldg(p.lg.gain + id) * v * reinterpret_cast<const float*>(ctl + 104)[t];
+      } else {
+        sc = __ldcg(p.scores + t * p.E + id);
+      }
+    }
+  };
+  // x: this warp's k blocks (warp + 8 i) of the token row this lane feeds to the mma
+  const int npx = d >> 6;
+  Frag64 fx[KB];
+  auto load_x = [&]() {
+    const uint4* xp = reinterpret_cast<const uint4*>(p.x + min(g, L - 1) * d + 64 * warp) + tg;
+#pragma unroll
+    for (int i = 0; i < KB; ++i) {
+      if (warp + kWarps * i < npx) {
+        fx[i].lo = ld_cg_v4(xp + 64 * i);          // 64 k blocks of 128 bytes = 8 warps further
+        fx[i].hi = ld_cg_v4(xp + 64 * i + 4);
+      } else {
+        fx[i].lo = fx[i].hi = make_uint4(0, 0, 0, 0);
+      }
+    }
+  };
+  // x goes first when it is stable: its short round trip then runs under the long issue of
+  // the weights instead of behind it
+  if constexpr (EARLY == 2) load_x();
+  if (ngroups > 0) issue_u(0);
+  cp_async_commit();
+  if (ngroups > 1) issue_u(1);
+  cp_async_commit();
+  if (ngroups > 0) prepare(0);
+  if constexpr (EARLY == 1) pdl_wait();     // x may come from the kernel just before
+  if constexpr (EARLY != 2) load_x();
+  const int slot = ctl[6];       // (written before the barriers inside derive_union)
+  uint16_t* hbuf = p.h_ring + (size_t)slot * p.h_slot;
+
+  for (int gi = 0; gi < ngroups; ++gi) {
+    const int rows = min(r1, r0 + (gi + 1) * rpg) - (r0 + gi * rpg);
+    // fragment addresses of rows g and g + 8 (same parity) of the two 16-row tiles, at this
+    // warp's first k block; rows beyond the stage read its last row (their results are dropped)
+    auto row_addr = [&](int m) {
+      m = min(m, rows - 1);
+      return wbase + (gi & 1) * slot_bytes + (m >> 1) * row_bytes + (m & 1) * half_u + 128 * warp +
+             16 * tg;
+    };
+    const uint32_t a0 = row_addr(g), b0 = row_addr(g + 8);
+    cp_async_wait_group<1>();      // all but the newest group: this stage has landed
+    __syncthreads();
+    float* mine = red + warp * (8 * ldr);
+    const int t2 = 2 * tg;
+    {
+      float c0[4] = {0.f, 0.f, 0.f, 0.f}, c1[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+      for (int i = 0; i < KB; ++i) {
+        if (warp + kWarps * i < npx) {
+          const uint4 alo = lds128(a0 + 1024 * i), ahi = lds128(a0 + 1024 * i + 64);
+          const uint4 blo = lds128(b0 + 1024 * i), bhi = lds128(b0 + 1024 * i + 64);
+          mma64(c0, c1, alo, ahi, blo, bhi, fx[i]);
+        }
+      }
+      // partial tile of this warp -> red[warp][t][m] (rows beyond the tile's width are padding)
+      if (g < ldr) {
+        mine[t2 * ldr + g] = c0[0] + c1[0];
+        mine[(t2 + 1) * ldr + g] = c0[1] + c1[1];
+      }
+      if (g + 8 < ldr) {
+        mine[t2 * ldr + g + 8] = c0[2] + c1[2];
+        mine[(t2 + 1) * ldr + g + 8] = c0[3] + c1[3];
+      }
+    }
+    if (rows > 16) {               // second tile of 16 rows
+      const uint32_t a1 = row_addr(g + 16), b1 = row_addr(g + 24);
+      float c0[4] = {0.f, 0.f, 0.f, 0.f}, c1[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+      for (int i = 0; i < KB; ++i) {
+        if (warp + kWarps * i < npx) {
+          const uint4 alo = lds128(a1 + 1024 * i), ahi = lds128(a1 + 1024 * i + 64);
+          const uint4 blo = lds128(b1 + 1024 * i), bhi = lds128(b1 + 1024 * i + 64);
+          mma64(c0, c1, alo, ahi, blo, bhi, fx[i]);
+        }
+      }
+      if (g + 16 < ldr) {
+        mine[t2 * ldr + g + 16] = c0[0] + c1[0];
+        mine[(t2 + 1) * ldr + g + 16] = c0[1] + c1[1];
+      }
+      if (g + 24 < ldr) {
+        mine[t2 * ldr + g + 24] = c0[2] + c1[2];
+        mine[(t2 + 1) * ldr + g + 24] = c0[3] + c1[3];
+      }
+    }
+    __syncthreads();               // partials complete; every warp is done with the slot
+    if (gi + 2 < ngroups) issue_u(gi + 2);
+    cp_async_commit();
+    if (hidx >= 0) {
+      const float* col = red + (tid >> 5) * ldr + (tid & 31);
+      float v = 0.0f;
+#pragma unroll
+      for (int w = 0; w < kWarps; ++w) v += col[w * (8 * ldr)];
+      hbuf[hidx] = (uint16_t)f32_to_bf16_bits(sc * swish_fast(v));
+    }
+    if (gi + 1 < ngroups) prepare(gi + 1);
+    // the next stage starts with a wait and a barrier, which also protects red
+  }
+  cp_async_wait_all();
+  __syncthreads();                 // every h element of this CTA has been stored
+  if (tid == kSyncThread) {
+    __threadfence();
+    asm volatile("red.relaxed.gpu.global.add.u64 [%0], 1;" ::"l"(p.ready + slot) : "memory");
+  }
+
+  // ---- down projection -------------------------------------------------------------------
+  // Slab of one expert: the CTA's columns as rows of 2 d_e bytes, even columns first, 64 bytes
+  // of padding, odd columns.
+  const int drow = 2 * d_e;
+  const int half_d = ((p.max_cols + 1) >> 1) * drow + 64;
+  const int slot_d = p.max_cols * drow + 64;
+  const int cap_slabs = p.cap_bytes / slot_d;
+  const int rsz = nu <= cap_slabs ? max(nu, 1) : max(1, cap_slabs / 2);
+  const int nrounds = (nu + rsz - 1) / rsz;
+  const int c0 = bx * p.cols_q + min(bx, p.cols_rem);
+  const int ncols = p.cols_q + (bx < p.cols_rem ? 1 : 0);
+  // A slab is ncols << kshift chunks of 16 bytes; chunk c = column c >> kshift, piece
+  // c & (2^kshift - 1). Thread tid copies chunks tid, tid + kCopyThreads, ... of every expert
+  // (one chunk per thread at the usual shapes).
+  const int kshift = sh - 3;                    // log2(chunks per D row)
+  const uint32_t estride16 = (uint32_t)d << kshift;
+  const int nchunks = tid < kCopyThreads ? ncols << kshift : 0;
+  auto issue_d = [&](int r) {
+    const int q0 = r * rsz, n = min(rsz, nu - q0);
+    for (int c = tid; c < nchunks; c += kCopyThreads) {
+      const int cc = c >> kshift, k = c & ((1 << kshift) - 1);
+      const uint32_t src0 = ((uint32_t)(c0 + cc) << kshift) + k;          // + id * d << kshift
+      uint32_t dst = wbase + (r & 1) * rsz * slot_d + (cc >> 1) * drow + (cc & 1) * half_d + k * 16;
+#pragma unroll 4
+      for (int i = 0; i < n; ++i, dst += slot_d)
+        cp_async16(dst, at16(p.D, src0 + (uint32_t)ids_sm[q0 + i] * estride16));
+    }
+  };
+  if (nrounds > 0) issue_d(0);
+  cp_async_commit();
+  if (nrounds > 1) issue_d(1);
+  cp_async_commit();
+  bool waited = EARLY < 2;
+  // the residual this CTA's outputs are added to: asked for as early as out may be read
+  float resid = 0.0f;
+  if (waited && p.accumulate && tid < 128) {
+    const int t = tid >> 4, m = tid & 15;
+    if (t < L && m < ncols) resid = __ldcg(p.out + t * d + c0 + m);
+  }
+  // hand-over: all CTAs of this call have stored their part of h
+  if (tid == kSyncThread) {
+    const unsigned long long target = *reinterpret_cast<const unsigned long long*>(ctl + 138);
+    const unsigned long long t0 = global_ns();
+    // once a wait has run out on this handle the later ones give up quickly, until the caller
+    // has read and cleared the status word
+    const bool before = (*reinterpret_cast<volatile uint32_t*>(p.status) & BLOCKFFN_DEV_WAIT_EXPIRED) != 0;
+    const unsigned long long limit = p.hold ? 2000000ull : before ? 1000000ull : p.wait_ns;
+    int expired = 0;
+    while (ld_acquire_u64(p.ready + slot) < target) {
+      if (global_ns() - t0 > limit) {
+        expired = 1;
+        break;
+      }
+    }
+    if (expired) {
+      ctl[5] = 1;
+      atomicOr(p.status, BLOCKFFN_DEV_WAIT_EXPIRED);
+    }
+  }
+  __syncthreads();
+  const bool dead = ctl[5] != 0;    // the wait ran out: out is left untouched
+
+  const int npairs = d_e >> 6;      // 64-wide k blocks per expert (a power of two)
+  const int pshift = sh - 6;
+  float acc0[1][4], acc1[1][4];
+  zero_acc<1>(acc0);
+  zero_acc<1>(acc1);
+  // rows (columns of out) g and g + 8 of a slab, clamped to the CTA's columns
+  auto col_off = [&](int m) {
+    m = min(m, max(ncols, 1) - 1);
+    return (m >> 1) * drow + (m & 1) * half_d + 16 * tg;
+  };
+  const uint32_t da_off = col_off(g), db_off = col_off(g + 8);
+  const uint4* hrow = reinterpret_cast<const uint4*>(hbuf + min(g, L - 1) * d_e) + tg;
+  const uint32_t hstep16 = (uint32_t)(L * d_e) >> 3;         // one expert further, in 16 bytes
+  for (int r = 0; r < nrounds && !dead; ++r) {
+    const int q0 = r * rsz, n = min(rsz, nu - q0);
+    const int nblk = n << pshift;
+    const uint32_t d_base = wbase + (r & 1) * rsz * slot_d;
+    // this warp's k blocks b = warp + 8 i of the round, in batches whose h fragments are all
+    // requested before the first is used; block b = expert b >> pshift, k block b & (npairs - 1)
+    Frag64 fh[kHB];
+    auto load_h = [&](int b0) {
+#pragma unroll
+      for (int i = 0; i < kHB; ++i) {
+        const int b = b0 + kWarps * i;
+        if (b < nblk) {
+          const uint4* hp = hrow + (uint32_t)(q0 + (b >> pshift)) * hstep16 + 8 * (b & (npairs - 1));
+          fh[i].lo = ld_cg_v4(hp);
+          fh[i].hi = ld_cg_v4(hp + 4);
+        }
+      }
+    };
+    load_h(warp);
+    cp_async_wait_group<1>();      // all but the newest group: this round's slabs have landed
+    __syncthreads();
+    for (int b0 = warp; b0 < nblk; b0 += kWarps * kHB) {
+      if (b0 != warp) load_h(b0);
+#pragma unroll
+      for (int i = 0; i < kHB; ++i) {
+        const int b = b0 + kWarps * i;
+        if (b < nblk) {
+          const uint32_t da = d_base + (b >> pshift) * slot_d + 128 * (b & (npairs - 1));
+          const uint4 alo = lds128(da + da_off), ahi = lds128(da + da_off + 64);
+          const uint4 blo = lds128(da + db_off), bhi = lds128(da + db_off + 64);
+          mma64(acc0[0], acc1[0], alo, ahi, blo, bhi, fh[i]);
+        }
+      }
+    }
+    __syncthreads();               // every warp is done with this round's slabs
+    if (r + 2 < nrounds) issue_d(r + 2);
+    cp_async_commit();
+  }
+  cp_async_wait_all();
+  if (!waited) pdl_wait();         // out (and x_next) may still be in use by the call before
+  if (!dead) {
+    if (nu > 0) {
+      store_partial<1>(red + warp * 128, 16, 0, acc0, acc1, g, tg);
+      __syncthreads();
+      if (tid < 128) {
+        const int t = tid >> 4, m = tid & 15;
+        if (t < L && m < ncols) {
+          float v = 0.0f;
+#pragma unroll
+          for (int w = 0; w < kWarps; ++w) v += red[w * 128 + tid];
+          const int o = t * d + c0 + m;
+          if (p.accumulate) v += EARLY < 2 ? resid : __ldcg(p.out + o);
+          p.out[o] = v;
+          if (p.x_next) p.x_next[o] = (uint16_t)f32_to_bf16_bits(v);
+        }
+      }
+    } else {                       // empty union: FFN(x) = 0
+      for (int e = tid; e < L * ncols; e += kThreads) {
+        const int t = e / ncols, m = e - t * ncols;
+        const int o = t * d + c0 + m;
+        const float v = p.accumulate ? __ldcg(p.out + o) : 0.0f;
+        p.out[o] = v;
+        if (p.x_next) p.x_next[o] = (uint16_t)f32_to_bf16_bits(v);
+      }
+    }
+  }
+  // CTA 0 publishes the routing it derived (after the wait: earlier readers are done)
+  if (blockIdx.x == 0) {
+    if (p.lg.a0 != nullptr && p.pub_scores != nullptr) {
+      const int words = (p.E + 31) >> 5;
+      const float* rinv = reinterpret_cast<const float*>(ctl + 104);
+      for (int t = warp; t < L; t += kWarps) {
+        for (int w = 0; w < words; ++w) {
+          const int e = 32 * w + lane;
+          float sv = 0.0f;
+          if (e < p.E) {
+            float v = __ldcg(p.lg.a0 + (size_t)t * p.E + e);
+            v = v > 0.0f ? v : 0.0f;
+            sv = __ldg(p.lg.gain + e) * v * rinv[t];
+            p.pub_scores[(size_t)t * p.E + e] = sv;
+          }
+          const uint32_t m = __ballot_sync(0xffffffffu, sv != 0.0f);
+          if (p.pub_tok && lane == 0) p.pub_tok[(size_t)t * words + w] = m;
+        }
+      }
+    }
+    if (p.ids_in == nullptr) {
+      const int words = (p.E + 31) >> 5;
+      const uint32_t* um = reinterpret_cast<const uint32_t*>(ctl + 8);
+      for (int e = tid; e < p.E; e += kThreads) {
+        if (p.pub_ids) p.pub_ids[e] = e < nu ? ids_sm[e] : -1;
+        if (p.pub_mask && e < words) p.pub_mask[e] = um[e];
+      }
+      if (tid == 0) {
+        if (p.pub_n) *p.pub_n = nu;
+        if (p.stats) {
+          atomicAdd(reinterpret_cast<unsigned long long*>(&p.stats->n_tokens),
+                    (unsigned long long)L);
+          atomicAdd(reinterpret_cast<unsigned long long*>(&p.stats->n_active),
+                    (unsigned long long)ctl[2]);
+          atomicAdd(reinterpret_cast<unsigned long long*>(&p.stats->n_chunks), 1ull);
+          atomicAdd(reinterpret_cast<unsigned long long*>(&p.stats->n_union),
+                    (unsigned long long)nu);
+        }
+      }
+    } else if (tid == 0 && ctl[3]) {
+      atomicOr(p.status, (uint32_t)ctl[3]);
+    }
+  }
+}
+
+// ---- host side ---------------------------------------------------------------------------
+struct LeanPlan {
+  int cap_bytes, red_rows, max_cols, cols_q, cols_rem, smem, kb;
+  bool ok;
+};
+
+// Shapes: L <= 8; d a multiple of 64 up to 2048 (x fragments of a warp fit its registers);
+// d_e a power of two >= 64; at most 16 output columns per CTA. The shared memory of a CTA is
+// sized for the union the caller expects (or the paper's sparsity, see make_plan of the
+// two-kernel form): three CTAs per SM when its share fits a third of an SM, else two, else one;
+// larger unions still run, in stages.
+LeanPlan lean_plan(const blockffn_config& cfg, int L, int grid) {
+  LeanPlan pl{};
+  pl.ok = false;
+  const int d = cfg.d, d_e = cfg.d_e, E = cfg.E;
+  if (L < 1 || L > 8 || grid < 1) return pl;
+  if (d % 64 || d > 512 * kMaxKB || d_e % 64 || (d_e & (d_e - 1)) || d_e > 4096 || E > 1024)
+    return pl;
+  if (d > 16 * grid) return pl;    // one column tile per CTA
+  pl.kb = (d / 64 + kWarps - 1) / kWarps;
+  pl.cols_q = d / grid;
+  pl.cols_rem = d % grid;
+  pl.max_cols = pl.cols_q + (pl.cols_rem ? 1 : 0);
+  int u_exp = (cfg.flags >> 17) & 0x7ff;
+  if (u_exp == 0) u_exp = (L == 1 ? E + 4 : 3 * E + 5) / (L == 1 ? 8 : 10);
+  if (u_exp < 1) u_exp = 1;
+  if (u_exp > E) u_exp = E;
+  const int rows_exp = (u_exp * d_e + grid - 1) / grid;
+  const int slot_d = pl.max_cols * 2 * d_e + 64;          // columns split even / odd around 64 bytes
+  const int need = max(rows_exp * 2 * d + 64, u_exp * slot_d);
+  const int base = kOffIds + align128(E * 4);
+  for (int per_sm = 3; per_sm >= 1; --per_sm) {
+    const int budget = (per_sm == 1 ? kSmemMax : (kSmemMax + 1024) / per_sm - 1024) & ~127;
+    // the up partial tile is as wide as a stage can be: the expected share, at most 32 rows
+    int red_rows = rows_exp < 32 ? rows_exp : 32;
+    if (red_rows < 8) red_rows = 8;
+    const int fixed = lean_layout(E, red_rows, 0).total;
+    const int cap = budget - fixed;
+    if (cap < need && per_sm > 1) continue;
+    if (cap < 2 * 2 * d + 128 || cap < 2 * slot_d) return pl;     // not even two rows / two slabs
+    pl.cap_bytes = cap & ~127;
+    // with room to spare let a stage hold up to 32 rows (two mma row tiles)
+    while (red_rows < 32 && (red_rows + 1) * 2 * d + 64 <= pl.cap_bytes &&
+           lean_layout(E, red_rows + 1, pl.cap_bytes).total <= budget)
+      ++red_rows;
+    pl.red_rows = red_rows;
+    pl.cap_bytes = (budget - lean_layout(E, red_rows, 0).total) & ~127;
+    pl.smem = lean_layout(E, red_rows, pl.cap_bytes).total;
+    (void)base;
+    pl.ok = pl.smem <= kSmemMax;
+    return pl;
+  }
+  return pl;
+}
+
+template <int KB, int MODE, int EARLY>
+cudaError_t lean_attr() {
+  const void* f = reinterpret_cast<const void*>(&expert_lean_kernel<KB, MODE, EARLY>);
+  cudaError_t e = cudaFuncSetAttribute(f, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemMax);
+  if (e != cudaSuccess) return e;
+  return cudaFuncSetAttribute(f, cudaFuncAttributePreferredSharedMemoryCarveout,
+                              cudaSharedmemCarveoutMaxShared);
+}
+template <int KB>
+cudaError_t lean_attrs_kb() {
+  cudaError_t e = lean_attr<KB, 0, 0>();
+  if (e == cudaSuccess) e = lean_attr<KB, 0, 1>();
+  if (e == cudaSuccess) e = lean_attr<KB, 0, 2>();
+  if (e == cudaSuccess) e = lean_attr<KB, 1, 0>();
+  if (e == cudaSuccess) e = lean_attr<KB, 1, 1>();
+  if (e == cudaSuccess) e = lean_attr<KB, 1, 2>();
+  if (e == cudaSuccess) e = lean_attr<KB, 2, 0>();
+  if (e == cudaSuccess) e = lean_attr<KB, 2, 2>();
+  return e;
+}
+
+template <int KB, int MODE>
+cudaError_t lean_launch_mode(const cudaLaunchConfig_t& lc, const LeanParams& p, int early) {
+  if constexpr (MODE == 2) {
+    return early == 2 ? cudaLaunchKernelEx(&lc, expert_lean_kernel<KB, 2, 2>, p)
+                      : cudaLaunchKernelEx(&lc, expert_lean_kernel<KB, 2, 0>, p);
+  } else {
+    return early == 2   ? cudaLaunchKernelEx(&lc, expert_lean_kernel<KB, MODE, 2>, p)
+           : early == 1 ? cudaLaunchKernelEx(&lc, expert_lean_kernel<KB, MODE, 1>, p)
+                        : cudaLaunchKernelEx(&lc, expert_lean_kernel<KB, MODE, 0>, p);
+  }
+}
+template <int KB>
+cudaError_t lean_launch_kb(const cudaLaunchConfig_t& lc, const LeanParams& p, int mode, int early) {
+  return mode == 2   ? lean_launch_mode<KB, 2>(lc, p, early)
+         : mode == 1 ? lean_launch_mode<KB, 1>(lc, p, early)
+                     : lean_launch_mode<KB, 0>(lc, p, early);
+}
+
+}  // namespace
+
+bool expert_lean_supported(const blockffn_ctx* c, int L) {
+  return c->lean_ring != nullptr && !(c->cfg.flags & BLOCKFFN_CFG_TWO_KERNELS) &&
+         lean_plan(c->cfg, L, c->num_sms).ok;
+}
+
+// Ring of kHRing intermediates of a chunk of 8 tokens; 0 when the shape never takes this kernel
+// (or the ring would be unreasonably large).
+size_t expert_lean_ws_bytes(const blockffn_config* cfg, int grid) {
+  if (!lean_plan(*cfg, cfg->L_max < 8 ? cfg->L_max : 8, grid).ok) return 0;
+  const size_t slot = ((size_t)cfg->E * 8 * cfg->d_e * sizeof(uint16_t) + 255) & ~(size_t)255;
+  if (kHRing * slot > ((size_t)64 << 20)) return 0;
+  return kHRing * slot;
+}
+
+cudaError_t expert_lean_setup(blockffn_ctx* c) {
+  (void)c;
+  cudaError_t e = lean_attrs_kb<1>();
+  if (e == cudaSuccess) e = lean_attrs_kb<2>();
+  if (e == cudaSuccess) e = lean_attrs_kb<3>();
+  if (e == cudaSuccess) e = lean_attrs_kb<4>();
+  return e;
+}
+
+cudaError_t launch_expert_lean(blockffn_ctx* c, const blockffn_weights* w, const void* x,
+                               const float* scores, int L, const int32_t* union_ids,
+                               const int32_t* n_union, float* out, void* x_next, int call_flags,
+                               const RoutingOut* pub, const RouterLogits* logits, bool logits_final,
+                               cudaStream_t st) {
+  const LeanPlan pl = lean_plan(c->cfg, L, c->num_sms);
+  if (!pl.ok || !c->lean_ring) return cudaErrorNotSupported;
+  LeanParams p{};
+  p.x = static_cast<const uint16_t*>(x);
+  p.U = static_cast<const uint16_t*>(w->U);
+  p.D = static_cast<const uint16_t*>(w->D);
+  p.scores = scores;
+  if (logits) p.lg = *logits;
+  p.ids_in = union_ids;
+  p.n_in = n_union;
+  p.h_ring = static_cast<uint16_t*>(c->lean_ring);
+  p.h_slot = (((size_t)c->cfg.E * 8 * c->cfg.d_e * sizeof(uint16_t) + 255) & ~(size_t)255) / 2;
+  p.seq = c->lean_seq;
+  p.ready = c->lean_seq + 1;
+  p.out = out;
+  p.x_next = static_cast<uint16_t*>(x_next);
+  p.L = L;
+  p.d = c->cfg.d;
+  p.E = c->cfg.E;
+  p.d_e = c->cfg.d_e;
+  p.de_shift = __builtin_ctz(c->cfg.d_e);
+  p.cap_bytes = pl.cap_bytes;
+  p.red_rows = pl.red_rows;
+  p.max_cols = pl.max_cols;
+  p.cols_q = pl.cols_q;
+  p.cols_rem = pl.cols_rem;
+  p.accumulate = (call_flags & BLOCKFFN_CALL_ACCUMULATE) ? 1 : 0;
+  p.hold = (c->cfg.flags & BLOCKFFN_CFG_TEST_EXPIRE_WAIT) ? 1 : 0;
+  p.wait_ns = 1000000000ull;      // one second
+  p.status = c->status;
+  if (pub) {
+    p.pub_mask = pub->union_mask;
+    p.pub_ids = pub->union_ids;
+    p.pub_n = pub->n_union;
+    p.stats = pub->stats;
+    p.pub_scores = pub->scores;
+    p.pub_tok = pub->tok_mask;
+  }
+  const bool chained = !(c->cfg.flags & BLOCKFFN_CFG_NO_CHAINING);
+  const int early = logits ? (logits_final ? 2 : 0)
+                    : (call_flags & BLOCKFFN_CALL_INDEPENDENT_X) ? 2
+                    : (call_flags & BLOCKFFN_CALL_INDEPENDENT)   ? 1
+                                                                 : 0;
+  const int mode = logits ? 2 : union_ids ? 1 : 0;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cudaLaunchConfig_t lc{};
+  lc.gridDim = dim3(c->num_sms);
+  lc.blockDim = dim3(kThreads);
+  lc.stream = st;
+  lc.attrs = attr;
+  lc.numAttrs = chained ? 1 : 0;
+  lc.dynamicSmemBytes = pl.smem;
+  cudaError_t e;
+  switch (pl.kb) {
+    case 1: e = lean_launch_kb<1>(lc, p, mode, early); break;
+    case 2: e = lean_launch_kb<2>(lc, p, mode, early); break;
+    case 3: e = lean_launch_kb<3>(lc, p, mode, early); break;
+    default: e = lean_launch_kb<4>(lc, p, mode, early); break;
+  }
+  if (e == cudaSuccess) c->launches += 1;
+  return e;
+}

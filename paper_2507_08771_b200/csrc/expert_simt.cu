@@ -8,6 +8,8 @@
 // rows of D for that column and over h, reduces, and writes out[t][c] (optionally
 // accumulating into an fp32 residual and emitting its bf16 rounding).
 // No atomics: every output element has exactly one writer.
+#include <mutex>
+
 #include "common.cuh"
 
 namespace {
@@ -198,8 +200,14 @@ namespace {
 constexpr int kMaxDevices = 64;
 // Device address of g_noalloc_scratch per device, looked up once per device. In host code
 // the array's name is only a handle for the runtime, never an address a kernel may be given.
-unsigned char* g_noalloc_ptr[kMaxDevices] = {};
-int g_noalloc_sms[kMaxDevices] = {};
+// The pair (address, SM count) of a device is written and read under the mutex, so that a
+// second host thread never sees one without the other.
+struct NoallocDevice {
+  unsigned char* ptr;
+  int sms;
+};
+NoallocDevice g_noalloc_dev[kMaxDevices] = {};
+std::mutex g_noalloc_mutex;
 }  // namespace
 
 extern "C" blockffn_status blockffn_expert_ffn_noalloc(
@@ -225,30 +233,35 @@ extern "C" blockffn_status blockffn_expert_ffn_noalloc(
     return BLOCKFFN_ERR_INVALID_ARG;
   int dev = -1;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return BLOCKFFN_ERR_CUDA;
-  if (!g_noalloc_ptr[dev]) {   // first call on this device, with this device current
-    unsigned char* ptr = nullptr;
-    int sms = 0;
-    if (cudaGetSymbolAddress(reinterpret_cast<void**>(&ptr), g_noalloc_scratch) != cudaSuccess ||
-        !ptr ||
-        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) {
-      cudaGetLastError();
-      return BLOCKFFN_ERR_CUDA;
+  NoallocDevice nd;
+  {
+    std::lock_guard<std::mutex> lock(g_noalloc_mutex);
+    if (!g_noalloc_dev[dev].ptr) {   // first call on this device, with this device current
+      unsigned char* ptr = nullptr;
+      int sms = 0;
+      if (cudaGetSymbolAddress(reinterpret_cast<void**>(&ptr), g_noalloc_scratch) != cudaSuccess ||
+          !ptr ||
+          cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) {
+        cudaGetLastError();
+        return BLOCKFFN_ERR_CUDA;
+      }
+      g_noalloc_dev[dev].sms = sms;
+      g_noalloc_dev[dev].ptr = ptr;
     }
-    g_noalloc_sms[dev] = sms;
-    g_noalloc_ptr[dev] = ptr;
+    nd = g_noalloc_dev[dev];
   }
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   // The status word is shared by all calls and keeps its last value: start it at zero.
-  if (cudaMemsetAsync(g_noalloc_ptr[dev], 0, BLOCKFFN_NOALLOC_HEADER, st) != cudaSuccess)
+  if (cudaMemsetAsync(nd.ptr, 0, BLOCKFFN_NOALLOC_HEADER, st) != cudaSuccess)
     return BLOCKFFN_ERR_CUDA;
   blockffn_ctx tmp{};          // a view for the launcher: nothing in it owns memory
   tmp.cfg = *cfg;
   tmp.cfg.L_max = L;           // h is laid out [q][L][d_e]
   tmp.device = dev;
-  tmp.num_sms = g_noalloc_sms[dev];
+  tmp.num_sms = nd.sms;
   tmp.words = (cfg->E + 31) / 32;
-  tmp.status = reinterpret_cast<uint32_t*>(g_noalloc_ptr[dev]);
-  tmp.h32 = reinterpret_cast<float*>(g_noalloc_ptr[dev] + BLOCKFFN_NOALLOC_HEADER);
+  tmp.status = reinterpret_cast<uint32_t*>(nd.ptr);
+  tmp.h32 = reinterpret_cast<float*>(nd.ptr + BLOCKFFN_NOALLOC_HEADER);
   const cudaError_t e =
       launch_expert_simt(&tmp, w, x, scores, L, union_ids, n_union, out, x_next, call_flags, st);
   return e == cudaSuccess ? BLOCKFFN_OK : BLOCKFFN_ERR_CUDA;
