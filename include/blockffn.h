@@ -88,6 +88,12 @@ typedef struct {
  * SM; this bit selects the older two-kernel form (up projection, down projection) for them
  * too. Same results within the tolerance; kept for comparison and as the path of longer chunks. */
 #define BLOCKFFN_CFG_TWO_KERNELS 0x20000000
+/* The one-kernel form runs a call whose x is promised stable (BLOCKFFN_CALL_INDEPENDENT_X) on
+ * a third of the SMs, so that three times as many such calls are in flight: every CTA reads all
+ * of x and of the intermediate from L2, and fewer, larger CTAs per call keep that broadcast
+ * small next to the weight stream. This bit gives those calls the whole device each, like the
+ * calls of a dependent chain.                                                              */
+#define BLOCKFFN_CFG_NO_SPLIT 0x40000000
 /* Test aid: the one-kernel form's hand-over waits for an arrival that never comes, gives up
  * after two milliseconds, sets BLOCKFFN_DEV_WAIT_EXPIRED and leaves out untouched. Exercises
  * the bounded wait without any fault.                                                      */

@@ -26,6 +26,7 @@ CALL_ACCUMULATE, CALL_INDEPENDENT, CALL_INDEPENDENT_X = 1, 2, 4
 CFG_NO_CHAINING = 0x10000
 CFG_TWO_KERNELS = 0x20000000
 CFG_TEST_EXPIRE_WAIT = 0x10000000
+CFG_NO_SPLIT = 0x40000000
 
 
 def cfg_expected_union(u: int) -> int:

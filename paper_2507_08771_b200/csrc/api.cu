@@ -87,7 +87,7 @@ blockffn_status blockffn_create(const blockffn_config* cfg, blockffn_handle* out
   if (!(cfg->rms_eps >= 0.0f)) return BLOCKFFN_ERR_INVALID_ARG;
   if (cfg->variant < BLOCKFFN_VARIANT_AUTO || cfg->variant > BLOCKFFN_VARIANT_MMA)
     return BLOCKFFN_ERR_INVALID_ARG;
-  if (cfg->flags & ~0x3fffffff) return BLOCKFFN_ERR_INVALID_ARG;
+  if (cfg->flags & ~0x7fffffff) return BLOCKFFN_ERR_INVALID_ARG;
   if (((cfg->flags >> 17) & 0x7ff) > cfg->E) return BLOCKFFN_ERR_INVALID_ARG;
   blockffn_ctx* c = new (std::nothrow) blockffn_ctx();
   if (!c) return BLOCKFFN_ERR_WORKSPACE;
@@ -119,7 +119,7 @@ blockffn_status blockffn_create(const blockffn_config* cfg, blockffn_handle* out
   const size_t o_h16 = take(expert_mma_h_bytes(cfg));
   const size_t lean_bytes = expert_lean_ws_bytes(cfg, c->num_sms);
   const size_t o_lean = take(lean_bytes);
-  const size_t o_seq = take(sizeof(unsigned long long) * 16);
+  const size_t o_seq = take(sizeof(unsigned long long) * 64);
   const size_t o_tk = take(sizeof(unsigned int) * 8);
   const size_t o_st = take(sizeof(uint32_t));
   void* base = nullptr;

@@ -13,7 +13,7 @@
 //   CTA b, call n:
 //     ticket           one atomic per CTA on the handle's call counter; ticket / grid is the
 //                      call's index n (all CTAs of a call take theirs before any CTA of the next
-//                      call exists, see below), n mod 8 its slot in the ring of h buffers
+//                      call exists, see below), n mod 16 its slot in the ring of h buffers
 //     Union(x)         derived by every CTA from the scores, the caller's list or raw logits
 //     up projection    the CTA's share of the union's neuron rows -> shared memory (16-byte
 //                      asynchronous copies), K split over the 8 warps, mma.sync m16n8k16 with
@@ -29,32 +29,36 @@
 //
 // Ordering between calls. Kernels are chained by programmatic dependent launch and trigger
 // their dependents only once the CTA holds its ticket, so tickets of successive calls never
-// interleave. Every kernel waits for its predecessor before it ends; a CTA of call n + R can
-// therefore exist only if fewer than R calls are incomplete, R - 1 being the number of CTAs
-// that fit one SM. With R = 8 ring slots (at most 7 CTAs of 256 threads... fit the 2048-thread
-// SM together with the CTA that replaces them) a slot is never reused while a CTA of its earlier
-// call is alive, and its arrival counter is an exact multiple of the grid size when a call
-// starts: the counters only ever grow, nothing is reset, graph replays need no host state.
+// interleave. Every kernel waits for its predecessor before it ends, so no CTA of a call exits
+// while an earlier call is incomplete: when a CTA of call n + R exists and call n is incomplete,
+// all CTAs of calls n + 1 .. n + R - 1 are resident, plus one of each end, i.e.
+// (R - 1) grid + 2 <= 3 SMs CTAs (the kernel is compiled for three CTAs per SM). With a grid of
+// a third of the SMs (calls that share the device) that allows R <= 9; the ring has 16 slots,
+// so a slot is never reused while a CTA of its earlier call is alive, and its arrival counter is
+// an exact multiple of the grid size when a call starts: the counters only ever grow, nothing is
+// reset, graph replays need no host state. Calls that own the device and calls that share it
+// have grids of different size and therefore a ring and a ticket counter each.
 // The polling thread issues no asynchronous copies: a fence or an acquire by a thread waits
 // for that thread's own copies in flight.
 #include "mma_tiles.cuh"
 
 namespace {
 
-constexpr int kHRing = 8;            // h buffers and arrival counters per handle
+constexpr int kHRing = 16;           // h buffers and arrival counters per ring (see the bound above)
+constexpr int kMinSmem = 60 * 1024;  // four such CTAs do not fit one SM (228 KB, 1 KB reserved each)
 constexpr int kSyncThread = kThreads - 1;
 constexpr int kCopyThreads = kThreads - 32;   // the last warp (the polling thread's) issues no D copies
 constexpr int kMaxKB = 4;            // 64-wide k blocks of x per warp: d <= 8 * 64 * kMaxKB
-constexpr int kHB = 5;               // h fragments a warp keeps in registers per batch
 
 struct LeanLayout {
   int off_red, off_w, total;
 };
-// red: cross-warp partials, up [8 warps][8 tokens][red_rows] f32, down [8 warps][8][16] f32
+// red: cross-warp partials [8 tokens][rows][8 warps] f32, rows = red_rows (up) or 16 per column
+// tile (down); red_rows is at least 16 (32 with two column tiles)
 __host__ __device__ inline LeanLayout lean_layout(int E, int red_rows, int cap_bytes) {
   LeanLayout s;
   s.off_red = kOffIds + align128(E * 4);
-  const int red = kWarps * 8 * 4 * (red_rows > 16 ? red_rows : 16);
+  const int red = kWarps * 8 * 4 * red_rows;
   s.off_w = s.off_red + align128(red);
   s.total = s.off_w + cap_bytes;
   return s;
@@ -76,6 +80,9 @@ struct LeanParams {
   uint16_t* x_next;
   int L, d, E, d_e, de_shift;
   int cap_bytes, red_rows;     // weight region; rows the up partial tile is sized for
+  int cap_rows, cap_slabs;     // rows of U / slabs of D the region holds (paddings included)
+  uint32_t magic_g;            // ceil(2^32 / grid): R / grid = mulhi(R, magic_g) for R < 2^24
+  uint32_t magic_cpr;          // ceil(2^16 / (d / 8)): tid / (d / 8) = tid * magic_cpr >> 16
   int max_cols, cols_q, cols_rem;
   int accumulate;
   int hold;                    // test aid: wait for an arrival that never comes
@@ -146,7 +153,8 @@ __device__ __forceinline__ void mma64(float (&c0)[4], float (&c1)[4], const uint
 
 // KB: 64-wide k blocks of x per warp (ceil(d / 512)); MODE as derive_union; EARLY: 0 wait first,
 // 1 routing inputs and weights before the wait, 2 x as well (the wait then comes before out).
-template <int KB, int MODE, int EARLY>
+// NC: 16-column tiles of out per CTA (1 .. 4).
+template <int KB, int NC, int MODE, int EARLY>
 __global__ void __launch_bounds__(kThreads, 3) expert_lean_kernel(const LeanParams p) {
   extern __shared__ __align__(128) unsigned char smem[];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -177,7 +185,7 @@ __global__ void __launch_bounds__(kThreads, 3) expert_lean_kernel(const LeanPara
     const unsigned long long n = ticket / (unsigned)G;
     ctl[6] = (int)(n & (kHRing - 1));
     *reinterpret_cast<unsigned long long*>(ctl + 138) =
-        p.hold ? ~0ull : ((n >> 3) + 1ull) * (unsigned)G;
+        p.hold ? ~0ull : (n / kHRing + 1ull) * (unsigned)G;
     pdl_trigger();
   };
   const int nu = derive_union<MODE>(p.scores, p.lg, p.ids_in, p.n_in, L, p.E, ids_sm, ctl,
@@ -185,22 +193,24 @@ __global__ void __launch_bounds__(kThreads, 3) expert_lean_kernel(const LeanPara
 
   // ---- up projection ---------------------------------------------------------------------
   const int R = nu * d_e;
-  const int rq = R / G, rrem = R - rq * G;
+  const int rq = (int)__umulhi((unsigned)R, p.magic_g), rrem = R - rq * G;
   const int r0 = bx * rq + min(bx, rrem), nrows = rq + (bx < rrem ? 1 : 0), r1 = r0 + nrows;
   const int row_bytes = 2 * d;
-  const int cap_rows = min((p.cap_bytes - 128) / row_bytes, 2 * p.red_rows);
-  const bool single = nrows <= min(p.red_rows, cap_rows);
-  const int slot_rows = single ? max(nrows, 1) : min(p.red_rows, cap_rows / 2);
-  const int ngroups = (nrows + slot_rows - 1) / slot_rows;
-  const int rpg = ngroups ? (nrows + ngroups - 1) / ngroups : 0;
+  const int cap_rows = p.cap_rows;
+  // one stage when the share fits (the usual case: no division on that path), else stages of
+  // half the region that are refilled as they free
+  const int ldr = min(p.red_rows, 32);       // a stage is at most two row tiles
+  const bool single = nrows <= min(ldr, cap_rows);
+  const int slot_rows = single ? max(nrows, 1) : min(ldr, cap_rows / 2);
+  const int ngroups = single ? (nrows > 0 ? 1 : 0) : (nrows + slot_rows - 1) / slot_rows;
+  const int rpg = single ? nrows : (nrows + ngroups - 1) / ngroups;
   const int half_u = ((slot_rows + 1) >> 1) * row_bytes + 64;   // where the odd rows start
   const int slot_bytes = slot_rows * row_bytes + 64;
   const int sh = p.de_shift;
-  const int ldr = p.red_rows;
   // This thread's part of a row copy: 16-byte chunk my_c of the rows my_sub, my_sub + rpi, ...
   const int cpr = d >> 3;                       // chunks per row (<= 256)
-  const int rpi = kThreads / cpr;               // rows the CTA copies per step
-  const int my_sub = tid / cpr, my_c = tid - my_sub * cpr;
+  const int rpi = cpr > 128 ? 1 : kThreads / cpr;   // rows the CTA copies per step
+  const int my_sub = (tid * p.magic_cpr) >> 16, my_c = tid - my_sub * cpr;
   const bool copies_u = my_sub < rpi;
   // stage gi: rows [r0 + gi rpg, ...) -> slot gi & 1, row m of the stage at
   // (m >> 1) row_bytes + (m & 1) half_u
@@ -208,14 +218,40 @@ __global__ void __launch_bounds__(kThreads, 3) expert_lean_kernel(const LeanPara
     const int ra = r0 + gi * rpg;
     const int rows = min(r1, ra + rpg) - ra;
     const uint32_t slot0 = wbase + (gi & 1) * slot_bytes + my_c * 16;
-    if (copies_u) {
-      int m = my_sub;
+    if (!copies_u) return;
+    if (rpi == 1) {
+      // every thread walks all rows: two running destinations (even rows, odd rows), the
+      // source index steps by one row inside an expert and jumps at an expert's end
+      uint32_t de = slot0, dd = slot0 + half_u;
+      int m = 0;
       while (m < rows) {
         const int r = ra + m, q = r >> sh;
         const int seg_end = min(rows, ((q + 1) << sh) - ra);     // rows of this expert end here
         uint32_t idx = (uint32_t)(ids_sm[q] * d_e + (r - (q << sh))) * (uint32_t)cpr + my_c;
+        if (m & 1) {               // start on an even row of the stage
+          cp_async16(dd, at16(p.U, idx));
+          dd += row_bytes;
+          idx += cpr;
+          ++m;
+        }
+#pragma unroll 2
+        for (; m + 1 < seg_end; m += 2, idx += 2 * cpr, de += row_bytes, dd += row_bytes) {
+          cp_async16(de, at16(p.U, idx));
+          cp_async16(dd, at16(p.U, idx + cpr));
+        }
+        if (m < seg_end) {
+          cp_async16(de, at16(p.U, idx));
+          de += row_bytes;
+          ++m;
+        }
+      }
+    } else {
+      int m = my_sub;
+      while (m < rows) {
+        const int r = ra + m, q = r >> sh;
+        const int seg_end = min(rows, ((q + 1) << sh) - ra);
+        uint32_t idx = (uint32_t)(ids_sm[q] * d_e + (r - (q << sh))) * (uint32_t)cpr + my_c;
         const uint32_t step = (uint32_t)rpi * cpr;
-#pragma unroll 4
         for (; m < seg_end; m += rpi, idx += step)
           cp_async16(slot0 + (m >> 1) * row_bytes + (m & 1) * half_u, at16(p.U, idx));
       }
@@ -283,8 +319,9 @@ __global__ void __launch_bounds__(kThreads, 3) expert_lean_kernel(const LeanPara
     const uint32_t a0 = row_addr(g), b0 = row_addr(g + 8);
     cp_async_wait_group<1>();      // all but the newest group: this stage has landed
     __syncthreads();
-    float* mine = red + warp * (8 * ldr);
-    const int t2 = 2 * tg;
+    // partial tiles -> red[t][m][warp]: the eight partials of an element are 32 contiguous bytes
+    float* mine = red + (2 * tg * ldr + g) * kWarps + warp;
+    const int nt = ldr * kWarps;           // one token further
     {
       float c0[4] = {0.f, 0.f, 0.f, 0.f}, c1[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
@@ -295,14 +332,13 @@ __global__ void __launch_bounds__(kThreads, 3) expert_lean_kernel(const LeanPara
           mma64(c0, c1, alo, ahi, blo, bhi, fx[i]);
         }
       }
-      // partial tile of this warp -> red[warp][t][m] (rows beyond the tile's width are padding)
       if (g < ldr) {
-        mine[t2 * ldr + g] = c0[0] + c1[0];
-        mine[(t2 + 1) * ldr + g] = c0[1] + c1[1];
+        mine[0] = c0[0] + c1[0];
+        mine[nt] = c0[1] + c1[1];
       }
       if (g + 8 < ldr) {
-        mine[t2 * ldr + g + 8] = c0[2] + c1[2];
-        mine[(t2 + 1) * ldr + g + 8] = c0[3] + c1[3];
+        mine[8 * kWarps] = c0[2] + c1[2];
+        mine[nt + 8 * kWarps] = c0[3] + c1[3];
       }
     }
     if (rows > 16) {               // second tile of 16 rows
@@ -317,22 +353,21 @@ __global__ void __launch_bounds__(kThreads, 3) expert_lean_kernel(const LeanPara
         }
       }
       if (g + 16 < ldr) {
-        mine[t2 * ldr + g + 16] = c0[0] + c1[0];
-        mine[(t2 + 1) * ldr + g + 16] = c0[1] + c1[1];
+        mine[16 * kWarps] = c0[0] + c1[0];
+        mine[nt + 16 * kWarps] = c0[1] + c1[1];
       }
       if (g + 24 < ldr) {
-        mine[t2 * ldr + g + 24] = c0[2] + c1[2];
-        mine[(t2 + 1) * ldr + g + 24] = c0[3] + c1[3];
+        mine[24 * kWarps] = c0[2] + c1[2];
+        mine[nt + 24 * kWarps] = c0[3] + c1[3];
       }
     }
     __syncthreads();               // partials complete; every warp is done with the slot
     if (gi + 2 < ngroups) issue_u(gi + 2);
     cp_async_commit();
     if (hidx >= 0) {
-      const float* col = red + (tid >> 5) * ldr + (tid & 31);
-      float v = 0.0f;
-#pragma unroll
-      for (int w = 0; w < kWarps; ++w) v += col[w * (8 * ldr)];
+      const float4* part = reinterpret_cast<const float4*>(red + ((tid >> 5) * ldr + (tid & 31)) * kWarps);
+      const float4 lo = part[0], hi = part[1];
+      const float v = ((lo.x + lo.y) + (lo.z + lo.w)) + ((hi.x + hi.y) + (hi.z + hi.w));
       hbuf[hidx] = (uint16_t)f32_to_bf16_bits(sc * swish_fast(v));
     }
     if (gi + 1 < ngroups) prepare(gi + 1);
@@ -346,19 +381,19 @@ __global__ void __launch_bounds__(kThreads, 3) expert_lean_kernel(const LeanPara
   }
 
   // ---- down projection -------------------------------------------------------------------
-  // Slab of one expert: the CTA's columns as rows of 2 d_e bytes, even columns first, 64 bytes
-  // of padding, odd columns.
+  // Slab of one expert: the CTA's columns (at most 16 NC, NC mma row tiles) as rows of 2 d_e
+  // bytes, even columns first, 64 bytes of padding, odd columns.
   const int drow = 2 * d_e;
   const int half_d = ((p.max_cols + 1) >> 1) * drow + 64;
   const int slot_d = p.max_cols * drow + 64;
-  const int cap_slabs = p.cap_bytes / slot_d;
-  const int rsz = nu <= cap_slabs ? max(nu, 1) : max(1, cap_slabs / 2);
-  const int nrounds = (nu + rsz - 1) / rsz;
+  const int cap_slabs = p.cap_slabs;
+  const bool one_round = nu <= cap_slabs;
+  const int rsz = one_round ? max(nu, 1) : max(1, cap_slabs / 2);
+  const int nrounds = one_round ? (nu > 0 ? 1 : 0) : (nu + rsz - 1) / rsz;
   const int c0 = bx * p.cols_q + min(bx, p.cols_rem);
   const int ncols = p.cols_q + (bx < p.cols_rem ? 1 : 0);
   // A slab is ncols << kshift chunks of 16 bytes; chunk c = column c >> kshift, piece
-  // c & (2^kshift - 1). Thread tid copies chunks tid, tid + kCopyThreads, ... of every expert
-  // (one chunk per thread at the usual shapes).
+  // c & (2^kshift - 1). Thread tid copies chunks tid, tid + kCopyThreads, ... of every expert.
   const int kshift = sh - 3;                    // log2(chunks per D row)
   const uint32_t estride16 = (uint32_t)d << kshift;
   const int nchunks = tid < kCopyThreads ? ncols << kshift : 0;
@@ -378,11 +413,14 @@ __global__ void __launch_bounds__(kThreads, 3) expert_lean_kernel(const LeanPara
   if (nrounds > 1) issue_d(1);
   cp_async_commit();
   bool waited = EARLY < 2;
-  // the residual this CTA's outputs are added to: asked for as early as out may be read
-  float resid = 0.0f;
-  if (waited && p.accumulate && tid < 128) {
-    const int t = tid >> 4, m = tid & 15;
-    if (t < L && m < ncols) resid = __ldcg(p.out + t * d + c0 + m);
+  // the residual this CTA's outputs are added to (thread tid: token tid / 32, columns tid % 32
+  // and, with more than two column tiles, 32 further): asked for as early as out may be read
+  const int ot = tid >> 5, om = tid & 31;
+  float resid[(NC + 1) / 2] = {};
+  if (waited && p.accumulate && ot < L) {
+#pragma unroll
+    for (int k = 0; k < (NC + 1) / 2; ++k)
+      if (om + 32 * k < ncols) resid[k] = __ldcg(p.out + ot * d + c0 + om + 32 * k);
   }
   // hand-over: all CTAs of this call have stored their part of h
   if (tid == kSyncThread) {
@@ -409,15 +447,22 @@ __global__ void __launch_bounds__(kThreads, 3) expert_lean_kernel(const LeanPara
 
   const int npairs = d_e >> 6;      // 64-wide k blocks per expert (a power of two)
   const int pshift = sh - 6;
-  float acc0[1][4], acc1[1][4];
-  zero_acc<1>(acc0);
-  zero_acc<1>(acc1);
-  // rows (columns of out) g and g + 8 of a slab, clamped to the CTA's columns
+  float acc[NC][2][4];
+#pragma unroll
+  for (int c = 0; c < NC; ++c)
+#pragma unroll
+    for (int v = 0; v < 4; ++v) acc[c][0][v] = acc[c][1][v] = 0.0f;
+  // rows (columns of out) g, g + 8 (, g + 16, g + 24) of a slab, clamped to the CTA's columns
   auto col_off = [&](int m) {
     m = min(m, max(ncols, 1) - 1);
     return (m >> 1) * drow + (m & 1) * half_d + 16 * tg;
   };
-  const uint32_t da_off = col_off(g), db_off = col_off(g + 8);
+  uint32_t offs[NC][2];
+#pragma unroll
+  for (int c = 0; c < NC; ++c) {
+    offs[c][0] = col_off(g + 16 * c);
+    offs[c][1] = col_off(g + 16 * c + 8);
+  }
   const uint4* hrow = reinterpret_cast<const uint4*>(hbuf + min(g, L - 1) * d_e) + tg;
   const uint32_t hstep16 = (uint32_t)(L * d_e) >> 3;         // one expert further, in 16 bytes
   for (int r = 0; r < nrounds && !dead; ++r) {
@@ -426,6 +471,9 @@ __global__ void __launch_bounds__(kThreads, 3) expert_lean_kernel(const LeanPara
     const uint32_t d_base = wbase + (r & 1) * rsz * slot_d;
     // this warp's k blocks b = warp + 8 i of the round, in batches whose h fragments are all
     // requested before the first is used; block b = expert b >> pshift, k block b & (npairs - 1)
+    // (fewer per batch with more column tiles: their accumulators need the registers, and a
+    // round then holds fewer experts anyway)
+    constexpr int kHB = NC == 1 ? 5 : NC == 2 ? 3 : 2;
     Frag64 fh[kHB];
     auto load_h = [&](int b0) {
 #pragma unroll
@@ -448,9 +496,12 @@ __global__ void __launch_bounds__(kThreads, 3) expert_lean_kernel(const LeanPara
         const int b = b0 + kWarps * i;
         if (b < nblk) {
           const uint32_t da = d_base + (b >> pshift) * slot_d + 128 * (b & (npairs - 1));
-          const uint4 alo = lds128(da + da_off), ahi = lds128(da + da_off + 64);
-          const uint4 blo = lds128(da + db_off), bhi = lds128(da + db_off + 64);
-          mma64(acc0[0], acc1[0], alo, ahi, blo, bhi, fh[i]);
+#pragma unroll
+          for (int c = 0; c < NC; ++c) {
+            const uint4 alo = lds128(da + offs[c][0]), ahi = lds128(da + offs[c][0] + 64);
+            const uint4 blo = lds128(da + offs[c][1]), bhi = lds128(da + offs[c][1] + 64);
+            mma64(acc[c][0], acc[c][1], alo, ahi, blo, bhi, fh[i]);
+          }
         }
       }
     }
@@ -462,24 +513,34 @@ __global__ void __launch_bounds__(kThreads, 3) expert_lean_kernel(const LeanPara
   if (!waited) pdl_wait();         // out (and x_next) may still be in use by the call before
   if (!dead) {
     if (nu > 0) {
-      store_partial<1>(red + warp * 128, 16, 0, acc0, acc1, g, tg);
-      __syncthreads();
-      if (tid < 128) {
-        const int t = tid >> 4, m = tid & 15;
-        if (t < L && m < ncols) {
-          float v = 0.0f;
+      // partial tiles -> red[t][m][warp] (m < 16 NC), then one thread per output element
+      float* mine = red + (2 * tg * (16 * NC) + g) * kWarps + warp;
 #pragma unroll
-          for (int w = 0; w < kWarps; ++w) v += red[w * 128 + tid];
-          const int o = t * d + c0 + m;
-          if (p.accumulate) v += EARLY < 2 ? resid : __ldcg(p.out + o);
-          p.out[o] = v;
-          if (p.x_next) p.x_next[o] = (uint16_t)f32_to_bf16_bits(v);
+      for (int c = 0; c < NC; ++c) {
+        mine[(16 * c) * kWarps] = acc[c][0][0] + acc[c][1][0];
+        mine[(16 * NC + 16 * c) * kWarps] = acc[c][0][1] + acc[c][1][1];
+        mine[(16 * c + 8) * kWarps] = acc[c][0][2] + acc[c][1][2];
+        mine[(16 * NC + 16 * c + 8) * kWarps] = acc[c][0][3] + acc[c][1][3];
+      }
+      __syncthreads();
+      if (ot < L) {
+#pragma unroll
+        for (int k = 0; k < (NC + 1) / 2; ++k) {
+          const int m = om + 32 * k;
+          if (m < ncols) {
+            const float4* part = reinterpret_cast<const float4*>(red + (ot * (16 * NC) + m) * kWarps);
+            const float4 lo = part[0], hi = part[1];
+            float v = ((lo.x + lo.y) + (lo.z + lo.w)) + ((hi.x + hi.y) + (hi.z + hi.w));
+            const int o = ot * d + c0 + m;
+            if (p.accumulate) v += EARLY < 2 ? resid[k] : __ldcg(p.out + o);
+            p.out[o] = v;
+            if (p.x_next) p.x_next[o] = (uint16_t)f32_to_bf16_bits(v);
+          }
         }
       }
-    } else {                       // empty union: FFN(x) = 0
-      for (int e = tid; e < L * ncols; e += kThreads) {
-        const int t = e / ncols, m = e - t * ncols;
-        const int o = t * d + c0 + m;
+    } else if (ot < L) {           // empty union: FFN(x) = 0
+      for (int m = om; m < ncols; m += 32) {
+        const int o = ot * d + c0 + m;
         const float v = p.accumulate ? __ldcg(p.out + o) : 0.0f;
         p.out[o] = v;
         if (p.x_next) p.x_next[o] = (uint16_t)f32_to_bf16_bits(v);
@@ -533,120 +594,161 @@ __global__ void __launch_bounds__(kThreads, 3) expert_lean_kernel(const LeanPara
 
 // ---- host side ---------------------------------------------------------------------------
 struct LeanPlan {
-  int cap_bytes, red_rows, max_cols, cols_q, cols_rem, smem, kb;
+  int grid, nc, cap_bytes, red_rows, max_cols, cols_q, cols_rem, smem, kb;
   bool ok;
 };
 
 // Shapes: L <= 8; d a multiple of 64 up to 2048 (x fragments of a warp fit its registers);
-// d_e a power of two >= 64; at most 16 output columns per CTA. The shared memory of a CTA is
-// sized for the union the caller expects (or the paper's sparsity, see make_plan of the
-// two-kernel form): three CTAs per SM when its share fits a third of an SM, else two, else one;
-// larger unions still run, in stages.
-LeanPlan lean_plan(const blockffn_config& cfg, int L, int grid) {
+// d_e a power of two >= 64.
+//
+// How many CTAs a call gets. Every CTA reads all of x and all of h from L2, whatever its share
+// of the weights: with one CTA per SM that broadcast is half as many bytes again as the weights
+// themselves, and an SM takes bytes in from L2 only about one and a half times as fast as its
+// share of the HBM stream. A call therefore runs on a fraction of the SMs (grid = SMs / split),
+// each CTA with a `split` times larger share (up to two column tiles of out), and `split` times
+// as many calls are in flight to cover the rest of the device.
+//
+// The shared memory of a CTA is sized so that `per_sm` CTAs fit one SM; a share that does not
+// fit goes through in stages.
+// shared: the call may share the device with its neighbours (it depends on none of them)
+LeanPlan lean_plan(const blockffn_config& cfg, int L, int sms, bool shared) {
   LeanPlan pl{};
   pl.ok = false;
   const int d = cfg.d, d_e = cfg.d_e, E = cfg.E;
-  if (L < 1 || L > 8 || grid < 1) return pl;
+  if (L < 1 || L > 8 || sms < 1) return pl;
   if (d % 64 || d > 512 * kMaxKB || d_e % 64 || (d_e & (d_e - 1)) || d_e > 4096 || E > 1024)
     return pl;
-  if (d > 16 * grid) return pl;    // one column tile per CTA
   pl.kb = (d / 64 + kWarps - 1) / kWarps;
-  pl.cols_q = d / grid;
-  pl.cols_rem = d % grid;
-  pl.max_cols = pl.cols_q + (pl.cols_rem ? 1 : 0);
   int u_exp = (cfg.flags >> 17) & 0x7ff;
   if (u_exp == 0) u_exp = (L == 1 ? E + 4 : 3 * E + 5) / (L == 1 ? 8 : 10);
   if (u_exp < 1) u_exp = 1;
   if (u_exp > E) u_exp = E;
-  const int rows_exp = (u_exp * d_e + grid - 1) / grid;
-  const int slot_d = pl.max_cols * 2 * d_e + 64;          // columns split even / odd around 64 bytes
-  const int need = max(rows_exp * 2 * d + 64, u_exp * slot_d);
-  const int base = kOffIds + align128(E * 4);
-  for (int per_sm = 3; per_sm >= 1; --per_sm) {
-    const int budget = (per_sm == 1 ? kSmemMax : (kSmemMax + 1024) / per_sm - 1024) & ~127;
-    // the up partial tile is as wide as a stage can be: the expected share, at most 32 rows
-    int red_rows = rows_exp < 32 ? rows_exp : 32;
-    if (red_rows < 8) red_rows = 8;
-    const int fixed = lean_layout(E, red_rows, 0).total;
-    const int cap = budget - fixed;
-    if (cap < need && per_sm > 1) continue;
-    if (cap < 2 * 2 * d + 128 || cap < 2 * slot_d) return pl;     // not even two rows / two slabs
-    pl.cap_bytes = cap & ~127;
-    // with room to spare let a stage hold up to 32 rows (two mma row tiles)
-    while (red_rows < 32 && (red_rows + 1) * 2 * d + 64 <= pl.cap_bytes &&
-           lean_layout(E, red_rows + 1, pl.cap_bytes).total <= budget)
-      ++red_rows;
+  // measured on B200 (d = 1536 and 2048, unions of 30 %): a third of the SMs per call is best
+  // for calls that do not depend on one another; a call in a dependent chain is alone on the
+  // device and takes all of it
+  int split = shared && !(cfg.flags & BLOCKFFN_CFG_NO_SPLIT) ? 3 : 1;
+  for (;; --split) {                               // at most four column tiles per CTA
+    pl.grid = (sms + split - 1) / split;
+    pl.nc = (d + 16 * pl.grid - 1) / (16 * pl.grid);
+    if (pl.nc <= 4 || split == 1) break;
+  }
+  if (pl.nc > 4) return pl;
+  pl.cols_q = d / pl.grid;
+  pl.cols_rem = d % pl.grid;
+  pl.max_cols = pl.cols_q + (pl.cols_rem ? 1 : 0);
+  const int rows_exp = (u_exp * d_e + pl.grid - 1) / pl.grid;
+  const int slot_d = pl.max_cols * 2 * d_e + 64;   // columns split even / odd around 64 bytes
+  const int need = max(min(rows_exp, 32) * 2 * d + 64, min(u_exp, 16) * slot_d);
+  // the partial tile (and a stage) is as wide as the expected share, between one row tile per
+  // column tile and two row tiles
+  int red_rows = rows_exp < 32 ? rows_exp : 32;
+  if (red_rows < 16 * pl.nc) red_rows = 16 * pl.nc;
+  const int fixed = lean_layout(E, red_rows, 0).total;
+  // A call that owns the device gets the most CTAs per SM (three at most) whose shared memory
+  // still holds the expected share in one stage; calls that share the device always run three
+  // to an SM and stream their larger shares through in stages.
+  for (int n = 3; n >= 1; --n) {
+    const int budget = (n == 1 ? kSmemMax : (kSmemMax + 1024) / n - 1024) & ~127;
+    const int cap = (budget - fixed) & ~127;
+    if (cap < need && n > 1 && split == 1) continue;
+    if (cap < 2 * 4 * 2 * d + 128 || cap < 2 * slot_d) {   // two stages of four rows, two slabs
+      if (n > 1) continue;
+      if (cap < 2 * 2 * d + 128 || cap < 2 * slot_d) return pl;
+    }
+    pl.cap_bytes = cap;
     pl.red_rows = red_rows;
-    pl.cap_bytes = (budget - lean_layout(E, red_rows, 0).total) & ~127;
-    pl.smem = lean_layout(E, red_rows, pl.cap_bytes).total;
-    (void)base;
-    pl.ok = pl.smem <= kSmemMax;
+    pl.smem = lean_layout(E, red_rows, cap).total;
+    pl.ok = true;
     return pl;
   }
   return pl;
 }
 
-template <int KB, int MODE, int EARLY>
+template <int KB, int NC, int MODE, int EARLY>
 cudaError_t lean_attr() {
-  const void* f = reinterpret_cast<const void*>(&expert_lean_kernel<KB, MODE, EARLY>);
+  const void* f = reinterpret_cast<const void*>(&expert_lean_kernel<KB, NC, MODE, EARLY>);
   cudaError_t e = cudaFuncSetAttribute(f, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemMax);
   if (e != cudaSuccess) return e;
   return cudaFuncSetAttribute(f, cudaFuncAttributePreferredSharedMemoryCarveout,
                               cudaSharedmemCarveoutMaxShared);
 }
-template <int KB>
+template <int KB, int NC>
 cudaError_t lean_attrs_kb() {
-  cudaError_t e = lean_attr<KB, 0, 0>();
-  if (e == cudaSuccess) e = lean_attr<KB, 0, 1>();
-  if (e == cudaSuccess) e = lean_attr<KB, 0, 2>();
-  if (e == cudaSuccess) e = lean_attr<KB, 1, 0>();
-  if (e == cudaSuccess) e = lean_attr<KB, 1, 1>();
-  if (e == cudaSuccess) e = lean_attr<KB, 1, 2>();
-  if (e == cudaSuccess) e = lean_attr<KB, 2, 0>();
-  if (e == cudaSuccess) e = lean_attr<KB, 2, 2>();
+  cudaError_t e = lean_attr<KB, NC, 0, 0>();
+  if (e == cudaSuccess) e = lean_attr<KB, NC, 0, 1>();
+  if (e == cudaSuccess) e = lean_attr<KB, NC, 0, 2>();
+  if (e == cudaSuccess) e = lean_attr<KB, NC, 1, 0>();
+  if (e == cudaSuccess) e = lean_attr<KB, NC, 1, 1>();
+  if (e == cudaSuccess) e = lean_attr<KB, NC, 1, 2>();
+  if (e == cudaSuccess) e = lean_attr<KB, NC, 2, 0>();
+  if (e == cudaSuccess) e = lean_attr<KB, NC, 2, 2>();
   return e;
 }
 
-template <int KB, int MODE>
+template <int KB, int NC, int MODE>
 cudaError_t lean_launch_mode(const cudaLaunchConfig_t& lc, const LeanParams& p, int early) {
   if constexpr (MODE == 2) {
-    return early == 2 ? cudaLaunchKernelEx(&lc, expert_lean_kernel<KB, 2, 2>, p)
-                      : cudaLaunchKernelEx(&lc, expert_lean_kernel<KB, 2, 0>, p);
+    return early == 2 ? cudaLaunchKernelEx(&lc, expert_lean_kernel<KB, NC, 2, 2>, p)
+                      : cudaLaunchKernelEx(&lc, expert_lean_kernel<KB, NC, 2, 0>, p);
   } else {
-    return early == 2   ? cudaLaunchKernelEx(&lc, expert_lean_kernel<KB, MODE, 2>, p)
-           : early == 1 ? cudaLaunchKernelEx(&lc, expert_lean_kernel<KB, MODE, 1>, p)
-                        : cudaLaunchKernelEx(&lc, expert_lean_kernel<KB, MODE, 0>, p);
+    return early == 2   ? cudaLaunchKernelEx(&lc, expert_lean_kernel<KB, NC, MODE, 2>, p)
+           : early == 1 ? cudaLaunchKernelEx(&lc, expert_lean_kernel<KB, NC, MODE, 1>, p)
+                        : cudaLaunchKernelEx(&lc, expert_lean_kernel<KB, NC, MODE, 0>, p);
   }
 }
-template <int KB>
+template <int KB, int NC>
 cudaError_t lean_launch_kb(const cudaLaunchConfig_t& lc, const LeanParams& p, int mode, int early) {
-  return mode == 2   ? lean_launch_mode<KB, 2>(lc, p, early)
-         : mode == 1 ? lean_launch_mode<KB, 1>(lc, p, early)
-                     : lean_launch_mode<KB, 0>(lc, p, early);
+  return mode == 2   ? lean_launch_mode<KB, NC, 2>(lc, p, early)
+         : mode == 1 ? lean_launch_mode<KB, NC, 1>(lc, p, early)
+                     : lean_launch_mode<KB, NC, 0>(lc, p, early);
+}
+template <int NC>
+cudaError_t lean_launch_nc(int kb, const cudaLaunchConfig_t& lc, const LeanParams& p, int mode,
+                           int early) {
+  switch (kb) {
+    case 1: return lean_launch_kb<1, NC>(lc, p, mode, early);
+    case 2: return lean_launch_kb<2, NC>(lc, p, mode, early);
+    case 3: return lean_launch_kb<3, NC>(lc, p, mode, early);
+    default: return lean_launch_kb<4, NC>(lc, p, mode, early);
+  }
 }
 
 }  // namespace
 
 bool expert_lean_supported(const blockffn_ctx* c, int L) {
   return c->lean_ring != nullptr && !(c->cfg.flags & BLOCKFFN_CFG_TWO_KERNELS) &&
-         lean_plan(c->cfg, L, c->num_sms).ok;
+         lean_plan(c->cfg, L, c->num_sms, false).ok && lean_plan(c->cfg, L, c->num_sms, true).ok;
 }
 
-// Ring of kHRing intermediates of a chunk of 8 tokens; 0 when the shape never takes this kernel
-// (or the ring would be unreasonably large).
-size_t expert_lean_ws_bytes(const blockffn_config* cfg, int grid) {
-  if (!lean_plan(*cfg, cfg->L_max < 8 ? cfg->L_max : 8, grid).ok) return 0;
+// Two rings (calls that own the device, calls that share it: their grids differ, so each kind
+// counts its own tickets) of kHRing intermediates of a chunk of 8 tokens; 0 when the shape never
+// takes this kernel (or the rings would be unreasonably large).
+size_t expert_lean_ws_bytes(const blockffn_config* cfg, int sms) {
+  const int L = cfg->L_max < 8 ? cfg->L_max : 8;
+  if (!lean_plan(*cfg, L, sms, false).ok || !lean_plan(*cfg, L, sms, true).ok) return 0;
   const size_t slot = ((size_t)cfg->E * 8 * cfg->d_e * sizeof(uint16_t) + 255) & ~(size_t)255;
-  if (kHRing * slot > ((size_t)64 << 20)) return 0;
-  return kHRing * slot;
+  if (2 * kHRing * slot > ((size_t)128 << 20)) return 0;
+  return 2 * kHRing * slot;
 }
 
 cudaError_t expert_lean_setup(blockffn_ctx* c) {
   (void)c;
-  cudaError_t e = lean_attrs_kb<1>();
-  if (e == cudaSuccess) e = lean_attrs_kb<2>();
-  if (e == cudaSuccess) e = lean_attrs_kb<3>();
-  if (e == cudaSuccess) e = lean_attrs_kb<4>();
+  cudaError_t e = lean_attrs_kb<1, 1>();
+  if (e == cudaSuccess) e = lean_attrs_kb<2, 1>();
+  if (e == cudaSuccess) e = lean_attrs_kb<3, 1>();
+  if (e == cudaSuccess) e = lean_attrs_kb<4, 1>();
+  if (e == cudaSuccess) e = lean_attrs_kb<1, 2>();
+  if (e == cudaSuccess) e = lean_attrs_kb<2, 2>();
+  if (e == cudaSuccess) e = lean_attrs_kb<3, 2>();
+  if (e == cudaSuccess) e = lean_attrs_kb<4, 2>();
+  if (e == cudaSuccess) e = lean_attrs_kb<1, 3>();
+  if (e == cudaSuccess) e = lean_attrs_kb<2, 3>();
+  if (e == cudaSuccess) e = lean_attrs_kb<3, 3>();
+  if (e == cudaSuccess) e = lean_attrs_kb<4, 3>();
+  if (e == cudaSuccess) e = lean_attrs_kb<1, 4>();
+  if (e == cudaSuccess) e = lean_attrs_kb<2, 4>();
+  if (e == cudaSuccess) e = lean_attrs_kb<3, 4>();
+  if (e == cudaSuccess) e = lean_attrs_kb<4, 4>();
   return e;
 }
 
@@ -655,7 +757,13 @@ cudaError_t launch_expert_lean(blockffn_ctx* c, const blockffn_weights* w, const
                                const int32_t* n_union, float* out, void* x_next, int call_flags,
                                const RoutingOut* pub, const RouterLogits* logits, bool logits_final,
                                cudaStream_t st) {
-  const LeanPlan pl = lean_plan(c->cfg, L, c->num_sms);
+  const int early = logits ? (logits_final ? 2 : 0)
+                    : (call_flags & BLOCKFFN_CALL_INDEPENDENT_X) ? 2
+                    : (call_flags & BLOCKFFN_CALL_INDEPENDENT)   ? 1
+                                                                 : 0;
+  // x stable: the call consumes nothing of its predecessors and shares the device with them
+  const bool shared = early == 2;
+  const LeanPlan pl = lean_plan(c->cfg, L, c->num_sms, shared);
   if (!pl.ok || !c->lean_ring) return cudaErrorNotSupported;
   LeanParams p{};
   p.x = static_cast<const uint16_t*>(x);
@@ -665,10 +773,10 @@ cudaError_t launch_expert_lean(blockffn_ctx* c, const blockffn_weights* w, const
   if (logits) p.lg = *logits;
   p.ids_in = union_ids;
   p.n_in = n_union;
-  p.h_ring = static_cast<uint16_t*>(c->lean_ring);
   p.h_slot = (((size_t)c->cfg.E * 8 * c->cfg.d_e * sizeof(uint16_t) + 255) & ~(size_t)255) / 2;
-  p.seq = c->lean_seq;
-  p.ready = c->lean_seq + 1;
+  p.h_ring = static_cast<uint16_t*>(c->lean_ring) + (shared ? kHRing * p.h_slot : 0);
+  p.seq = c->lean_seq + (shared ? 32 : 0);
+  p.ready = p.seq + 1;
   p.out = out;
   p.x_next = static_cast<uint16_t*>(x_next);
   p.L = L;
@@ -678,6 +786,11 @@ cudaError_t launch_expert_lean(blockffn_ctx* c, const blockffn_weights* w, const
   p.de_shift = __builtin_ctz(c->cfg.d_e);
   p.cap_bytes = pl.cap_bytes;
   p.red_rows = pl.red_rows;
+  p.cap_rows = (pl.cap_bytes - 128) / (2 * c->cfg.d);
+  if (p.cap_rows > 64) p.cap_rows = 64;
+  p.cap_slabs = pl.cap_bytes / (pl.max_cols * 2 * c->cfg.d_e + 64);
+  p.magic_g = (uint32_t)((0x100000000ull + (unsigned)pl.grid - 1) / (unsigned)pl.grid);
+  p.magic_cpr = (uint32_t)((0x10000u + (unsigned)(c->cfg.d / 8) - 1) / (unsigned)(c->cfg.d / 8));
   p.max_cols = pl.max_cols;
   p.cols_q = pl.cols_q;
   p.cols_rem = pl.cols_rem;
@@ -694,28 +807,23 @@ cudaError_t launch_expert_lean(blockffn_ctx* c, const blockffn_weights* w, const
     p.pub_tok = pub->tok_mask;
   }
   const bool chained = !(c->cfg.flags & BLOCKFFN_CFG_NO_CHAINING);
-  const int early = logits ? (logits_final ? 2 : 0)
-                    : (call_flags & BLOCKFFN_CALL_INDEPENDENT_X) ? 2
-                    : (call_flags & BLOCKFFN_CALL_INDEPENDENT)   ? 1
-                                                                 : 0;
   const int mode = logits ? 2 : union_ids ? 1 : 0;
   cudaLaunchAttribute attr[1];
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cudaLaunchConfig_t lc{};
-  lc.gridDim = dim3(c->num_sms);
+  lc.gridDim = dim3(pl.grid);
   lc.blockDim = dim3(kThreads);
   lc.stream = st;
   lc.attrs = attr;
   lc.numAttrs = chained ? 1 : 0;
-  lc.dynamicSmemBytes = pl.smem;
-  cudaError_t e;
-  switch (pl.kb) {
-    case 1: e = lean_launch_kb<1>(lc, p, mode, early); break;
-    case 2: e = lean_launch_kb<2>(lc, p, mode, early); break;
-    case 3: e = lean_launch_kb<3>(lc, p, mode, early); break;
-    default: e = lean_launch_kb<4>(lc, p, mode, early); break;
-  }
+  // never less than a quarter of an SM's shared memory: at most three CTAs then fit one SM,
+  // whatever the shape, which is what the size of the ring rests on
+  lc.dynamicSmemBytes = pl.smem > kMinSmem ? pl.smem : kMinSmem;
+  const cudaError_t e = pl.nc == 4   ? lean_launch_nc<4>(pl.kb, lc, p, mode, early)
+                        : pl.nc == 3 ? lean_launch_nc<3>(pl.kb, lc, p, mode, early)
+                        : pl.nc == 2 ? lean_launch_nc<2>(pl.kb, lc, p, mode, early)
+                                     : lean_launch_nc<1>(pl.kb, lc, p, mode, early);
   if (e == cudaSuccess) c->launches += 1;
   return e;
 }
