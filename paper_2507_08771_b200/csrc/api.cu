@@ -21,13 +21,18 @@ bool use_mma(const blockffn_ctx* c, int L) {
   return c->cfg.variant != BLOCKFFN_VARIANT_SIMT && expert_mma_supported(c, L);
 }
 
-// Tensor-core expert stage: one kernel per call where the shape allows it, else the pair.
+// Tensor-core expert stage: one kernel per call or the up/down pair.
 cudaError_t launch_tensor_core(blockffn_ctx* c, const blockffn_weights* w, const void* x,
                                const float* scores, int L, const int32_t* union_ids,
                                const int32_t* n_union, float* out, void* x_next, int call_flags,
                                const RoutingOut* pub, const RouterLogits* logits, bool logits_final,
                                cudaStream_t st) {
-  if (expert_lean_supported(c, L))
+  // The one-kernel form pays off where calls overlap freely, i.e. where x is stable (for a
+  // router-on call: the router has finished before the expert stage starts). A call in a
+  // dependent chain (x comes from the call before) runs as the pair, whose two hand-overs are
+  // shorter than a grid-wide exchange inside one kernel.
+  const bool x_stable = logits ? logits_final : (call_flags & BLOCKFFN_CALL_INDEPENDENT_X) != 0;
+  if (x_stable && expert_lean_supported(c, L))
     return launch_expert_lean(c, w, x, scores, L, union_ids, n_union, out, x_next, call_flags, pub,
                               logits, logits_final, st);
   return launch_expert_mma(c, w, x, scores, L, union_ids, n_union, out, x_next, call_flags, pub,

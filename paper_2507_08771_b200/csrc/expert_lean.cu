@@ -151,10 +151,10 @@ __device__ __forceinline__ void mma64(float (&c0)[4], float (&c1)[4], const uint
   mma_bf16(c1, ahi.z, bhi.z, ahi.w, bhi.w, x.hi.z, x.hi.w);
 }
 
-// KB: 64-wide k blocks of x per warp (ceil(d / 512)); MODE as derive_union; EARLY: 0 wait first,
-// 1 routing inputs and weights before the wait, 2 x as well (the wait then comes before out).
-// NC: 16-column tiles of out per CTA (1 .. 4).
-template <int KB, int NC, int MODE, int EARLY>
+// KB: 64-wide k blocks of x per warp (ceil(d / 512)); NC: 16-column tiles of out per CTA
+// (1 .. 4); MODE as derive_union. Everything the call reads is stable (x included): nothing
+// waits for the kernel before it until out is touched.
+template <int KB, int NC, int MODE>
 __global__ void __launch_bounds__(kThreads, 3) expert_lean_kernel(const LeanParams p) {
   extern __shared__ __align__(128) unsigned char smem[];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -169,12 +169,6 @@ __global__ void __launch_bounds__(kThreads, 3) expert_lean_kernel(const LeanPara
   const int G = gridDim.x, bx = blockIdx.x;
 
   if (tid < 8) ctl[tid] = 0;
-  if constexpr (EARLY == 0) {
-    if constexpr (MODE == 2) {
-      if (tid * 32 < p.E) asm volatile("prefetch.global.L2 [%0];" ::"l"(p.lg.gain + tid * 32));
-    }
-    pdl_wait();
-  }
   unsigned long long ticket = 0;
   if (tid == 0) ticket = atomicAdd(p.seq, 1ull);
   __syncthreads();
@@ -294,16 +288,14 @@ __global__ void __launch_bounds__(kThreads, 3) expert_lean_kernel(const LeanPara
       }
     }
   };
-  // x goes first when it is stable: its short round trip then runs under the long issue of
-  // the weights instead of behind it
-  if constexpr (EARLY == 2) load_x();
+  // x goes first: its short round trip then runs under the long issue of the weights instead
+  // of behind it
+  load_x();
   if (ngroups > 0) issue_u(0);
   cp_async_commit();
   if (ngroups > 1) issue_u(1);
   cp_async_commit();
   if (ngroups > 0) prepare(0);
-  if constexpr (EARLY == 1) pdl_wait();     // x may come from the kernel just before
-  if constexpr (EARLY != 2) load_x();
   const int slot = ctl[6];       // (written before the barriers inside derive_union)
   uint16_t* hbuf = p.h_ring + (size_t)slot * p.h_slot;
 
@@ -412,16 +404,7 @@ __global__ void __launch_bounds__(kThreads, 3) expert_lean_kernel(const LeanPara
   cp_async_commit();
   if (nrounds > 1) issue_d(1);
   cp_async_commit();
-  bool waited = EARLY < 2;
-  // the residual this CTA's outputs are added to (thread tid: token tid / 32, columns tid % 32
-  // and, with more than two column tiles, 32 further): asked for as early as out may be read
-  const int ot = tid >> 5, om = tid & 31;
-  float resid[(NC + 1) / 2] = {};
-  if (waited && p.accumulate && ot < L) {
-#pragma unroll
-    for (int k = 0; k < (NC + 1) / 2; ++k)
-      if (om + 32 * k < ncols) resid[k] = __ldcg(p.out + ot * d + c0 + om + 32 * k);
-  }
+  const int ot = tid >> 5, om = tid & 31;   // this thread's outputs: token ot, columns om (+ 32)
   // hand-over: all CTAs of this call have stored their part of h
   if (tid == kSyncThread) {
     const unsigned long long target = *reinterpret_cast<const unsigned long long*>(ctl + 138);
@@ -510,7 +493,7 @@ __global__ void __launch_bounds__(kThreads, 3) expert_lean_kernel(const LeanPara
     cp_async_commit();
   }
   cp_async_wait_all();
-  if (!waited) pdl_wait();         // out (and x_next) may still be in use by the call before
+  pdl_wait();                      // out (and x_next) may still be in use by the call before
   if (!dead) {
     if (nu > 0) {
       // partial tiles -> red[t][m][warp] (m < 16 NC), then one thread per output element
@@ -532,7 +515,7 @@ __global__ void __launch_bounds__(kThreads, 3) expert_lean_kernel(const LeanPara
             const float4 lo = part[0], hi = part[1];
             float v = ((lo.x + lo.y) + (lo.z + lo.w)) + ((hi.x + hi.y) + (hi.z + hi.w));
             const int o = ot * d + c0 + m;
-            if (p.accumulate) v += EARLY < 2 ? resid[k] : __ldcg(p.out + o);
+            if (p.accumulate) v += __ldcg(p.out + o);
             p.out[o] = v;
             if (p.x_next) p.x_next[o] = (uint16_t)f32_to_bf16_bits(v);
           }
@@ -664,9 +647,9 @@ LeanPlan lean_plan(const blockffn_config& cfg, int L, int sms, bool shared) {
   return pl;
 }
 
-template <int KB, int NC, int MODE, int EARLY>
+template <int KB, int NC, int MODE>
 cudaError_t lean_attr() {
-  const void* f = reinterpret_cast<const void*>(&expert_lean_kernel<KB, NC, MODE, EARLY>);
+  const void* f = reinterpret_cast<const void*>(&expert_lean_kernel<KB, NC, MODE>);
   cudaError_t e = cudaFuncSetAttribute(f, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemMax);
   if (e != cudaSuccess) return e;
   return cudaFuncSetAttribute(f, cudaFuncAttributePreferredSharedMemoryCarveout,
@@ -674,42 +657,25 @@ cudaError_t lean_attr() {
 }
 template <int KB, int NC>
 cudaError_t lean_attrs_kb() {
-  cudaError_t e = lean_attr<KB, NC, 0, 0>();
-  if (e == cudaSuccess) e = lean_attr<KB, NC, 0, 1>();
-  if (e == cudaSuccess) e = lean_attr<KB, NC, 0, 2>();
-  if (e == cudaSuccess) e = lean_attr<KB, NC, 1, 0>();
-  if (e == cudaSuccess) e = lean_attr<KB, NC, 1, 1>();
-  if (e == cudaSuccess) e = lean_attr<KB, NC, 1, 2>();
-  if (e == cudaSuccess) e = lean_attr<KB, NC, 2, 0>();
-  if (e == cudaSuccess) e = lean_attr<KB, NC, 2, 2>();
+  cudaError_t e = lean_attr<KB, NC, 0>();
+  if (e == cudaSuccess) e = lean_attr<KB, NC, 1>();
+  if (e == cudaSuccess) e = lean_attr<KB, NC, 2>();
   return e;
 }
 
-template <int KB, int NC, int MODE>
-cudaError_t lean_launch_mode(const cudaLaunchConfig_t& lc, const LeanParams& p, int early) {
-  if constexpr (MODE == 2) {
-    return early == 2 ? cudaLaunchKernelEx(&lc, expert_lean_kernel<KB, NC, 2, 2>, p)
-                      : cudaLaunchKernelEx(&lc, expert_lean_kernel<KB, NC, 2, 0>, p);
-  } else {
-    return early == 2   ? cudaLaunchKernelEx(&lc, expert_lean_kernel<KB, NC, MODE, 2>, p)
-           : early == 1 ? cudaLaunchKernelEx(&lc, expert_lean_kernel<KB, NC, MODE, 1>, p)
-                        : cudaLaunchKernelEx(&lc, expert_lean_kernel<KB, NC, MODE, 0>, p);
-  }
-}
 template <int KB, int NC>
-cudaError_t lean_launch_kb(const cudaLaunchConfig_t& lc, const LeanParams& p, int mode, int early) {
-  return mode == 2   ? lean_launch_mode<KB, NC, 2>(lc, p, early)
-         : mode == 1 ? lean_launch_mode<KB, NC, 1>(lc, p, early)
-                     : lean_launch_mode<KB, NC, 0>(lc, p, early);
+cudaError_t lean_launch_kb(const cudaLaunchConfig_t& lc, const LeanParams& p, int mode) {
+  return mode == 2   ? cudaLaunchKernelEx(&lc, expert_lean_kernel<KB, NC, 2>, p)
+         : mode == 1 ? cudaLaunchKernelEx(&lc, expert_lean_kernel<KB, NC, 1>, p)
+                     : cudaLaunchKernelEx(&lc, expert_lean_kernel<KB, NC, 0>, p);
 }
 template <int NC>
-cudaError_t lean_launch_nc(int kb, const cudaLaunchConfig_t& lc, const LeanParams& p, int mode,
-                           int early) {
+cudaError_t lean_launch_nc(int kb, const cudaLaunchConfig_t& lc, const LeanParams& p, int mode) {
   switch (kb) {
-    case 1: return lean_launch_kb<1, NC>(lc, p, mode, early);
-    case 2: return lean_launch_kb<2, NC>(lc, p, mode, early);
-    case 3: return lean_launch_kb<3, NC>(lc, p, mode, early);
-    default: return lean_launch_kb<4, NC>(lc, p, mode, early);
+    case 1: return lean_launch_kb<1, NC>(lc, p, mode);
+    case 2: return lean_launch_kb<2, NC>(lc, p, mode);
+    case 3: return lean_launch_kb<3, NC>(lc, p, mode);
+    default: return lean_launch_kb<4, NC>(lc, p, mode);
   }
 }
 
@@ -757,12 +723,12 @@ cudaError_t launch_expert_lean(blockffn_ctx* c, const blockffn_weights* w, const
                                const int32_t* n_union, float* out, void* x_next, int call_flags,
                                const RoutingOut* pub, const RouterLogits* logits, bool logits_final,
                                cudaStream_t st) {
-  const int early = logits ? (logits_final ? 2 : 0)
-                    : (call_flags & BLOCKFFN_CALL_INDEPENDENT_X) ? 2
-                    : (call_flags & BLOCKFFN_CALL_INDEPENDENT)   ? 1
-                                                                 : 0;
-  // x stable: the call consumes nothing of its predecessors and shares the device with them
-  const bool shared = early == 2;
+  // Only for calls whose x is stable (for a router-on call: whose router has finished).
+  if (logits ? !logits_final : !(call_flags & BLOCKFFN_CALL_INDEPENDENT_X)) return cudaErrorNotSupported;
+  // No router in front: the call consumes nothing of its predecessors and shares the device
+  // with them (a router-on call is ordered behind its router by events, which keeps too few of
+  // them in flight for a third of the device each).
+  const bool shared = !logits;
   const LeanPlan pl = lean_plan(c->cfg, L, c->num_sms, shared);
   if (!pl.ok || !c->lean_ring) return cudaErrorNotSupported;
   LeanParams p{};
@@ -820,10 +786,10 @@ cudaError_t launch_expert_lean(blockffn_ctx* c, const blockffn_weights* w, const
   // never less than a quarter of an SM's shared memory: at most three CTAs then fit one SM,
   // whatever the shape, which is what the size of the ring rests on
   lc.dynamicSmemBytes = pl.smem > kMinSmem ? pl.smem : kMinSmem;
-  const cudaError_t e = pl.nc == 4   ? lean_launch_nc<4>(pl.kb, lc, p, mode, early)
-                        : pl.nc == 3 ? lean_launch_nc<3>(pl.kb, lc, p, mode, early)
-                        : pl.nc == 2 ? lean_launch_nc<2>(pl.kb, lc, p, mode, early)
-                                     : lean_launch_nc<1>(pl.kb, lc, p, mode, early);
+  const cudaError_t e = pl.nc == 4   ? lean_launch_nc<4>(pl.kb, lc, p, mode)
+                        : pl.nc == 3 ? lean_launch_nc<3>(pl.kb, lc, p, mode)
+                        : pl.nc == 2 ? lean_launch_nc<2>(pl.kb, lc, p, mode)
+                                     : lean_launch_nc<1>(pl.kb, lc, p, mode);
   if (e == cudaSuccess) c->launches += 1;
   return e;
 }
