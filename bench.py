@@ -62,6 +62,20 @@ def measured_peak():
         return FALLBACK_HBM_GBS, "fallback"
 
 
+def measured_traffic(config, L, kernel):
+    """dram__bytes_read + dram__bytes_write per call from the ncu capture summarised in
+    profiles/dram_traffic.md (rows `| config | L | kernel | bytes |`), or None if that
+    configuration was not captured."""
+    try:
+        for line in open(os.path.join(ROOT, "profiles", "dram_traffic.md")):
+            f = [v.strip() for v in line.strip().strip("|").split("|")]
+            if len(f) >= 4 and f[0] == str(config) and f[1] == str(L) and f[2] == kernel:
+                return int(f[3])
+    except (OSError, ValueError):
+        pass
+    return None
+
+
 def copies_needed(active_bytes):
     """Enough weight copies that twice the L2 is streamed between two uses of one copy."""
     return max(8, int(math.ceil(2 * L2_BYTES / active_bytes)) + 1)
@@ -136,11 +150,12 @@ class ClockSampler:
 class Workload:
     """Device-resident synthetic inputs for one benchmark configuration."""
 
-    def __init__(self, cfg_index, L, chunks, variant, device, flags=0, u=None):
+    def __init__(self, cfg_index, L, chunks, variant, device, flags=0, u=None, stack_layers=0):
         import torch
         from paper_2507_08771_b200 import binding as B
         self.torch, self.B = torch, B
         self.idx, self.chunks, self.device = cfg_index, chunks, device
+        self.stack = cfg_index == 4 or stack_layers > 0
         self.sh = sh = I.SHAPES[cfg_index]
         self.L = L or sh.L
         seed = I.config_seed(cfg_index)
@@ -148,12 +163,16 @@ class Workload:
         self.active_bytes = sh.active_bytes(self.u)
         # successive chunks of configs 1-3 are independent inputs; the stack (4) feeds each layer
         # the previous layer's output, so only its routing inputs and weights are stable
-        self.call_flags = B.CALL_INDEPENDENT if cfg_index == 4 else B.CALL_INDEPENDENT_X
+        self.call_flags = B.CALL_INDEPENDENT if self.stack else B.CALL_INDEPENDENT_X
         self.layer = B.Layer(sh.d, sh.E, sh.d_e, L_max=max(self.L, 8), variant=variant, device=device,
                              flags=flags)
         if cfg_index == 4:
             self.n_copies = I.STACK_LAYERS          # 24 distinct layers, 1.6 GB >> L2
             host = [I.make_experts(sh.d, sh.E, sh.d_e, seed, layer=l) for l in range(self.n_copies)]
+        elif stack_layers:
+            self.n_copies = stack_layers             # same values, distinct device addresses
+            one = I.make_experts(sh.d, sh.E, sh.d_e, seed)
+            host = [one] * self.n_copies
         else:
             self.n_copies = copies_needed(self.active_bytes)
             one = I.make_experts(sh.d, sh.E, sh.d_e, seed)
@@ -165,8 +184,8 @@ class Workload:
         self.host_weights = host
         # per-chunk inputs, on the host (pinned) and on the device
         n = chunks
-        if cfg_index == 4:
-            # chunk c runs through all 24 layers; scores differ per (layer, chunk)
+        if self.stack:
+            # chunk c runs through all layers; scores differ per (layer, chunk)
             self.calls_per_chunk = self.n_copies
             sc = np.stack([np.stack([I.make_scores(sh.E, self.L, self.u, seed, layer=l, chunk=c)
                                      for l in range(self.n_copies)]) for c in range(n)])
@@ -192,7 +211,7 @@ class Workload:
         """Chunks [lo, hi) of the step."""
         B, lay = self.B, self.layer
         hi = self.chunks if hi is None else hi
-        if self.idx == 4:
+        if self.stack:
             for c in range(lo, hi):
                 # residual stream: out[c] starts as h0 = f32(x[c]); x ping-pongs in bf16
                 self.out[c].copy_(self.x[c])
@@ -220,10 +239,10 @@ class Workload:
         B, lay = self.B, self.layer
         for c in range(self.chunks):
             for l in range(self.calls_per_chunk):
-                k = l if self.idx == 4 else c % self.n_copies
+                k = l if self.stack else c % self.n_copies
                 B.blockffn_expert_ffn(lay.h, self.dws[k].struct, self.x[c], self.scores[c, l], self.L,
                                       self.ids[c, l], self.nu[c, l:l + 1], self.out[c], None,
-                                      B.CALL_INDEPENDENT if self.idx == 4 else self.call_flags, stream)
+                                      B.CALL_INDEPENDENT if self.stack else self.call_flags, stream)
 
 
 def max_over_ranks(values, world, device=None):
@@ -307,7 +326,10 @@ def capture(torch, stream, fn):
     return g
 
 
-def time_replays(torch, stream, graph, steps, warmup, pre=None, post=None):
+def time_replays(torch, stream, graph, steps, warmup, pre=None, post=None, per_replay=None):
+    """ms per step over `steps` back-to-back replays (events around the whole run, on the stream
+    the graph is launched on). per_replay (a list) also receives each replay's own time: an
+    event between consecutive replays costs nothing measurable next to a step of milliseconds."""
     with torch.cuda.stream(stream):
         for _ in range(warmup):
             if pre:
@@ -316,23 +338,25 @@ def time_replays(torch, stream, graph, steps, warmup, pre=None, post=None):
             if post:
                 post()
         stream.synchronize()
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        e0.record(stream)
-        for _ in range(steps):
+        marks = [torch.cuda.Event(enable_timing=True) for _ in range(steps + 1)]
+        marks[0].record(stream)
+        for k in range(steps):
             if pre:
                 pre()
             graph.replay()
             if post:
                 post()
-        e1.record(stream)
+            marks[k + 1].record(stream)
         stream.synchronize()
-    return e0.elapsed_time(e1) / steps      # ms per step
+    if per_replay is not None:
+        per_replay.extend(marks[k].elapsed_time(marks[k + 1]) for k in range(steps))
+    return marks[0].elapsed_time(marks[steps]) / steps      # ms per step
 
 
 # ----------------------------------------------------------------------------
 # CPU oracle legs
 # ----------------------------------------------------------------------------
-def oracle_sample(cfg_index, L, budget_s, max_chunks):
+def oracle_sample(cfg_index, L, budget_s, max_chunks, union_only=True):
     """Times the CPU oracle (as it stands, one thread) on successive chunks of the
     workload until the time budget is used. Returns (GB/s of active weights, us/chunk, n)."""
     import oracle
@@ -346,11 +370,42 @@ def oracle_sample(cfg_index, L, budget_s, max_chunks):
         x = I.make_x(sh.d, L, seed, chunk=n)
         s = I.make_scores(sh.E, L, sh.u, seed, chunk=n)
         t0 = time.perf_counter()
-        oracle.layer_forward_scores(x, s, U, D, union_only=True)
+        oracle.layer_forward_scores(x, s, U, D, union_only=union_only)
         t_total += time.perf_counter() - t0
         n += 1
     per = t_total / n
     return sh.active_bytes() / per / 1e9, per * 1e6, n
+
+
+def oracle_all_cores(cfg_index, L, chunks_per_thread):
+    """The same oracle, union-restricted, one chunk per call, on every core this process may use
+    (one host thread per core, each working through its own chunks; the C routine runs outside
+    the interpreter lock). Returns (GB/s of active weights, us per chunk of wall time, threads)."""
+    import concurrent.futures
+    import oracle
+    sh = I.SHAPES[cfg_index]
+    L = L or sh.L
+    seed = I.config_seed(cfg_index)
+    U, D = I.make_experts(sh.d, sh.E, sh.d_e, seed)
+    oracle.build()
+    try:
+        threads = len(os.sched_getaffinity(0))
+    except AttributeError:
+        threads = os.cpu_count() or 1
+    n = threads * chunks_per_thread
+    xs = [I.make_x(sh.d, L, seed, chunk=c) for c in range(n)]
+    ss = [I.make_scores(sh.E, L, sh.u, seed, chunk=c) for c in range(n)]
+
+    def work(k):
+        for c in range(k, n, threads):
+            oracle.layer_forward_scores(xs[c], ss[c], U, D, union_only=True)
+
+    with concurrent.futures.ThreadPoolExecutor(threads) as pool:
+        t0 = time.perf_counter()
+        list(pool.map(work, range(threads)))
+        wall = time.perf_counter() - t0
+    per = wall / n
+    return sh.active_bytes() / per / 1e9, per * 1e6, threads, n
 
 
 def run_reference(args):
@@ -442,33 +497,59 @@ def run_ours(args):
         sampler.start()
         time.sleep(0.3)          # nvidia-smi needs a moment before its first sample
         sampler.mark()
-    ms_step = time_replays(torch, stream, g_step, args.steps, args.warmup)
+    per_step = []
+    ms_step = time_replays(torch, stream, g_step, args.steps, args.warmup, per_replay=per_step)
     barrier()
 
     # end to end: host buffers in, host buffers out, copies inside the timed region
     barrier()
     ms_e2e = time_end_to_end(torch, wl, device, max(3, args.steps // 2), 3)
-    # one call on its own: enqueued on an idle device, events right around it (launch latency,
-    # cold routing inputs and weights, no overlap with a neighbour)
-    iso = []
+    # One call on its own: enqueued on an idle device, events right around it (launch latency,
+    # cold routing inputs and weights, no overlap with a neighbour). The same call is also timed
+    # on the host alone (time spent in the Python binding and the library's launch code, no
+    # synchronisation inside), which is what the device sits idle for between the two events when
+    # nothing is queued ahead of it.
+    iso, host_us = [], []
     with torch.cuda.stream(stream):
         for c in range(min(32, wl.chunks)):
             stream.synchronize()
             a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
             a.record(stream)
+            t0 = time.perf_counter()
             wl.enqueue_step(stream, c, c + 1)
+            host_us.append((time.perf_counter() - t0) * 1e6)
             b.record(stream)
             stream.synchronize()
             iso.append(a.elapsed_time(b) * 1e3)
     isolated_us = float(np.median(iso[4:])) if len(iso) > 4 else float(np.median(iso))
+    host_call_us = float(np.median(host_us[4:])) if len(host_us) > 4 else float(np.median(host_us))
+    # the same single call as a one-node graph (no Python, no launch code between the events)
+    g_one = capture(torch, stream, lambda st: wl.enqueue_step(st, 0, 1))
+    one = []
+    with torch.cuda.stream(stream):
+        for _ in range(12):
+            stream.synchronize()
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream)
+            g_one.replay()
+            b.record(stream)
+            stream.synchronize()
+            one.append(a.elapsed_time(b) * 1e3)
+    isolated_graph_us = float(np.median(one[2:]))
     barrier()
-    ms_expert = time_replays(torch, stream, g_expert, args.steps, args.warmup)
+    per_expert = []
+    ms_expert = time_replays(torch, stream, g_expert, args.steps, args.warmup, per_replay=per_expert)
     barrier()
+    # stage level: the union entry point alone (one launch per chunk), from its own graph
+    g_union = capture(torch, stream, wl.enqueue_unions)
+    per_union = []
+    time_replays(torch, stream, g_union, max(3, args.steps // 2), 2, per_replay=per_union)
     clocks = sampler.stop() if rank == 0 else {}
     status = lay.last_status()
     assert status == 0, f"device status word {status}"
-    lay_is_mma = args.variant != 1 and expert_launches // max(wl.calls_per_step, 1) == 2 and sh.d % 64 == 0
+    launches_per_call = expert_launches // max(wl.calls_per_step, 1)
     assert torch.isfinite(wl.out).all()
+    ms_step_median, ms_expert_median = float(np.median(per_step)), float(np.median(per_expert))
 
     ms_step, ms_e2e, ms_expert = max_over_ranks([ms_step, ms_e2e, ms_expert], world, device)
 
@@ -494,7 +575,16 @@ def run_ours(args):
         "data": "synthetic",
         "latency_us_per_chunk": ms_step * 1e3 / wl.chunks,
         "latency_us_per_layer_call": ms_step * 1e3 / calls,
+        "latency_us_per_layer_call_median_replay": ms_step_median * 1e3 / calls,
         "latency_us_isolated_call": isolated_us,
+        "latency_isolated_call": {
+            "us_events_around_python_call": isolated_us, "us_host_time_in_binding_and_launch": host_call_us,
+            "us_events_around_one_node_graph": isolated_graph_us,
+            "note": "on an idle device the events bracket the host's own launch work; the graph leg "
+                    "has no host work between the events: launch latency plus one cold call"},
+        "stage_us_per_call": {"chunk_union_entry_point": float(np.median(per_union)) * 1e3 / calls,
+                              "expert_ffn_entry_point": ms_expert_median * 1e3 / calls,
+                              "layer_forward_scores": ms_step_median * 1e3 / calls},
         "pct_of_nominal_8TBs": 100.0 * value / world / NOMINAL_HBM_GBS,
         "config": {
             "workload": f"config {args.config}: {sh.name} (scores-in: chunk union + expert FFN)",
@@ -512,21 +602,37 @@ def run_ours(args):
         "gpu_launches": launches_per_step * args.steps,
         "gpu_launches_per_step": launches_per_step,
         "roofline": {
-            "bound": "hbm", "kernel": "expert_up_mma + expert_down_mma (the chained pair of one call; 51 % / 48 % of the ncu launch list)",
+            "bound": "hbm",
+            "kernel": ("expert_lean_kernel (one launch per call: up projection, hand-over, down projection)"
+                       if launches_per_call == 1 else
+                       "expert_up_mma + expert_down_mma (the chained pair of one call)"
+                       if launches_per_call == 2 and args.variant != 1 else "expert_up_simt + expert_down_simt"),
             "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-            "peak_kind": f"of {peak_kind}", "us_per_launch": us_expert,
-            "algorithmic_bytes_per_launch": alg_bytes, "launches_per_call": expert_launches // calls,
-            # dram__bytes_read + write of one up + one down launch (ncu, config 1, see profiles/);
-            # other configurations: not captured
-            "traffic": 11130112 if (args.config == 1 and wl.L == 8 and lay_is_mma) else None,
+            "peak_kind": f"of {peak_kind}", "us_per_launch": us_expert / max(launches_per_call, 1),
+            "us_per_call": us_expert, "us_per_call_median_replay": ms_expert_median * 1e3 / calls,
+            "algorithmic_bytes_per_launch": alg_bytes, "launches_per_call": launches_per_call,
+            # dram__bytes_read + write of one call's launches (ncu, see profiles/dram_traffic.md)
+            "traffic": measured_traffic(args.config, wl.L, "lean" if launches_per_call == 1 else "pair"),
         },
     }
     if not args.no_cpu_baseline and world == 1:
-        gbs, us, n = oracle_sample(args.config, wl.L, budget_s=12.0, max_chunks=64)
+        gbs, us, n = oracle_sample(args.config, wl.L, budget_s=8.0, max_chunks=64)
+        gbs_all, us_all, n_all = oracle_sample(args.config, wl.L, budget_s=4.0, max_chunks=8, union_only=False)
+        gbs_mt, us_mt, threads, n_mt = oracle_all_cores(args.config, wl.L, chunks_per_thread=12)
         line["cpu_baseline"] = {
             "value": gbs, "unit": "GB/s", "cores": 1, "kind": "oracle", "us_per_chunk": us,
             "sample": f"{n} chunks of the same workload (one layer call each), union-restricted "
-                      f"sum, float64, single thread"}
+                      f"sum, float64, single thread",
+            "legs": {
+                "single_thread_all_experts": {
+                    "value": gbs_all, "unit": "GB/s", "us_per_chunk": us_all, "cores": 1,
+                    "sample": f"{n_all} chunks, the definition's sum over all {sh.E} experts"},
+                "single_thread_union_only": {"value": gbs, "unit": "GB/s", "us_per_chunk": us,
+                                             "cores": 1, "sample": f"{n} chunks"},
+                "all_cores_union_only": {
+                    "value": gbs_mt, "unit": "GB/s", "us_per_chunk": us_mt, "cores": threads,
+                    "sample": f"{n_mt} chunks over {threads} host threads (the affinity mask of "
+                              f"this process), one chunk per oracle call"}}}
     if not args.no_extras and world == 1:
         del wl, g_step, g_expert
         torch.cuda.empty_cache()
@@ -567,6 +673,14 @@ class RouterWorkload:
         for c in range(self.chunks):
             B.blockffn_layer_forward(lay.h, self.dws[c % len(self.dws)].struct, self.x[c], self.sh.L,
                                      self.out[c], None, lay.stats, self.call_flags, stream)
+
+    def enqueue_router_only(self, stream):
+        """The router entry point alone (Eq. 3 + per-token masks), one launch per chunk."""
+        B, lay = self.B, self.layer
+        if not hasattr(self, "scores_out"):
+            self.scores_out = self.torch.zeros(self.chunks, self.sh.L, self.sh.E, device=self.out.device)
+        for c in range(self.chunks):
+            B.blockffn_router(lay.h, self.dws[0].struct, self.x[c], self.sh.L, self.scores_out[c], None, stream)
 
     def sparsity(self):
         hs = self.layer.stats_host()
@@ -649,8 +763,11 @@ def extras(args, torch, device, peak):
     rows = []
     for L in I.L_SWEEP:
         row = {"L": L}
-        for name, variant in (("tensor_core", 0), ("cuda_core", 1)):
-            wl = Workload(2, L, chunks, variant, device, args.flags)
+        for name, variant, form in (("tensor_core", 0, 0), ("tensor_core_pair", 0, B.CFG_TWO_KERNELS),
+                                    ("cuda_core", 1, 0)):
+            if name == "tensor_core_pair" and L > 8:
+                continue                    # chunks longer than 8 tokens already run as the pair
+            wl = Workload(2, L, chunks, variant, device, args.flags | form)
             us = timed(wl) * 1e3 / wl.calls_per_step
             hs = wl.layer.stats_host()
             row[name] = {"us_per_call": us, "GBps": wl.active_bytes / us / 1e3,
@@ -684,7 +801,13 @@ def extras(args, torch, device, peak):
         mean_u = ufrac * sh.E
         full[name] = {"rho": r, "us_per_call": us, "tls": tls, "mean_union": mean_u,
                       "GBps": mean_u * sh.expert_bytes / us / 1e3,
-                      "launches_per_call": 3}
+                      "launches_per_call": 2}
+        if r is None:                   # stage level: the router entry point from its own graph
+            st2 = torch.cuda.Stream(device)
+            g2 = capture(torch, st2, wl.enqueue_router_only)
+            per = []
+            time_replays(torch, st2, g2, max(3, args.steps // 2), 2, per_replay=per)
+            full["router_entry_point_us_per_call"] = float(np.median(per)) * 1e3 / chunks
         del wl
         torch.cuda.empty_cache()
     sweep_rows, dense_us = [], None
@@ -723,6 +846,16 @@ def extras(args, torch, device, peak):
         torch.cuda.empty_cache()
     rows["tree_time_vs_dense"] = rows["tree_32_tokens"]["us_per_call"] / rows["dense_32_tokens"]["us_per_call"]
     rows["one_token_time_vs_dense"] = rows["one_token"]["us_per_call"] / rows["dense_one_token"]["us_per_call"]
+    # the whole FFN stack of that model: 36 layers, residual between layers, scores-in, one 32-token
+    # tree per pass (4.8 GB of expert weights at distinct addresses; the layers share their values)
+    for name, L, u in (("stack_36_layers_tree_32_tokens", 32, sh5.u), ("stack_36_layers_one_token", 1, u1)):
+        wl = Workload(5, L, 8, 0, device, args.flags | B.cfg_expected_union(u), u=u, stack_layers=36)
+        ms = timed(wl)
+        us_pass = ms * 1e3 / wl.chunks
+        rows[name] = {"L": L, "u": u, "layers": 36, "us_per_pass": us_pass, "us_per_layer": us_pass / 36,
+                      "GBps": 36 * wl.active_bytes / us_pass / 1e3}
+        del wl
+        torch.cuda.empty_cache()
     out["paper_2p8b_shape"] = rows
 
     # config 4: 24-layer stack, residual between layers
