@@ -32,7 +32,7 @@ cudaError_t launch_tensor_core(blockffn_ctx* c, const blockffn_weights* w, const
   // dependent chain (x comes from the call before) runs as the pair, whose two hand-overs are
   // shorter than a grid-wide exchange inside one kernel.
   const bool x_stable = logits ? logits_final : (call_flags & BLOCKFFN_CALL_INDEPENDENT_X) != 0;
-  if (x_stable && expert_lean_supported(c, L))
+  if (x_stable && expert_lean_supported(c, L, logits != nullptr))
     return launch_expert_lean(c, w, x, scores, L, union_ids, n_union, out, x_next, call_flags, pub,
                               logits, logits_final, st);
   return launch_expert_mma(c, w, x, scores, L, union_ids, n_union, out, x_next, call_flags, pub,

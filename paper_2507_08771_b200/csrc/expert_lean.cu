@@ -575,33 +575,36 @@ __global__ void __launch_bounds__(kThreads, 3) expert_lean_kernel(const LeanPara
   }
 }
 
+#include "expert_wide.cuh"   // expert_wide_kernel: the same for chunks of 9 .. 32 tokens
+
 // ---- host side ---------------------------------------------------------------------------
 struct LeanPlan {
-  int grid, nc, cap_bytes, red_rows, max_cols, cols_q, cols_rem, smem, kb;
+  int grid, nc, ntg, cap_bytes, red_rows, max_cols, cols_q, cols_rem, smem, kb, slot_d;
   bool ok;
 };
 
-// Shapes: L <= 8; d a multiple of 64 up to 2048 (x fragments of a warp fit its registers);
-// d_e a power of two >= 64.
+// Shapes: d a multiple of 64 up to 2048 (x fragments of a warp fit its registers); d_e a power
+// of two >= 64; L <= 32 (up to 8 tokens: one token group; 9 .. 16: two; 17 .. 32: four, these
+// only for calls that share the device and do not come with raw router logits).
 //
 // How many CTAs a call gets. Every CTA reads all of x and all of h from L2, whatever its share
 // of the weights: with one CTA per SM that broadcast is half as many bytes again as the weights
 // themselves, and an SM takes bytes in from L2 only about one and a half times as fast as its
 // share of the HBM stream. A call therefore runs on a fraction of the SMs (grid = SMs / split),
-// each CTA with a `split` times larger share (up to two column tiles of out), and `split` times
-// as many calls are in flight to cover the rest of the device.
+// each CTA with a `split` times larger share (up to three column tiles of out), and `split`
+// times as many calls are in flight to cover the rest of the device.
 //
-// The shared memory of a CTA is sized so that `per_sm` CTAs fit one SM; a share that does not
-// fit goes through in stages.
 // shared: the call may share the device with its neighbours (it depends on none of them)
 LeanPlan lean_plan(const blockffn_config& cfg, int L, int sms, bool shared) {
   LeanPlan pl{};
   pl.ok = false;
   const int d = cfg.d, d_e = cfg.d_e, E = cfg.E;
-  if (L < 1 || L > 8 || sms < 1) return pl;
+  if (L < 1 || L > 32 || sms < 1) return pl;
+  if (L > 8 && !shared) return pl;
   if (d % 64 || d > 512 * kMaxKB || d_e % 64 || (d_e & (d_e - 1)) || d_e > 4096 || E > 1024)
     return pl;
   pl.kb = (d / 64 + kWarps - 1) / kWarps;
+  pl.ntg = L <= 8 ? 1 : L <= 16 ? 2 : 4;
   int u_exp = (cfg.flags >> 17) & 0x7ff;
   if (u_exp == 0) u_exp = (L == 1 ? E + 4 : 3 * E + 5) / (L == 1 ? 8 : 10);
   if (u_exp < 1) u_exp = 1;
@@ -610,46 +613,51 @@ LeanPlan lean_plan(const blockffn_config& cfg, int L, int sms, bool shared) {
   // for calls that do not depend on one another; a call in a dependent chain is alone on the
   // device and takes all of it
   int split = shared && !(cfg.flags & BLOCKFFN_CFG_NO_SPLIT) ? 3 : 1;
-  for (;; --split) {                               // at most four column tiles per CTA
+  for (;; --split) {                               // at most three column tiles per CTA
     pl.grid = (sms + split - 1) / split;
     pl.nc = (d + 16 * pl.grid - 1) / (16 * pl.grid);
-    if (pl.nc <= 4 || split == 1) break;
+    if (pl.nc <= 3 || split == 1) break;
   }
-  if (pl.nc > 4) return pl;
+  if (pl.nc > 3) return pl;
   pl.cols_q = d / pl.grid;
   pl.cols_rem = d % pl.grid;
   pl.max_cols = pl.cols_q + (pl.cols_rem ? 1 : 0);
   const int rows_exp = (u_exp * d_e + pl.grid - 1) / pl.grid;
-  const int slot_d = pl.max_cols * 2 * d_e + 64;   // columns split even / odd around 64 bytes
-  const int need = max(min(rows_exp, 32) * 2 * d + 64, min(u_exp, 16) * slot_d);
+  // an expert's slot in the down projection: its slab of D (columns split even / odd around
+  // 64 bytes) and, with several token groups, its h tile
+  pl.slot_d = pl.max_cols * 2 * d_e + 64 + (pl.ntg > 1 ? 8 * pl.ntg * 2 * d_e + 64 : 0);
+  const int need = max(min(rows_exp, 32) * 2 * d + 64, min(u_exp, 16) * pl.slot_d);
   // the partial tile (and a stage) is as wide as the expected share, between one row tile per
   // column tile and two row tiles
   int red_rows = rows_exp < 32 ? rows_exp : 32;
   if (red_rows < 16 * pl.nc) red_rows = 16 * pl.nc;
-  const int fixed = lean_layout(E, red_rows, 0).total;
+  const int fixed = lean_layout(E, red_rows * pl.ntg, 0).total;
   // A call that owns the device gets the most CTAs per SM (three at most) whose shared memory
   // still holds the expected share in one stage; calls that share the device always run three
-  // to an SM and stream their larger shares through in stages.
-  for (int n = 3; n >= 1; --n) {
+  // to an SM and stream their larger shares through in stages; chunks of more than 8 tokens
+  // take a whole SM (their registers allow no more).
+  for (int n = pl.ntg > 1 ? 1 : 3; n >= 1; --n) {
     const int budget = (n == 1 ? kSmemMax : (kSmemMax + 1024) / n - 1024) & ~127;
     const int cap = (budget - fixed) & ~127;
     if (cap < need && n > 1 && split == 1) continue;
-    if (cap < 2 * 4 * 2 * d + 128 || cap < 2 * slot_d) {   // two stages of four rows, two slabs
+    if (cap < 2 * 4 * 2 * d + 128 || cap < 2 * pl.slot_d) {   // two stages of four rows, two slots
       if (n > 1) continue;
-      if (cap < 2 * 2 * d + 128 || cap < 2 * slot_d) return pl;
+      if (cap < 2 * 2 * d + 128 || cap < 2 * pl.slot_d) return pl;
     }
+    if (pl.ntg > 1 && cap < 8 * pl.ntg * 16 * pl.nc * kWarps * 4) return pl;   // the final partials
     pl.cap_bytes = cap;
     pl.red_rows = red_rows;
-    pl.smem = lean_layout(E, red_rows, cap).total;
+    pl.smem = lean_layout(E, red_rows * pl.ntg, cap).total;
     pl.ok = true;
     return pl;
   }
   return pl;
 }
 
-template <int KB, int NC, int MODE>
+template <int KB, int NC, int NTG, int MODE>
 cudaError_t lean_attr() {
-  const void* f = reinterpret_cast<const void*>(&expert_lean_kernel<KB, NC, MODE>);
+  const void* f = NTG == 1 ? reinterpret_cast<const void*>(&expert_lean_kernel<KB, NC, MODE>)
+                           : reinterpret_cast<const void*>(&expert_wide_kernel<KB, NC, NTG == 1 ? 2 : NTG, MODE>);
   cudaError_t e = cudaFuncSetAttribute(f, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemMax);
   if (e != cudaSuccess) return e;
   return cudaFuncSetAttribute(f, cudaFuncAttributePreferredSharedMemoryCarveout,
@@ -657,43 +665,62 @@ cudaError_t lean_attr() {
 }
 template <int KB, int NC>
 cudaError_t lean_attrs_kb() {
-  cudaError_t e = lean_attr<KB, NC, 0>();
-  if (e == cudaSuccess) e = lean_attr<KB, NC, 1>();
-  if (e == cudaSuccess) e = lean_attr<KB, NC, 2>();
+  cudaError_t e = lean_attr<KB, NC, 1, 0>();
+  if (e == cudaSuccess) e = lean_attr<KB, NC, 1, 1>();
+  if (e == cudaSuccess) e = lean_attr<KB, NC, 1, 2>();
+  if (e == cudaSuccess) e = lean_attr<KB, NC, 2, 0>();
+  if (e == cudaSuccess) e = lean_attr<KB, NC, 2, 1>();
+  if (e == cudaSuccess) e = lean_attr<KB, NC, 4, 0>();
+  if (e == cudaSuccess) e = lean_attr<KB, NC, 4, 1>();
   return e;
 }
 
 template <int KB, int NC>
-cudaError_t lean_launch_kb(const cudaLaunchConfig_t& lc, const LeanParams& p, int mode) {
-  return mode == 2   ? cudaLaunchKernelEx(&lc, expert_lean_kernel<KB, NC, 2>, p)
-         : mode == 1 ? cudaLaunchKernelEx(&lc, expert_lean_kernel<KB, NC, 1>, p)
-                     : cudaLaunchKernelEx(&lc, expert_lean_kernel<KB, NC, 0>, p);
+cudaError_t lean_launch_kb(const cudaLaunchConfig_t& lc, const LeanParams& p, int ntg, int mode) {
+  if (ntg == 1)
+    return mode == 2   ? cudaLaunchKernelEx(&lc, expert_lean_kernel<KB, NC, 2>, p)
+           : mode == 1 ? cudaLaunchKernelEx(&lc, expert_lean_kernel<KB, NC, 1>, p)
+                       : cudaLaunchKernelEx(&lc, expert_lean_kernel<KB, NC, 0>, p);
+  if (mode == 2) return cudaErrorNotSupported;
+  if (ntg == 2)
+    return mode == 1 ? cudaLaunchKernelEx(&lc, expert_wide_kernel<KB, NC, 2, 1>, p)
+                     : cudaLaunchKernelEx(&lc, expert_wide_kernel<KB, NC, 2, 0>, p);
+  return mode == 1 ? cudaLaunchKernelEx(&lc, expert_wide_kernel<KB, NC, 4, 1>, p)
+                   : cudaLaunchKernelEx(&lc, expert_wide_kernel<KB, NC, 4, 0>, p);
 }
 template <int NC>
-cudaError_t lean_launch_nc(int kb, const cudaLaunchConfig_t& lc, const LeanParams& p, int mode) {
+cudaError_t lean_launch_nc(int kb, const cudaLaunchConfig_t& lc, const LeanParams& p, int ntg,
+                           int mode) {
   switch (kb) {
-    case 1: return lean_launch_kb<1, NC>(lc, p, mode);
-    case 2: return lean_launch_kb<2, NC>(lc, p, mode);
-    case 3: return lean_launch_kb<3, NC>(lc, p, mode);
-    default: return lean_launch_kb<4, NC>(lc, p, mode);
+    case 1: return lean_launch_kb<1, NC>(lc, p, ntg, mode);
+    case 2: return lean_launch_kb<2, NC>(lc, p, ntg, mode);
+    case 3: return lean_launch_kb<3, NC>(lc, p, ntg, mode);
+    default: return lean_launch_kb<4, NC>(lc, p, ntg, mode);
   }
+}
+
+size_t lean_h_slot_bytes(const blockffn_config& cfg) {
+  return ((size_t)cfg.E * cfg.L_max * cfg.d_e * sizeof(uint16_t) + 255) & ~(size_t)255;
 }
 
 }  // namespace
 
-bool expert_lean_supported(const blockffn_ctx* c, int L) {
-  return c->lean_ring != nullptr && !(c->cfg.flags & BLOCKFFN_CFG_TWO_KERNELS) &&
-         lean_plan(c->cfg, L, c->num_sms, false).ok && lean_plan(c->cfg, L, c->num_sms, true).ok;
+// Whether a call of L tokens whose x is stable takes the one-kernel form (with_logits: it comes
+// with raw router logits, i.e. it is the expert stage of a router-on layer call).
+bool expert_lean_supported(const blockffn_ctx* c, int L, bool with_logits) {
+  if (c->lean_ring == nullptr || (c->cfg.flags & BLOCKFFN_CFG_TWO_KERNELS)) return false;
+  if (with_logits && L > 8) return false;
+  return lean_plan(c->cfg, L, c->num_sms, !with_logits).ok;
 }
 
 // Two rings (calls that own the device, calls that share it: their grids differ, so each kind
-// counts its own tickets) of kHRing intermediates of a chunk of 8 tokens; 0 when the shape never
-// takes this kernel (or the rings would be unreasonably large).
+// counts its own tickets) of kHRing intermediates of a chunk of L_max tokens; 0 when the shape
+// never takes this kernel (or the rings would be unreasonably large).
 size_t expert_lean_ws_bytes(const blockffn_config* cfg, int sms) {
   const int L = cfg->L_max < 8 ? cfg->L_max : 8;
   if (!lean_plan(*cfg, L, sms, false).ok || !lean_plan(*cfg, L, sms, true).ok) return 0;
-  const size_t slot = ((size_t)cfg->E * 8 * cfg->d_e * sizeof(uint16_t) + 255) & ~(size_t)255;
-  if (2 * kHRing * slot > ((size_t)128 << 20)) return 0;
+  const size_t slot = lean_h_slot_bytes(*cfg);
+  if (2 * kHRing * slot > ((size_t)256 << 20)) return 0;
   return 2 * kHRing * slot;
 }
 
@@ -711,10 +738,6 @@ cudaError_t expert_lean_setup(blockffn_ctx* c) {
   if (e == cudaSuccess) e = lean_attrs_kb<2, 3>();
   if (e == cudaSuccess) e = lean_attrs_kb<3, 3>();
   if (e == cudaSuccess) e = lean_attrs_kb<4, 3>();
-  if (e == cudaSuccess) e = lean_attrs_kb<1, 4>();
-  if (e == cudaSuccess) e = lean_attrs_kb<2, 4>();
-  if (e == cudaSuccess) e = lean_attrs_kb<3, 4>();
-  if (e == cudaSuccess) e = lean_attrs_kb<4, 4>();
   return e;
 }
 
@@ -725,12 +748,13 @@ cudaError_t launch_expert_lean(blockffn_ctx* c, const blockffn_weights* w, const
                                cudaStream_t st) {
   // Only for calls whose x is stable (for a router-on call: whose router has finished).
   if (logits ? !logits_final : !(call_flags & BLOCKFFN_CALL_INDEPENDENT_X)) return cudaErrorNotSupported;
+  if (!expert_lean_supported(c, L, logits != nullptr)) return cudaErrorNotSupported;
   // No router in front: the call consumes nothing of its predecessors and shares the device
   // with them (a router-on call is ordered behind its router by events, which keeps too few of
   // them in flight for a third of the device each).
   const bool shared = !logits;
   const LeanPlan pl = lean_plan(c->cfg, L, c->num_sms, shared);
-  if (!pl.ok || !c->lean_ring) return cudaErrorNotSupported;
+  if (!pl.ok) return cudaErrorNotSupported;
   LeanParams p{};
   p.x = static_cast<const uint16_t*>(x);
   p.U = static_cast<const uint16_t*>(w->U);
@@ -739,7 +763,7 @@ cudaError_t launch_expert_lean(blockffn_ctx* c, const blockffn_weights* w, const
   if (logits) p.lg = *logits;
   p.ids_in = union_ids;
   p.n_in = n_union;
-  p.h_slot = (((size_t)c->cfg.E * 8 * c->cfg.d_e * sizeof(uint16_t) + 255) & ~(size_t)255) / 2;
+  p.h_slot = lean_h_slot_bytes(c->cfg) / 2;
   p.h_ring = static_cast<uint16_t*>(c->lean_ring) + (shared ? kHRing * p.h_slot : 0);
   p.seq = c->lean_seq + (shared ? 32 : 0);
   p.ready = p.seq + 1;
@@ -752,9 +776,9 @@ cudaError_t launch_expert_lean(blockffn_ctx* c, const blockffn_weights* w, const
   p.de_shift = __builtin_ctz(c->cfg.d_e);
   p.cap_bytes = pl.cap_bytes;
   p.red_rows = pl.red_rows;
-  p.cap_rows = (pl.cap_bytes - 128) / (2 * c->cfg.d);
-  if (p.cap_rows > 64) p.cap_rows = 64;
-  p.cap_slabs = pl.cap_bytes / (pl.max_cols * 2 * c->cfg.d_e + 64);
+  p.cap_rows = (pl.cap_bytes - 256) / (2 * c->cfg.d);     // up to three stages, 64 bytes of padding each
+  if (p.cap_rows > 96) p.cap_rows = 96;
+  p.cap_slabs = pl.cap_bytes / pl.slot_d;
   p.magic_g = (uint32_t)((0x100000000ull + (unsigned)pl.grid - 1) / (unsigned)pl.grid);
   p.magic_cpr = (uint32_t)((0x10000u + (unsigned)(c->cfg.d / 8) - 1) / (unsigned)(c->cfg.d / 8));
   p.max_cols = pl.max_cols;
@@ -786,10 +810,9 @@ cudaError_t launch_expert_lean(blockffn_ctx* c, const blockffn_weights* w, const
   // never less than a quarter of an SM's shared memory: at most three CTAs then fit one SM,
   // whatever the shape, which is what the size of the ring rests on
   lc.dynamicSmemBytes = pl.smem > kMinSmem ? pl.smem : kMinSmem;
-  const cudaError_t e = pl.nc == 4   ? lean_launch_nc<4>(pl.kb, lc, p, mode)
-                        : pl.nc == 3 ? lean_launch_nc<3>(pl.kb, lc, p, mode)
-                        : pl.nc == 2 ? lean_launch_nc<2>(pl.kb, lc, p, mode)
-                                     : lean_launch_nc<1>(pl.kb, lc, p, mode);
+  const cudaError_t e = pl.nc == 3   ? lean_launch_nc<3>(pl.kb, lc, p, pl.ntg, mode)
+                        : pl.nc == 2 ? lean_launch_nc<2>(pl.kb, lc, p, pl.ntg, mode)
+                                     : lean_launch_nc<1>(pl.kb, lc, p, pl.ntg, mode);
   if (e == cudaSuccess) c->launches += 1;
   return e;
 }

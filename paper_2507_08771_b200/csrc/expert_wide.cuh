@@ -1,0 +1,508 @@
+// One-kernel expert stage for chunks of 9 .. 32 tokens (Eq. 1, Eq. 2 over Union(x), Sec. 3.3).
+// Included by expert_lean.cu inside its unnamed namespace: it shares that file's parameters,
+// shared-memory layout, ring of h buffers and helpers.
+#pragma once
+
+// The same kernel for chunks of 9 .. 32 tokens: NTG groups of 8 tokens (2 or 4) per weight
+// fragment. (A kernel of its own rather than NTG = 1 of this template: written for any NTG the
+// single-group case kept a few more values live and spilled, which cost 15 % at 8 tokens.)
+//
+// Chunks of more than 8 tokens take a whole SM per CTA: the x fragments of all token
+// groups stay in registers (up to 128 of them), every weight fragment read from shared memory is
+// used for all groups at once, and in the down projection the intermediate h of a round's experts
+// is staged in shared memory next to their slabs of D, because its fragments for all groups no
+// longer fit the registers next to NC x NTG accumulator tiles.
+template <int KB, int NC, int NTG, int MODE>
+__global__ void __launch_bounds__(kThreads, 1) expert_wide_kernel(const LeanParams p) {
+  extern __shared__ __align__(128) unsigned char smem[];
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int d = p.d, d_e = p.d_e, L = p.L;
+  const LeanLayout lay = lean_layout(p.E, p.red_rows * NTG, p.cap_bytes);
+  const uint32_t sbase = smem_u32(smem);
+  const uint32_t wbase = sbase + lay.off_w;
+  int* ctl = reinterpret_cast<int*>(smem + kOffCtl);
+  int* ids_sm = reinterpret_cast<int*>(smem + kOffIds);
+  float* red = reinterpret_cast<float*>(smem + lay.off_red);
+  const int g = lane >> 2, tg = lane & 3;
+  const int G = gridDim.x, bx = blockIdx.x;
+
+  if (tid < 8) ctl[tid] = 0;
+  unsigned long long ticket = 0;
+  if (tid == 0) ticket = atomicAdd(p.seq, 1ull);
+  __syncthreads();
+  // Thread 0 turns its ticket into the call's ring slot and lets the dependents go while the
+  // routing loads are in flight: every CTA of this call then holds its ticket before a CTA of
+  // the next call exists, and the next call starts as early as that allows.
+  auto on_ticket = [&]() {
+    const unsigned long long n = ticket / (unsigned)G;
+    ctl[6] = (int)(n & (kHRing - 1));
+    *reinterpret_cast<unsigned long long*>(ctl + 138) =
+        p.hold ? ~0ull : (n / kHRing + 1ull) * (unsigned)G;
+    pdl_trigger();
+  };
+  const int nu = derive_union<MODE>(p.scores, p.lg, p.ids_in, p.n_in, L, p.E, ids_sm, ctl,
+                                    reinterpret_cast<uint32_t*>(red), on_ticket);
+
+  // ---- up projection ---------------------------------------------------------------------
+  const int R = nu * d_e;
+  const int rq = (int)__umulhi((unsigned)R, p.magic_g), rrem = R - rq * G;
+  const int r0 = bx * rq + min(bx, rrem), nrows = rq + (bx < rrem ? 1 : 0), r1 = r0 + nrows;
+  const int row_bytes = 2 * d;
+  const int cap_rows = p.cap_rows;
+  // one stage when the share fits (the usual case: no division on that path), else stages of
+  // half the region that are refilled as they free
+  // (chunks of more than 8 tokens have a whole SM's shared memory: three stages in the ring, so
+  // that two are in flight under the math of the third)
+  constexpr int NS = NTG == 1 ? 2 : 3;
+  const int ldr = min(p.red_rows, 32);       // a stage is at most two row tiles
+  const bool single = nrows <= min(ldr, cap_rows);
+  const int slot_rows = single ? max(nrows, 1) : min(ldr, cap_rows / NS);
+  const int ngroups = single ? (nrows > 0 ? 1 : 0) : (nrows + slot_rows - 1) / slot_rows;
+  const int rpg = single ? nrows : (nrows + ngroups - 1) / ngroups;
+  const int half_u = ((slot_rows + 1) >> 1) * row_bytes + 64;   // where the odd rows start
+  const int slot_bytes = slot_rows * row_bytes + 64;
+  const int sh = p.de_shift;
+  // This thread's part of a row copy: 16-byte chunk my_c of the rows my_sub, my_sub + rpi, ...
+  const int cpr = d >> 3;                       // chunks per row (<= 256)
+  const int rpi = cpr > 128 ? 1 : kThreads / cpr;   // rows the CTA copies per step
+  const int my_sub = (tid * p.magic_cpr) >> 16, my_c = tid - my_sub * cpr;
+  const bool copies_u = my_sub < rpi;
+  // stage gi: rows [r0 + gi rpg, ...) -> slot gi % NS, row m of the stage at
+  // (m >> 1) row_bytes + (m & 1) half_u
+  auto issue_u = [&](int gi) {
+    const int ra = r0 + gi * rpg;
+    const int rows = min(r1, ra + rpg) - ra;
+    const uint32_t slot0 = wbase + (gi % NS) * slot_bytes + my_c * 16;
+    if (!copies_u) return;
+    if (rpi == 1) {
+      // every thread walks all rows: two running destinations (even rows, odd rows), the
+      // source index steps by one row inside an expert and jumps at an expert's end
+      uint32_t de = slot0, dd = slot0 + half_u;
+      int m = 0;
+      while (m < rows) {
+        const int r = ra + m, q = r >> sh;
+        const int seg_end = min(rows, ((q + 1) << sh) - ra);     // rows of this expert end here
+        uint32_t idx = (uint32_t)(ids_sm[q] * d_e + (r - (q << sh))) * (uint32_t)cpr + my_c;
+        if (m & 1) {               // start on an even row of the stage
+          cp_async16(dd, at16(p.U, idx));
+          dd += row_bytes;
+          idx += cpr;
+          ++m;
+        }
+#pragma unroll 2
+        for (; m + 1 < seg_end; m += 2, idx += 2 * cpr, de += row_bytes, dd += row_bytes) {
+          cp_async16(de, at16(p.U, idx));
+          cp_async16(dd, at16(p.U, idx + cpr));
+        }
+        if (m < seg_end) {
+          cp_async16(de, at16(p.U, idx));
+          de += row_bytes;
+          ++m;
+        }
+      }
+    } else {
+      int m = my_sub;
+      while (m < rows) {
+        const int r = ra + m, q = r >> sh;
+        const int seg_end = min(rows, ((q + 1) << sh) - ra);
+        uint32_t idx = (uint32_t)(ids_sm[q] * d_e + (r - (q << sh))) * (uint32_t)cpr + my_c;
+        const uint32_t step = (uint32_t)rpi * cpr;
+        for (; m < seg_end; m += rpi, idx += step)
+          cp_async16(slot0 + (m >> 1) * row_bytes + (m & 1) * half_u, at16(p.U, idx));
+      }
+    }
+  };
+  // score and h element (expert slot, token, neuron) this thread finishes in a stage, per token
+  // group: token 8 n + tid / 32, row tid % 32 of the stage
+  float sc[NTG];
+  int hidx[NTG];        // element index into the h buffer, -1: nothing to finish
+  auto prepare = [&](int gi) {
+    const int ra = r0 + gi * rpg, rows = min(r1, ra + rpg) - ra;
+    const int m = tid & 31;
+    const int hq = (ra + m) >> sh;
+    const int id = m < rows ? ids_sm[hq] : 0;
+#pragma unroll
+    for (int n = 0; n < NTG; ++n) {
+      const int t = 8 * n + (tid >> 5);
+      sc[n] = 0.0f;
+      hidx[n] = -1;
+      if (t < L && m < rows) {
+        hidx[n] = (hq * L + t) * d_e + (ra + m - (hq << sh));
+        if constexpr (MODE == 2) {
+          float v = __ldcg(p.lg.a0 + t * p.E + id);
+          v = v > 0.0f ? v : 0.0f;
+          sc[n] = __ldg(p.lg.gain + id) * v * reinterpret_cast<const float*>(ctl + 104)[t];
+        } else {
+          sc[n] = __ldcg(p.scores + t * p.E + id);
+        }
+      }
+    }
+  };
+  // x: this warp's k blocks (warp + 8 i) of the token rows this lane feeds to the mma
+  const int npx = d >> 6;
+  Frag64 fx[NTG][KB];
+  auto load_x = [&]() {
+#pragma unroll
+    for (int n = 0; n < NTG; ++n) {
+      const uint4* xp = reinterpret_cast<const uint4*>(p.x + min(8 * n + g, L - 1) * d + 64 * warp) + tg;
+#pragma unroll
+      for (int i = 0; i < KB; ++i) {
+        if (warp + kWarps * i < npx) {
+          fx[n][i].lo = ld_cg_v4(xp + 64 * i);       // 64 k blocks of 128 bytes = 8 warps further
+          fx[n][i].hi = ld_cg_v4(xp + 64 * i + 4);
+        } else {
+          fx[n][i].lo = fx[n][i].hi = make_uint4(0, 0, 0, 0);
+        }
+      }
+    }
+  };
+  // x goes first: its short round trip then runs under the long issue of the weights instead
+  // of behind it
+  load_x();
+#pragma unroll
+  for (int gi = 0; gi < NS; ++gi) {          // one commit group per stage, empty ones included
+    if (gi < ngroups) issue_u(gi);
+    cp_async_commit();
+  }
+  if (ngroups > 0) prepare(0);
+  const int slot = ctl[6];       // (written before the barriers inside derive_union)
+  uint16_t* hbuf = p.h_ring + (size_t)slot * p.h_slot;
+
+  for (int gi = 0; gi < ngroups; ++gi) {
+    const int rows = min(r1, r0 + (gi + 1) * rpg) - (r0 + gi * rpg);
+    // fragment addresses of rows g and g + 8 (same parity) of the two 16-row tiles, at this
+    // warp's first k block; rows beyond the stage read its last row (their results are dropped)
+    auto row_addr = [&](int m) {
+      m = min(m, rows - 1);
+      return wbase + (gi % NS) * slot_bytes + (m >> 1) * row_bytes + (m & 1) * half_u + 128 * warp +
+             16 * tg;
+    };
+    cp_async_wait_group<NS - 1>(); // all but the NS - 1 newest groups: this stage has landed
+    __syncthreads();
+    // partial tiles -> red[t][m][warp]: the eight partials of an element are 32 contiguous bytes
+    float* mine = red + (2 * tg * ldr + g) * kWarps + warp;
+    const int nt = ldr * kWarps;           // one token further
+    auto do_tile = [&](const int tile) {
+      const uint32_t a0 = row_addr(g + 16 * tile), b0 = row_addr(g + 16 * tile + 8);
+      float c0[NTG][4], c1[NTG][4];
+#pragma unroll
+      for (int n = 0; n < NTG; ++n)
+#pragma unroll
+        for (int v = 0; v < 4; ++v) c0[n][v] = c1[n][v] = 0.0f;
+#pragma unroll
+      for (int i = 0; i < KB; ++i) {
+        if (warp + kWarps * i < npx) {
+          const uint4 alo = lds128(a0 + 1024 * i), ahi = lds128(a0 + 1024 * i + 64);
+          const uint4 blo = lds128(b0 + 1024 * i), bhi = lds128(b0 + 1024 * i + 64);
+#pragma unroll
+          for (int n = 0; n < NTG; ++n) mma64(c0[n], c1[n], alo, ahi, blo, bhi, fx[n][i]);
+        }
+      }
+      const int m0 = g + 16 * tile;
+#pragma unroll
+      for (int n = 0; n < NTG; ++n) {
+        float* o = mine + (8 * n * ldr + 16 * tile) * kWarps;
+        if (m0 < ldr) {
+          o[0] = c0[n][0] + c1[n][0];
+          o[nt] = c0[n][1] + c1[n][1];
+        }
+        if (m0 + 8 < ldr) {
+          o[8 * kWarps] = c0[n][2] + c1[n][2];
+          o[nt + 8 * kWarps] = c0[n][3] + c1[n][3];
+        }
+      }
+    };
+    do_tile(0);
+    if (rows > 16) do_tile(1);     // second tile of 16 rows
+    __syncthreads();               // partials complete; every warp is done with the slot
+    if (gi + NS < ngroups) issue_u(gi + NS);
+    cp_async_commit();
+#pragma unroll
+    for (int n = 0; n < NTG; ++n) {
+      if (hidx[n] >= 0) {
+        const float4* part =
+            reinterpret_cast<const float4*>(red + ((8 * n + (tid >> 5)) * ldr + (tid & 31)) * kWarps);
+        const float4 lo = part[0], hi = part[1];
+        const float v = ((lo.x + lo.y) + (lo.z + lo.w)) + ((hi.x + hi.y) + (hi.z + hi.w));
+        hbuf[hidx[n]] = (uint16_t)f32_to_bf16_bits(sc[n] * swish_fast(v));
+      }
+    }
+    if (gi + 1 < ngroups) prepare(gi + 1);
+    // the next stage starts with a wait and a barrier, which also protects red
+  }
+  cp_async_wait_all();
+  __syncthreads();                 // every h element of this CTA has been stored
+  if (tid == kSyncThread) {
+    __threadfence();
+    asm volatile("red.relaxed.gpu.global.add.u64 [%0], 1;" ::"l"(p.ready + slot) : "memory");
+  }
+
+  // ---- down projection -------------------------------------------------------------------
+  // Slab of one expert: the CTA's columns (at most 16 NC, NC mma row tiles) as rows of 2 d_e
+  // bytes, even columns first, 64 bytes of padding, odd columns. With several token groups the
+  // expert's h tile follows its slab: token rows of 2 d_e bytes, split even / odd the same way.
+  const int drow = 2 * d_e;
+  const int half_d = ((p.max_cols + 1) >> 1) * drow + 64;
+  const int half_h = 4 * NTG * drow + 64;
+  const int slot_d = p.max_cols * drow + 64 + (NTG > 1 ? 8 * NTG * drow + 64 : 0);
+  const int h_off = p.max_cols * drow + 64;     // the h tile inside an expert's slot
+  const int cap_slabs = p.cap_slabs;
+  const bool one_round = nu <= cap_slabs;
+  const int rsz = one_round ? max(nu, 1) : max(1, cap_slabs / 2);
+  const int nrounds = one_round ? (nu > 0 ? 1 : 0) : (nu + rsz - 1) / rsz;
+  const int c0 = bx * p.cols_q + min(bx, p.cols_rem);
+  const int ncols = p.cols_q + (bx < p.cols_rem ? 1 : 0);
+  // A slab is ncols << kshift chunks of 16 bytes; chunk c = column c >> kshift, piece
+  // c & (2^kshift - 1). Thread tid copies chunks tid, tid + kCopyThreads, ... of every expert.
+  const int kshift = sh - 3;                    // log2(chunks per D row)
+  const uint32_t estride16 = (uint32_t)d << kshift;
+  const int nchunks = tid < kCopyThreads ? ncols << kshift : 0;
+  auto issue_d = [&](int r) {
+    const int q0 = r * rsz, n = min(rsz, nu - q0);
+    for (int c = tid; c < nchunks; c += kCopyThreads) {
+      const int cc = c >> kshift, k = c & ((1 << kshift) - 1);
+      const uint32_t src0 = ((uint32_t)(c0 + cc) << kshift) + k;          // + id * d << kshift
+      uint32_t dst = wbase + (r & 1) * rsz * slot_d + (cc >> 1) * drow + (cc & 1) * half_d + k * 16;
+#pragma unroll 4
+      for (int i = 0; i < n; ++i, dst += slot_d)
+        cp_async16(dst, at16(p.D, src0 + (uint32_t)ids_sm[q0 + i] * estride16));
+    }
+  };
+  // (several token groups) the h tiles of a round's experts: L rows of 2 d_e bytes per expert,
+  // contiguous in the h buffer; chunk c = token c >> kshift, piece c & (2^kshift - 1)
+  auto issue_h = [&](int r) {
+    const int q0 = r * rsz, n = min(rsz, nu - q0);
+    const uint32_t hstep16 = (uint32_t)(L * d_e) >> 3;
+    for (int c = tid; c < (L << kshift); c += kThreads) {
+      const int t = c >> kshift, k = c & ((1 << kshift) - 1);
+      uint32_t dst = wbase + (r & 1) * rsz * slot_d + h_off + (t >> 1) * drow + (t & 1) * half_h + k * 16;
+      uint32_t src = (uint32_t)q0 * hstep16 + c;
+      for (int i = 0; i < n; ++i, dst += slot_d, src += hstep16) cp_async16(dst, at16(hbuf, src));
+    }
+  };
+  if (nrounds > 0) issue_d(0);
+  cp_async_commit();
+  if (nrounds > 1) issue_d(1);
+  cp_async_commit();
+  const int ot = tid >> 5, om = tid & 31;   // this thread's outputs: tokens ot (+ 8), columns om (+ 32)
+  // hand-over: all CTAs of this call have stored their part of h
+  if (tid == kSyncThread) {
+    const unsigned long long target = *reinterpret_cast<const unsigned long long*>(ctl + 138);
+    const unsigned long long t0 = global_ns();
+    // once a wait has run out on this handle the later ones give up quickly, until the caller
+    // has read and cleared the status word
+    const bool before = (*reinterpret_cast<volatile uint32_t*>(p.status) & BLOCKFFN_DEV_WAIT_EXPIRED) != 0;
+    const unsigned long long limit = p.hold ? 2000000ull : before ? 1000000ull : p.wait_ns;
+    int expired = 0;
+    while (ld_acquire_u64(p.ready + slot) < target) {
+      if (global_ns() - t0 > limit) {
+        expired = 1;
+        break;
+      }
+    }
+    if (expired) {
+      ctl[5] = 1;
+      atomicOr(p.status, BLOCKFFN_DEV_WAIT_EXPIRED);
+    }
+  }
+  __syncthreads();
+  const bool dead = ctl[5] != 0;    // the wait ran out: out is left untouched
+  if constexpr (NTG > 1) {
+    if (!dead) {
+      if (nrounds > 0) issue_h(0);
+      cp_async_commit();
+      if (nrounds > 1) issue_h(1);
+      cp_async_commit();
+    }
+  }
+
+  const int npairs = d_e >> 6;      // 64-wide k blocks per expert (a power of two)
+  const int pshift = sh - 6;
+  float acc[NC][NTG][2][4];
+#pragma unroll
+  for (int c = 0; c < NC; ++c)
+#pragma unroll
+    for (int n = 0; n < NTG; ++n)
+#pragma unroll
+      for (int v = 0; v < 4; ++v) acc[c][n][0][v] = acc[c][n][1][v] = 0.0f;
+  // rows (columns of out) g, g + 8 (, g + 16, g + 24) of a slab, clamped to the CTA's columns
+  auto col_off = [&](int m) {
+    m = min(m, max(ncols, 1) - 1);
+    return (m >> 1) * drow + (m & 1) * half_d + 16 * tg;
+  };
+  uint32_t offs[NC][2];
+#pragma unroll
+  for (int c = 0; c < NC; ++c) {
+    offs[c][0] = col_off(g + 16 * c);
+    offs[c][1] = col_off(g + 16 * c + 8);
+  }
+  const uint4* hrow = reinterpret_cast<const uint4*>(hbuf + min(g, L - 1) * d_e) + tg;
+  const uint32_t hstep16 = (uint32_t)(L * d_e) >> 3;         // one expert further, in 16 bytes
+  // (several token groups) token rows 8 n + g of an h tile in shared memory (rows beyond the
+  // chunk hold whatever the buffer held: their columns of the result are dropped)
+  const uint32_t hs_off = h_off + (g >> 1) * drow + (g & 1) * half_h + 16 * tg;
+  for (int r = 0; r < nrounds && !dead; ++r) {
+    const int q0 = r * rsz, n = min(rsz, nu - q0);
+    const int nblk = n << pshift;
+    const uint32_t d_base = wbase + (r & 1) * rsz * slot_d;
+    if constexpr (NTG == 1) {
+      // this warp's k blocks b = warp + 8 i of the round, in batches whose h fragments are all
+      // requested before the first is used; block b = expert b >> pshift, k block b & (npairs - 1)
+      // (fewer per batch with more column tiles: their accumulators need the registers, and a
+      // round then holds fewer experts anyway)
+      constexpr int kHB = NC == 1 ? 5 : NC == 2 ? 3 : 2;
+      Frag64 fh[kHB];
+      auto load_h = [&](int b0) {
+#pragma unroll
+        for (int i = 0; i < kHB; ++i) {
+          const int b = b0 + kWarps * i;
+          if (b < nblk) {
+            const uint4* hp = hrow + (uint32_t)(q0 + (b >> pshift)) * hstep16 + 8 * (b & (npairs - 1));
+            fh[i].lo = ld_cg_v4(hp);
+            fh[i].hi = ld_cg_v4(hp + 4);
+          }
+        }
+      };
+      load_h(warp);
+      cp_async_wait_group<1>();    // all but the newest group: this round's slabs have landed
+      __syncthreads();
+      for (int b0 = warp; b0 < nblk; b0 += kWarps * kHB) {
+        if (b0 != warp) load_h(b0);
+#pragma unroll
+        for (int i = 0; i < kHB; ++i) {
+          const int b = b0 + kWarps * i;
+          if (b < nblk) {
+            const uint32_t da = d_base + (b >> pshift) * slot_d + 128 * (b & (npairs - 1));
+#pragma unroll
+            for (int c = 0; c < NC; ++c) {
+              const uint4 alo = lds128(da + offs[c][0]), ahi = lds128(da + offs[c][0] + 64);
+              const uint4 blo = lds128(da + offs[c][1]), bhi = lds128(da + offs[c][1] + 64);
+              mma64(acc[c][0][0], acc[c][0][1], alo, ahi, blo, bhi, fh[i]);
+            }
+          }
+        }
+      }
+    } else {
+      cp_async_wait_group<1>();    // this round's slabs and h tiles have landed
+      __syncthreads();
+#pragma unroll 1
+      for (int b = warp; b < nblk; b += kWarps) {
+        const uint32_t da = d_base + (b >> pshift) * slot_d + 128 * (b & (npairs - 1));
+        Frag64 fh[NTG];
+#pragma unroll
+        for (int n2 = 0; n2 < NTG; ++n2) {
+          fh[n2].lo = lds128(da + hs_off + 4 * n2 * drow);      // 8 token rows = 4 row pairs further
+          fh[n2].hi = lds128(da + hs_off + 4 * n2 * drow + 64);
+        }
+#pragma unroll
+        for (int c = 0; c < NC; ++c) {
+          const uint4 alo = lds128(da + offs[c][0]), ahi = lds128(da + offs[c][0] + 64);
+          const uint4 blo = lds128(da + offs[c][1]), bhi = lds128(da + offs[c][1] + 64);
+#pragma unroll
+          for (int n2 = 0; n2 < NTG; ++n2)
+            mma64(acc[c][n2][0], acc[c][n2][1], alo, ahi, blo, bhi, fh[n2]);
+        }
+      }
+    }
+    __syncthreads();               // every warp is done with this round's slabs
+    if (r + 2 < nrounds) {
+      issue_d(r + 2);
+      if constexpr (NTG > 1) issue_h(r + 2);
+    }
+    cp_async_commit();
+  }
+  cp_async_wait_all();
+  pdl_wait();                      // out (and x_next) may still be in use by the call before
+  if (!dead) {
+    if (nu > 0) {
+      // partial tiles -> part[t][m][warp] (m < 16 NC), then one thread per output element; with
+      // several token groups the partials take the weight region, which is free by now
+      float* part0 = NTG == 1 ? red : reinterpret_cast<float*>(smem + lay.off_w);
+      float* mine = part0 + (2 * tg * (16 * NC) + g) * kWarps + warp;
+#pragma unroll
+      for (int n = 0; n < NTG; ++n) {
+#pragma unroll
+        for (int c = 0; c < NC; ++c) {
+          float* o = mine + (8 * n * (16 * NC) + 16 * c) * kWarps;
+          o[0] = acc[c][n][0][0] + acc[c][n][1][0];
+          o[(16 * NC) * kWarps] = acc[c][n][0][1] + acc[c][n][1][1];
+          o[8 * kWarps] = acc[c][n][0][2] + acc[c][n][1][2];
+          o[(16 * NC + 8) * kWarps] = acc[c][n][0][3] + acc[c][n][1][3];
+        }
+      }
+      __syncthreads();
+#pragma unroll
+      for (int n = 0; n < NTG; ++n) {
+        const int t = ot + 8 * n;
+        if (t < L) {
+#pragma unroll
+          for (int k = 0; k < (NC + 1) / 2; ++k) {
+            const int m = om + 32 * k;
+            if (m < ncols) {
+              const float4* part = reinterpret_cast<const float4*>(part0 + (t * (16 * NC) + m) * kWarps);
+              const float4 lo = part[0], hi = part[1];
+              float v = ((lo.x + lo.y) + (lo.z + lo.w)) + ((hi.x + hi.y) + (hi.z + hi.w));
+              const int o = t * d + c0 + m;
+              if (p.accumulate) v += __ldcg(p.out + o);
+              p.out[o] = v;
+              if (p.x_next) p.x_next[o] = (uint16_t)f32_to_bf16_bits(v);
+            }
+          }
+        }
+      }
+    } else {                       // empty union: FFN(x) = 0
+      for (int t = ot; t < L; t += 8) {
+        for (int m = om; m < ncols; m += 32) {
+          const int o = t * d + c0 + m;
+          const float v = p.accumulate ? __ldcg(p.out + o) : 0.0f;
+          p.out[o] = v;
+          if (p.x_next) p.x_next[o] = (uint16_t)f32_to_bf16_bits(v);
+        }
+      }
+    }
+  }
+  // CTA 0 publishes the routing it derived (after the wait: earlier readers are done)
+  if (blockIdx.x == 0) {
+    if (p.lg.a0 != nullptr && p.pub_scores != nullptr) {
+      const int words = (p.E + 31) >> 5;
+      const float* rinv = reinterpret_cast<const float*>(ctl + 104);
+      for (int t = warp; t < L; t += kWarps) {
+        for (int w = 0; w < words; ++w) {
+          const int e = 32 * w + lane;
+          float sv = 0.0f;
+          if (e < p.E) {
+            float v = __ldcg(p.lg.a0 + (size_t)t * p.E + e);
+            v = v > 0.0f ? v : 0.0f;
+            sv = __ldg(p.lg.gain + e) * v * rinv[t];
+            p.pub_scores[(size_t)t * p.E + e] = sv;
+          }
+          const uint32_t m = __ballot_sync(0xffffffffu, sv != 0.0f);
+          if (p.pub_tok && lane == 0) p.pub_tok[(size_t)t * words + w] = m;
+        }
+      }
+    }
+    if (p.ids_in == nullptr) {
+      const int words = (p.E + 31) >> 5;
+      const uint32_t* um = reinterpret_cast<const uint32_t*>(ctl + 8);
+      for (int e = tid; e < p.E; e += kThreads) {
+        if (p.pub_ids) p.pub_ids[e] = e < nu ? ids_sm[e] : -1;
+        if (p.pub_mask && e < words) p.pub_mask[e] = um[e];
+      }
+      if (tid == 0) {
+        if (p.pub_n) *p.pub_n = nu;
+        if (p.stats) {
+          atomicAdd(reinterpret_cast<unsigned long long*>(&p.stats->n_tokens),
+                    (unsigned long long)L);
+          atomicAdd(reinterpret_cast<unsigned long long*>(&p.stats->n_active),
+                    (unsigned long long)ctl[2]);
+          atomicAdd(reinterpret_cast<unsigned long long*>(&p.stats->n_chunks), 1ull);
+          atomicAdd(reinterpret_cast<unsigned long long*>(&p.stats->n_union),
+                    (unsigned long long)nu);
+        }
+      }
+    } else if (tid == 0 && ctl[3]) {
+      atomicOr(p.status, (uint32_t)ctl[3]);
+    }
+  }
+}
+

@@ -179,12 +179,14 @@ def test_expert_ffn(variant, d, E, d_e, L, p):
     (256, 16, 64, 4, 0.5), (768, 48, 64, 8, 0.2), (1280, 40, 128, 5, 0.2), (1536, 48, 128, 8, 0.25),
     (1792, 56, 128, 7, 0.15), (2048, 64, 128, 8, 0.12), (2048, 64, 128, 8, 1.0), (2048, 128, 128, 1, 0.1),
     (2048, 128, 128, 8, 0.05), (512, 128, 256, 3, 0.2), (1024, 1000, 64, 8, 0.02), (64, 5, 64, 8, 0.6),
-    (2048, 64, 128, 16, 0.1)])
+    (2048, 64, 128, 16, 0.1), (2048, 64, 128, 32, 0.1), (1536, 48, 128, 17, 0.2), (768, 48, 64, 9, 0.2),
+    (2048, 128, 128, 31, 0.3), (512, 24, 64, 32, 0.5), (2048, 64, 128, 12, 1.0)])
 def test_expert_ffn_under_call_promises(kind, d, E, d_e, L, p):
     """The expert stage under the two per-call promises. With x promised stable the one-kernel form
     runs a call on a third of the SMs (up to four column tiles of out and several stages per CTA);
-    with only the weights promised stable it owns the device. Shapes cover one to four column
-    tiles, one and several stages, unions from a few experts to all of them."""
+    with only the weights promised stable it owns the device. Shapes cover one to three column
+    tiles, one and several stages, unions from a few experts to all of them, and chunks of 9 to
+    32 tokens (two and four token groups per weight fragment in the one-kernel form)."""
     seed = 3000 + d + E + L
     sh, w = small_layer(d, E, d_e, seed)
     rng = np.random.default_rng(seed)
@@ -661,11 +663,15 @@ def graph_of(fn):
         stream.synchronize()
 
 
-@pytest.mark.parametrize("cfg,flag", [(1, B.CALL_INDEPENDENT_X), (2, B.CALL_INDEPENDENT_X),
-                                      (2, B.CALL_INDEPENDENT), (2, 0)])
-def test_bench_launch_configuration_scores_in(cfg, flag):
+@pytest.mark.parametrize("cfg,flag,L", [(1, B.CALL_INDEPENDENT_X, None), (2, B.CALL_INDEPENDENT_X, None),
+                                        (2, B.CALL_INDEPENDENT, None), (2, 0, None),
+                                        (2, B.CALL_INDEPENDENT_X, 16), (2, B.CALL_INDEPENDENT_X, 32),
+                                        (5, B.CALL_INDEPENDENT_X, 32)])
+def test_bench_launch_configuration_scores_in(cfg, flag, L):
     sh, seed = I.SHAPES[cfg], I.config_seed(cfg)
-    n_chunks, n_copies = 24, 3
+    if L is not None:
+        sh = I.Shape(sh.name, d=sh.d, E=sh.E, d_e=sh.d_e, L=L, union_frac=sh.u / sh.E)
+    n_chunks, n_copies = (24, 3) if L is None else (12, 2)
     w = I.make_layer(sh, seed, with_router=False)
     layer = B.Layer(sh.d, sh.E, sh.d_e, L_max=sh.L)
     dws = [layer.upload_weights(w) for _ in range(n_copies)]
