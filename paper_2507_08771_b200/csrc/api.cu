@@ -124,7 +124,7 @@ blockffn_status blockffn_create(const blockffn_config* cfg, blockffn_handle* out
   const size_t o_h16 = take(expert_mma_h_bytes(cfg));
   const size_t lean_bytes = expert_lean_ws_bytes(cfg, c->num_sms);
   const size_t o_lean = take(lean_bytes);
-  const size_t o_seq = take(sizeof(unsigned long long) * 64);
+  const size_t o_seq = take(sizeof(unsigned long long) * 96);
   const size_t o_tk = take(sizeof(unsigned int) * 8);
   const size_t o_st = take(sizeof(uint32_t));
   void* base = nullptr;

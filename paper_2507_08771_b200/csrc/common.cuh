@@ -40,7 +40,7 @@ struct blockffn_ctx {
   float* h32;           // [E][L_max][d_e] fp32 intermediate (SIMT variant)
   void* h16;            // bf16 intermediate (MMA variant), slot-major padded rows
   void* lean_ring;      // ring of bf16 intermediates of the one-kernel form (NULL: not used)
-  unsigned long long* lean_seq;   // per ring (two of them, 32 words apart): [0] call tickets,
+  unsigned long long* lean_seq;   // per ring (three of them, 32 words apart): [0] call tickets,
                                   // [1 .. 16] arrival counters of the ring slots
   unsigned int* ticket; // last-block-done counters [8]
   uint32_t* status;     // sticky device status word

@@ -579,7 +579,7 @@ __global__ void __launch_bounds__(kThreads, 3) expert_lean_kernel(const LeanPara
 
 // ---- host side ---------------------------------------------------------------------------
 struct LeanPlan {
-  int grid, nc, ntg, cap_bytes, red_rows, max_cols, cols_q, cols_rem, smem, kb, slot_d;
+  int grid, slices, nc, ntg, cap_bytes, red_rows, max_cols, cols_q, cols_rem, smem, kb, slot_d;
   bool ok;
 };
 
@@ -604,7 +604,8 @@ LeanPlan lean_plan(const blockffn_config& cfg, int L, int sms, bool shared) {
   if (d % 64 || d > 512 * kMaxKB || d_e % 64 || (d_e & (d_e - 1)) || d_e > 4096 || E > 1024)
     return pl;
   pl.kb = (d / 64 + kWarps - 1) / kWarps;
-  pl.ntg = L <= 8 ? 1 : L <= 16 ? 2 : 4;
+  pl.slices = L > 16 ? 2 : 1;
+  pl.ntg = L <= 8 ? 1 : 2;            // longer chunks: slices of at most 16 tokens, two groups each
   int u_exp = (cfg.flags >> 17) & 0x7ff;
   if (u_exp == 0) u_exp = (L == 1 ? E + 4 : 3 * E + 5) / (L == 1 ? 8 : 10);
   if (u_exp < 1) u_exp = 1;
@@ -636,7 +637,7 @@ LeanPlan lean_plan(const blockffn_config& cfg, int L, int sms, bool shared) {
   // still holds the expected share in one stage; calls that share the device always run three
   // to an SM and stream their larger shares through in stages; chunks of more than 8 tokens
   // take a whole SM (their registers allow no more).
-  for (int n = pl.ntg > 1 ? 1 : 3; n >= 1; --n) {
+  for (int n = pl.ntg == 2 ? 2 : 3; n >= 1; --n) {
     const int budget = (n == 1 ? kSmemMax : (kSmemMax + 1024) / n - 1024) & ~127;
     const int cap = (budget - fixed) & ~127;
     if (cap < need && n > 1 && split == 1) continue;
@@ -644,7 +645,14 @@ LeanPlan lean_plan(const blockffn_config& cfg, int L, int sms, bool shared) {
       if (n > 1) continue;
       if (cap < 2 * 2 * d + 128 || cap < 2 * pl.slot_d) return pl;
     }
-    if (pl.ntg > 1 && cap < 8 * pl.ntg * 16 * pl.nc * kWarps * 4) return pl;   // the final partials
+    if (pl.ntg > 1 && cap < 8 * pl.ntg * 16 * pl.nc * kWarps * 4) {            // the final partials
+      if (n > 1) continue;
+      return pl;
+    }
+    // The hand-over inside the kernel needs every CTA of the call resident at once: n CTAs fit
+    // an SM (by shared memory here, and the kernels are compiled for at least as many by
+    // registers), so the call must not have more than n per SM.
+    if ((long long)pl.grid * pl.slices > (long long)sms * n) return pl;
     pl.cap_bytes = cap;
     pl.red_rows = red_rows;
     pl.smem = lean_layout(E, red_rows * pl.ntg, cap).total;
@@ -670,8 +678,6 @@ cudaError_t lean_attrs_kb() {
   if (e == cudaSuccess) e = lean_attr<KB, NC, 1, 2>();
   if (e == cudaSuccess) e = lean_attr<KB, NC, 2, 0>();
   if (e == cudaSuccess) e = lean_attr<KB, NC, 2, 1>();
-  if (e == cudaSuccess) e = lean_attr<KB, NC, 4, 0>();
-  if (e == cudaSuccess) e = lean_attr<KB, NC, 4, 1>();
   return e;
 }
 
@@ -682,11 +688,8 @@ cudaError_t lean_launch_kb(const cudaLaunchConfig_t& lc, const LeanParams& p, in
            : mode == 1 ? cudaLaunchKernelEx(&lc, expert_lean_kernel<KB, NC, 1>, p)
                        : cudaLaunchKernelEx(&lc, expert_lean_kernel<KB, NC, 0>, p);
   if (mode == 2) return cudaErrorNotSupported;
-  if (ntg == 2)
-    return mode == 1 ? cudaLaunchKernelEx(&lc, expert_wide_kernel<KB, NC, 2, 1>, p)
-                     : cudaLaunchKernelEx(&lc, expert_wide_kernel<KB, NC, 2, 0>, p);
-  return mode == 1 ? cudaLaunchKernelEx(&lc, expert_wide_kernel<KB, NC, 4, 1>, p)
-                   : cudaLaunchKernelEx(&lc, expert_wide_kernel<KB, NC, 4, 0>, p);
+  return mode == 1 ? cudaLaunchKernelEx(&lc, expert_wide_kernel<KB, NC, 2, 1>, p)
+                   : cudaLaunchKernelEx(&lc, expert_wide_kernel<KB, NC, 2, 0>, p);
 }
 template <int NC>
 cudaError_t lean_launch_nc(int kb, const cudaLaunchConfig_t& lc, const LeanParams& p, int ntg,
@@ -713,15 +716,16 @@ bool expert_lean_supported(const blockffn_ctx* c, int L, bool with_logits) {
   return lean_plan(c->cfg, L, c->num_sms, !with_logits).ok;
 }
 
-// Two rings (calls that own the device, calls that share it: their grids differ, so each kind
-// counts its own tickets) of kHRing intermediates of a chunk of L_max tokens; 0 when the shape
-// never takes this kernel (or the rings would be unreasonably large).
+// Three rings (calls that own the device, calls that share it, calls that share it in two token
+// slices: their grids differ, so each kind counts its own tickets) of kHRing intermediates of a
+// chunk of L_max tokens; 0 when the shape never takes this kernel (or the rings would be
+// unreasonably large).
 size_t expert_lean_ws_bytes(const blockffn_config* cfg, int sms) {
   const int L = cfg->L_max < 8 ? cfg->L_max : 8;
   if (!lean_plan(*cfg, L, sms, false).ok || !lean_plan(*cfg, L, sms, true).ok) return 0;
   const size_t slot = lean_h_slot_bytes(*cfg);
-  if (2 * kHRing * slot > ((size_t)256 << 20)) return 0;
-  return 2 * kHRing * slot;
+  if (3 * kHRing * slot > ((size_t)256 << 20)) return 0;
+  return 3 * kHRing * slot;
 }
 
 cudaError_t expert_lean_setup(blockffn_ctx* c) {
@@ -764,8 +768,11 @@ cudaError_t launch_expert_lean(blockffn_ctx* c, const blockffn_weights* w, const
   p.ids_in = union_ids;
   p.n_in = n_union;
   p.h_slot = lean_h_slot_bytes(c->cfg) / 2;
-  p.h_ring = static_cast<uint16_t*>(c->lean_ring) + (shared ? kHRing * p.h_slot : 0);
-  p.seq = c->lean_seq + (shared ? 32 : 0);
+  // a ring and a ticket counter per kind of call: tickets only identify a call when every call
+  // that draws from the counter has the same number of CTAs
+  const int ring = !shared ? 0 : pl.slices == 1 ? 1 : 2;
+  p.h_ring = static_cast<uint16_t*>(c->lean_ring) + (size_t)ring * kHRing * p.h_slot;
+  p.seq = c->lean_seq + 32 * ring;
   p.ready = p.seq + 1;
   p.out = out;
   p.x_next = static_cast<uint16_t*>(x_next);
@@ -802,7 +809,7 @@ cudaError_t launch_expert_lean(blockffn_ctx* c, const blockffn_weights* w, const
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cudaLaunchConfig_t lc{};
-  lc.gridDim = dim3(pl.grid);
+  lc.gridDim = dim3(pl.grid, pl.slices);
   lc.blockDim = dim3(kThreads);
   lc.stream = st;
   lc.attrs = attr;

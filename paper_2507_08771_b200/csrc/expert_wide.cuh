@@ -13,10 +13,15 @@
 // is staged in shared memory next to their slabs of D, because its fragments for all groups no
 // longer fit the registers next to NC x NTG accumulator tiles.
 template <int KB, int NC, int NTG, int MODE>
-__global__ void __launch_bounds__(kThreads, 1) expert_wide_kernel(const LeanParams p) {
+__global__ void __launch_bounds__(kThreads, NTG == 2 ? 2 : 1) expert_wide_kernel(const LeanParams p) {
   extern __shared__ __align__(128) unsigned char smem[];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int d = p.d, d_e = p.d_e, L = p.L;
+  // A chunk of more than 16 tokens is two slices of at most 16 (blockIdx.y): the slices share
+  // the call's union, its weights (read from DRAM once, the second reader finds them in L2), its
+  // ticket and its h buffer, and differ in their tokens. Lf: tokens of the chunk; tok0, L: the
+  // slice's first token and token count.
+  const int d = p.d, d_e = p.d_e, Lf = p.L;
+  const int tok0 = blockIdx.y * 16, L = min(16, Lf - tok0);
   const LeanLayout lay = lean_layout(p.E, p.red_rows * NTG, p.cap_bytes);
   const uint32_t sbase = smem_u32(smem);
   const uint32_t wbase = sbase + lay.off_w;
@@ -24,7 +29,8 @@ __global__ void __launch_bounds__(kThreads, 1) expert_wide_kernel(const LeanPara
   int* ids_sm = reinterpret_cast<int*>(smem + kOffIds);
   float* red = reinterpret_cast<float*>(smem + lay.off_red);
   const int g = lane >> 2, tg = lane & 3;
-  const int G = gridDim.x, bx = blockIdx.x;
+  const int G = gridDim.x, bx = blockIdx.x;   // the weights are shared out over gridDim.x
+  const unsigned Gt = gridDim.x * gridDim.y;  // CTAs of the call
 
   if (tid < 8) ctl[tid] = 0;
   unsigned long long ticket = 0;
@@ -34,13 +40,13 @@ __global__ void __launch_bounds__(kThreads, 1) expert_wide_kernel(const LeanPara
   // routing loads are in flight: every CTA of this call then holds its ticket before a CTA of
   // the next call exists, and the next call starts as early as that allows.
   auto on_ticket = [&]() {
-    const unsigned long long n = ticket / (unsigned)G;
+    const unsigned long long n = ticket / Gt;
     ctl[6] = (int)(n & (kHRing - 1));
     *reinterpret_cast<unsigned long long*>(ctl + 138) =
-        p.hold ? ~0ull : (n / kHRing + 1ull) * (unsigned)G;
+        p.hold ? ~0ull : (n / kHRing + 1ull) * Gt;
     pdl_trigger();
   };
-  const int nu = derive_union<MODE>(p.scores, p.lg, p.ids_in, p.n_in, L, p.E, ids_sm, ctl,
+  const int nu = derive_union<MODE>(p.scores, p.lg, p.ids_in, p.n_in, Lf, p.E, ids_sm, ctl,
                                     reinterpret_cast<uint32_t*>(red), on_ticket);
 
   // ---- up projection ---------------------------------------------------------------------
@@ -53,7 +59,7 @@ __global__ void __launch_bounds__(kThreads, 1) expert_wide_kernel(const LeanPara
   // half the region that are refilled as they free
   // (chunks of more than 8 tokens have a whole SM's shared memory: three stages in the ring, so
   // that two are in flight under the math of the third)
-  constexpr int NS = NTG == 1 ? 2 : 3;
+  constexpr int NS = NTG <= 2 ? 2 : 3;
   const int ldr = min(p.red_rows, 32);       // a stage is at most two row tiles
   const bool single = nrows <= min(ldr, cap_rows);
   const int slot_rows = single ? max(nrows, 1) : min(ldr, cap_rows / NS);
@@ -127,13 +133,13 @@ __global__ void __launch_bounds__(kThreads, 1) expert_wide_kernel(const LeanPara
       sc[n] = 0.0f;
       hidx[n] = -1;
       if (t < L && m < rows) {
-        hidx[n] = (hq * L + t) * d_e + (ra + m - (hq << sh));
+        hidx[n] = (hq * Lf + tok0 + t) * d_e + (ra + m - (hq << sh));
         if constexpr (MODE == 2) {
-          float v = __ldcg(p.lg.a0 + t * p.E + id);
+          float v = __ldcg(p.lg.a0 + (tok0 + t) * p.E + id);
           v = v > 0.0f ? v : 0.0f;
-          sc[n] = __ldg(p.lg.gain + id) * v * reinterpret_cast<const float*>(ctl + 104)[t];
+          sc[n] = __ldg(p.lg.gain + id) * v * reinterpret_cast<const float*>(ctl + 104)[tok0 + t];
         } else {
-          sc[n] = __ldcg(p.scores + t * p.E + id);
+          sc[n] = __ldcg(p.scores + (tok0 + t) * p.E + id);
         }
       }
     }
@@ -144,7 +150,7 @@ __global__ void __launch_bounds__(kThreads, 1) expert_wide_kernel(const LeanPara
   auto load_x = [&]() {
 #pragma unroll
     for (int n = 0; n < NTG; ++n) {
-      const uint4* xp = reinterpret_cast<const uint4*>(p.x + min(8 * n + g, L - 1) * d + 64 * warp) + tg;
+      const uint4* xp = reinterpret_cast<const uint4*>(p.x + (tok0 + min(8 * n + g, L - 1)) * d + 64 * warp) + tg;
 #pragma unroll
       for (int i = 0; i < KB; ++i) {
         if (warp + kWarps * i < npx) {
@@ -272,11 +278,11 @@ __global__ void __launch_bounds__(kThreads, 1) expert_wide_kernel(const LeanPara
   // contiguous in the h buffer; chunk c = token c >> kshift, piece c & (2^kshift - 1)
   auto issue_h = [&](int r) {
     const int q0 = r * rsz, n = min(rsz, nu - q0);
-    const uint32_t hstep16 = (uint32_t)(L * d_e) >> 3;
+    const uint32_t hstep16 = (uint32_t)(Lf * d_e) >> 3;
     for (int c = tid; c < (L << kshift); c += kThreads) {
       const int t = c >> kshift, k = c & ((1 << kshift) - 1);
       uint32_t dst = wbase + (r & 1) * rsz * slot_d + h_off + (t >> 1) * drow + (t & 1) * half_h + k * 16;
-      uint32_t src = (uint32_t)q0 * hstep16 + c;
+      uint32_t src = (uint32_t)q0 * hstep16 + ((uint32_t)tok0 << kshift) + c;
       for (int i = 0; i < n; ++i, dst += slot_d, src += hstep16) cp_async16(dst, at16(hbuf, src));
     }
   };
@@ -336,8 +342,8 @@ __global__ void __launch_bounds__(kThreads, 1) expert_wide_kernel(const LeanPara
     offs[c][0] = col_off(g + 16 * c);
     offs[c][1] = col_off(g + 16 * c + 8);
   }
-  const uint4* hrow = reinterpret_cast<const uint4*>(hbuf + min(g, L - 1) * d_e) + tg;
-  const uint32_t hstep16 = (uint32_t)(L * d_e) >> 3;         // one expert further, in 16 bytes
+  const uint4* hrow = reinterpret_cast<const uint4*>(hbuf + (tok0 + min(g, L - 1)) * d_e) + tg;
+  const uint32_t hstep16 = (uint32_t)(Lf * d_e) >> 3;        // one expert further, in 16 bytes
   // (several token groups) token rows 8 n + g of an h tile in shared memory (rows beyond the
   // chunk hold whatever the buffer held: their columns of the result are dropped)
   const uint32_t hs_off = h_off + (g >> 1) * drow + (g & 1) * half_h + 16 * tg;
@@ -442,7 +448,7 @@ __global__ void __launch_bounds__(kThreads, 1) expert_wide_kernel(const LeanPara
               const float4* part = reinterpret_cast<const float4*>(part0 + (t * (16 * NC) + m) * kWarps);
               const float4 lo = part[0], hi = part[1];
               float v = ((lo.x + lo.y) + (lo.z + lo.w)) + ((hi.x + hi.y) + (hi.z + hi.w));
-              const int o = t * d + c0 + m;
+              const int o = (tok0 + t) * d + c0 + m;
               if (p.accumulate) v += __ldcg(p.out + o);
               p.out[o] = v;
               if (p.x_next) p.x_next[o] = (uint16_t)f32_to_bf16_bits(v);
@@ -453,7 +459,7 @@ __global__ void __launch_bounds__(kThreads, 1) expert_wide_kernel(const LeanPara
     } else {                       // empty union: FFN(x) = 0
       for (int t = ot; t < L; t += 8) {
         for (int m = om; m < ncols; m += 32) {
-          const int o = t * d + c0 + m;
+          const int o = (tok0 + t) * d + c0 + m;
           const float v = p.accumulate ? __ldcg(p.out + o) : 0.0f;
           p.out[o] = v;
           if (p.x_next) p.x_next[o] = (uint16_t)f32_to_bf16_bits(v);
@@ -462,11 +468,11 @@ __global__ void __launch_bounds__(kThreads, 1) expert_wide_kernel(const LeanPara
     }
   }
   // CTA 0 publishes the routing it derived (after the wait: earlier readers are done)
-  if (blockIdx.x == 0) {
+  if (blockIdx.x == 0 && blockIdx.y == 0) {
     if (p.lg.a0 != nullptr && p.pub_scores != nullptr) {
       const int words = (p.E + 31) >> 5;
       const float* rinv = reinterpret_cast<const float*>(ctl + 104);
-      for (int t = warp; t < L; t += kWarps) {
+      for (int t = warp; t < Lf; t += kWarps) {
         for (int w = 0; w < words; ++w) {
           const int e = 32 * w + lane;
           float sv = 0.0f;
@@ -492,7 +498,7 @@ __global__ void __launch_bounds__(kThreads, 1) expert_wide_kernel(const LeanPara
         if (p.pub_n) *p.pub_n = nu;
         if (p.stats) {
           atomicAdd(reinterpret_cast<unsigned long long*>(&p.stats->n_tokens),
-                    (unsigned long long)L);
+                    (unsigned long long)Lf);
           atomicAdd(reinterpret_cast<unsigned long long*>(&p.stats->n_active),
                     (unsigned long long)ctl[2]);
           atomicAdd(reinterpret_cast<unsigned long long*>(&p.stats->n_chunks), 1ull);

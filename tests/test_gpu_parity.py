@@ -213,6 +213,26 @@ def test_expert_ffn_under_call_promises(kind, d, E, d_e, L, p):
     assert layer.last_status() == 0
 
 
+@pytest.mark.parametrize("L", [8, 16, 32])
+def test_stable_x_calls_that_keep_the_whole_device(L):
+    """BLOCKFFN_CFG_NO_SPLIT: calls with stable x get all SMs each. A chunk of more than 16 tokens
+    would then need two CTAs per SM resident at once for its hand-over; where the shared memory
+    of the shape does not allow that the library must take the two-kernel form instead of
+    waiting for CTAs that cannot start."""
+    sh, seed = I.SHAPES[2], I.config_seed(2)
+    w = I.make_layer(sh, seed, with_router=False)
+    layer = B.Layer(sh.d, sh.E, sh.d_e, L_max=32, flags=B.CFG_NO_SPLIT)
+    dw = layer.upload_weights(w)
+    for chunk in range(3):
+        x = I.make_x(sh.d, L, seed, chunk=chunk)
+        s = I.make_scores(sh.E, L, sh.u, seed, chunk=chunk)
+        ref = oracle.layer_forward_scores(x, s, w["U"], w["D"], union_only=True)
+        res = layer.forward_scores(dw, B.to_device_bf16(x), dev(s), call_flags=B.CALL_INDEPENDENT_X)
+        torch.cuda.synchronize()
+        assert layer.last_status() == 0
+        assert_close(res.out.cpu().numpy(), ref.out, f"no split, L={L}")
+
+
 @pytest.mark.parametrize("variant", VARIANTS)
 @pytest.mark.parametrize("d,E,d_e,L", [(512, 24, 64, 6), (2048, 64, 128, 8), (1536, 48, 128, 19)])
 def test_expert_ffn_signed_and_nan_scores(variant, d, E, d_e, L):
