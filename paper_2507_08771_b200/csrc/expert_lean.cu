@@ -1,30 +1,36 @@
-// Expert stage (Eq. 1, Eq. 2 restricted to Union(x), Sec. 3.3) for chunks of at most 8 tokens:
-// one kernel per call, several calls in flight per SM.
+// Expert stage (Eq. 1, Eq. 2 restricted to Union(x), Sec. 3.3) as one kernel per call, for
+// calls whose inputs are all stable (x included), so that several calls are in flight per SM.
+// expert_lean_kernel takes chunks of up to 8 tokens, expert_wide_kernel (expert_wide.cuh) chunks
+// of 9 to 32.
 //
 // A call lasts a few microseconds, most of which is memory latency: the routing inputs, then
 // the weights they select, then the intermediate every CTA needs from every other. What the
 // device sustains is therefore set by how many calls are in flight per SM, i.e. by how little
-// shared memory and how few registers one CTA holds. This kernel keeps only the weights in
-// shared memory; the small operands (x for the up projection, the intermediate h for the
-// down projection) go from L2 straight into the registers of the one warp that uses them:
-// with K split over the warps no two warps read the same element, so a shared tile would
-// only be a detour. Three CTAs (three successive calls) then fit one SM at d = 2048.
+// shared memory and how few registers one CTA holds, and by how few instructions and bytes from
+// L2 a call spends next to its weight stream. This kernel keeps only the weights in shared
+// memory; the small operands (x for the up projection, the intermediate h for the down
+// projection) go from L2 straight into the registers of the one warp that uses them: with K
+// split over the warps no two warps read the same element, so a shared tile would only be a
+// detour. Three CTAs (of three different calls) fit one SM, and a call runs on a third of the
+// SMs (see lean_plan), so that nine calls are in flight.
 //
 //   CTA b, call n:
-//     ticket           one atomic per CTA on the handle's call counter; ticket / grid is the
-//                      call's index n (all CTAs of a call take theirs before any CTA of the next
-//                      call exists, see below), n mod 16 its slot in the ring of h buffers
-//     Union(x)         derived by every CTA from the scores, the caller's list or raw logits
+//     ticket           one atomic per CTA on the ring's call counter; ticket / CTAs per call is
+//                      the call's index n (all CTAs of a call take theirs before any CTA of the
+//                      next call exists, see below), n mod 16 its slot in the ring of h buffers
+//     Union(x)         derived by every CTA from the scores, the caller's list or raw logits;
+//                      thread 0 releases the dependent launch while those loads are in flight
 //     up projection    the CTA's share of the union's neuron rows -> shared memory (16-byte
-//                      asynchronous copies), K split over the 8 warps, mma.sync m16n8k16 with
-//                      the weights as the M operand and the tokens as N, cross-warp sum, Swish,
-//                      router score, bf16 -> h ring slot (global, L2)
+//                      asynchronous copies, in stages when the share exceeds the region), K split
+//                      over the 8 warps, mma.sync m16n8k16 with the weights as the M operand and
+//                      the tokens as N, cross-warp sum, Swish, router score, bf16 -> h ring slot
+//                      (global, L2)
 //     hand-over        one arrival per CTA on the slot's counter (after a fence); the D slabs of
 //                      the CTA's output columns are requested into the same shared memory; then
 //                      one thread polls the counter until all CTAs of the call have arrived
 //                      (bounded: BLOCKFFN_DEV_WAIT_EXPIRED) and the warps fetch their h fragments
-//     down projection  out[t][c] over all union experts for the CTA's <= 16 columns, one writer
-//                      per element, fixed summation order
+//     down projection  out[t][c] over all union experts for the CTA's columns (up to three tiles
+//                      of 16), one writer per element, fixed summation order
 //     griddepcontrol.wait before out is touched (and before the kernel ends)
 //
 // Ordering between calls. Kernels are chained by programmatic dependent launch and trigger
@@ -32,12 +38,15 @@
 // interleave. Every kernel waits for its predecessor before it ends, so no CTA of a call exits
 // while an earlier call is incomplete: when a CTA of call n + R exists and call n is incomplete,
 // all CTAs of calls n + 1 .. n + R - 1 are resident, plus one of each end, i.e.
-// (R - 1) grid + 2 <= 3 SMs CTAs (the kernel is compiled for three CTAs per SM). With a grid of
-// a third of the SMs (calls that share the device) that allows R <= 9; the ring has 16 slots,
-// so a slot is never reused while a CTA of its earlier call is alive, and its arrival counter is
-// an exact multiple of the grid size when a call starts: the counters only ever grow, nothing is
-// reset, graph replays need no host state. Calls that own the device and calls that share it
-// have grids of different size and therefore a ring and a ticket counter each.
+// (R - 1) grid + 2 <= 3 SMs CTAs (at most three CTAs fit one SM: every launch asks for more than
+// a quarter of its shared memory). With a grid of a third of the SMs that allows R <= 9; the
+// ring has 16 slots, so a slot is never reused while a CTA of its earlier call is alive, and
+// its arrival counter is an exact multiple of the call's CTA count when a call starts: the
+// counters only ever grow, nothing is reset, graph replays need no host state. A ticket
+// identifies a call only if every call drawing from the counter has the same number of CTAs, so
+// each kind of call (whole device; a third of it; a third of it in two token slices) has a ring
+// and a counter of its own. The hand-over also needs all CTAs of a call resident at once:
+// lean_plan refuses grids for which that is not guaranteed.
 // The polling thread issues no asynchronous copies: a fence or an acquire by a thread waits
 // for that thread's own copies in flight.
 #include "mma_tiles.cuh"
