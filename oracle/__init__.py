@@ -80,6 +80,35 @@ def router(x, W_r, gain, bias=None, eps=1e-6):
     return a0, s
 
 
+def router_relu_only(x, W_r, bias=None):
+    """Sec. 4.2.3 ablation: the router without RMSNorm, scores = ReLU(W_router^T x).
+
+    Returns (a0, scores), float64 [L][E]."""
+    x, W_r, bias = _u16(x), _u16(W_r), _f32(bias)
+    L, d = x.shape
+    E = W_r.shape[0]
+    assert W_r.shape == (E, d)
+    a0 = np.empty((L, E), np.float64)
+    s = np.empty((L, E), np.float64)
+    _load().oracle_router_relu_only(_p(x, ctypes.c_uint16), _p(W_r, ctypes.c_uint16),
+                                    _p(bias, ctypes.c_float), L, d, E, _p(a0, ctypes.c_double),
+                                    _p(s, ctypes.c_double))
+    return a0, s
+
+
+def reuse_ratio(scores, acc=None):
+    """Sec. 4.1.2: adds the sum of |S_i n S_{i+1}| / |S_i| over the successive token pairs of one
+    sequence to acc[0] and the number of pairs counted to acc[1] (float64[2], created when None).
+    The sequence's reuse ratio is acc[0] / acc[1]."""
+    scores = np.ascontiguousarray(scores, dtype=np.float64)
+    L, E = scores.shape
+    if acc is None:
+        acc = np.zeros(2, np.float64)
+    assert acc.dtype == np.float64 and acc.shape == (2,)
+    _load().oracle_reuse_ratio(_p(scores, ctypes.c_double), L, E, _p(acc, ctypes.c_double))
+    return acc
+
+
 def token_masks(scores):
     """Sec. 3.3 sparse pattern of A(x): bit i of row t set iff scores[t, i] != 0."""
     scores = np.ascontiguousarray(scores, dtype=np.float64)
@@ -169,8 +198,15 @@ def layer_forward_scores(x, scores_f32, U, D, union_only=False, stats=None) -> L
 
 
 def layer_forward(x, W_r, gain, U, D, bias=None, eps=1e-6, union_only=False,
-                  stats=None) -> LayerResult:
-    """Full layer: Eq. 3 router -> Union(x) -> Eq. 1/2."""
+                  stats=None, rmsnorm=True) -> LayerResult:
+    """Full layer: Eq. 3 router -> Union(x) -> Eq. 1/2. rmsnorm=False takes the router of the
+    Sec. 4.2.3 ablation instead (gain and eps unused), step by step through the same routines."""
+    if not rmsnorm:
+        a0, s = router_relu_only(x, W_r, bias)
+        tm = token_masks(s)
+        um, ids, n = chunk_union(tm, W_r.shape[0], stats)
+        out = expert_ffn(x, s, U, D, expert_ids=ids[:n] if union_only else None)
+        return LayerResult(a0, s, tm, um, ids, n, out)
     x, W_r, U, D = _u16(x), _u16(W_r), _u16(U), _u16(D)
     gain, bias = _f32(gain), _f32(bias)
     L, d = x.shape

@@ -31,7 +31,11 @@
  *     value (-0.0 is zero, NaN counts as nonzero);
  *   - the score multiplies the activated intermediate, before the down
  *     projection;
- *   - the union id list is in ascending expert order.
+ *   - the union id list is in ascending expert order;
+ *   - the router without RMSNorm (Sec. 4.2.3) has no gain either: its scores are
+ *     the ReLU of the logits;
+ *   - the reuse ratio (Sec. 4.1.2) leaves out a pair whose first token activates
+ *     no expert (its ratio is 0/0).
  * "parity unpinned" (no independent source fixes them): the eps value, beta = 1,
  * the place where the score multiplies. Everything else is pinned by the CPU
  * tests (brute force, closed forms, library reductions, invariants).
@@ -84,6 +88,21 @@ ORACLE_API void oracle_router(const uint16_t* x, const uint16_t* W_r, const floa
   free(a1);
 }
 
+/* The router of the RMSNorm ablation (Sec. 4.2.3, the ReMoE-style router of Table 1): the
+ * activation values are the ReLU of the logits themselves, A = ReLU(W_router^T x); no
+ * normalisation, hence no gain and no eps. */
+ORACLE_API void oracle_router_relu_only(const uint16_t* x, const uint16_t* W_r, const float* bias,
+                                        int L, int d, int E, double* a0, double* scores) {
+  for (int t = 0; t < L; ++t)
+    for (int i = 0; i < E; ++i) {
+      double acc = bias ? (double)bias[i] : 0.0;
+      for (int k = 0; k < d; ++k)
+        acc += widen_bf16(x[(size_t)t * d + k]) * widen_bf16(W_r[(size_t)i * d + k]);
+      if (a0) a0[(size_t)t * E + i] = acc;
+      scores[(size_t)t * E + i] = acc > 0.0 ? acc : 0.0;
+    }
+}
+
 /* The sparse pattern of A(x) (Sec. 3.3): bit i of token t's mask is set iff the
  * score is nonzero. Bits at and beyond E are zero. */
 ORACLE_API void oracle_token_masks(const double* scores, int L, int E, uint32_t* tok_mask) {
@@ -131,6 +150,25 @@ ORACLE_API double oracle_tls(const uint64_t* stats, int E) {
 }
 ORACLE_API double oracle_cls(const uint64_t* stats, int E) {
   return 1.0 - (double)stats[3] / ((double)stats[2] * (double)E);
+}
+
+/* Reuse ratio (Sec. 4.1.2): with S_i the experts token i of a sequence activates, the ratio of
+ * the sequence is the mean over its L - 1 successive pairs of |S_i n S_{i+1}| / |S_i|.
+ * acc[0] += the sum of the pairs' ratios, in token order; acc[1] += the number of pairs
+ * counted. A token that activates no expert has no ratio: its pair is left out of both. */
+ORACLE_API void oracle_reuse_ratio(const double* scores, int L, int E, double* acc) {
+  for (int i = 0; i + 1 < L; ++i) {
+    int n_i = 0, n_both = 0;
+    for (int e = 0; e < E; ++e) {
+      int now = scores[(size_t)i * E + e] != 0.0;
+      int next = scores[(size_t)(i + 1) * E + e] != 0.0;
+      n_i += now;
+      n_both += now && next;
+    }
+    if (n_i == 0) continue;
+    acc[0] += (double)n_both / (double)n_i;
+    acc[1] += 1.0;
+  }
 }
 
 /* Eq. 1 with Eq. 2:  out[t] = sum_i A_i(x_t) * W_down^(i)T Swish(W_up^(i)T x_t).

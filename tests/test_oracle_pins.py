@@ -381,6 +381,122 @@ def test_scores_in_layer_matches_pieces():
     assert np.array_equal(r.out, oracle.expert_ffn(x, sc.astype(np.float64), w["U"], w["D"]))
 
 
+
+
+# ----------------------------------------------------------------------------
+# router without RMSNorm (Sec. 4.2.3) and the reuse ratio (Sec. 4.1.2)
+# ----------------------------------------------------------------------------
+@pytest.mark.parametrize("L,d,E,with_bias", [(2, 5, 3, False), (3, 7, 6, True)])
+def test_router_relu_only_brute_force_and_library(L, d, E, with_bias):
+    rng = np.random.default_rng(40 + E)
+    xb, Wb = bf(rng.standard_normal((L, d))), bf(rng.standard_normal((E, d)))
+    bias = rng.standard_normal(E).astype(np.float32) if with_bias else None
+    a0, s = oracle.router_relu_only(xb, Wb, bias)
+    for t in range(L):                                    # brute force, plain Python floats
+        for i in range(E):
+            acc = 0.0 if bias is None else float(bias[i])
+            for k in range(d):
+                acc += float(wide(xb)[t][k]) * float(wide(Wb)[i][k])
+            assert a0[t, i] == pytest.approx(acc, rel=1e-13, abs=1e-13)
+            assert s[t, i] == pytest.approx(max(acc, 0.0), rel=1e-13, abs=1e-13)
+    tb = None if bias is None else torch.from_numpy(bias.astype(np.float64))
+    ts = torch.relu(torch.nn.functional.linear(torch.from_numpy(wide(xb)), torch.from_numpy(wide(Wb)), tb))
+    np.testing.assert_allclose(s, ts.numpy(), rtol=1e-12, atol=1e-13)
+    assert (s >= 0).all() and ((s == 0) == (a0 <= 0)).all()
+
+
+def test_router_relu_only_is_the_router_with_the_norm_taken_out():
+    # Eq. 3 = RMSNorm applied to exactly these values: dividing the normalised scores by the
+    # gain and multiplying the root mean square back must return them, and both share one mask
+    rng = np.random.default_rng(41)
+    L, d, E, eps = 4, 48, 20, 1e-6
+    xb, Wb = bf(rng.standard_normal((L, d))), bf(rng.standard_normal((E, d)) / math.sqrt(d))
+    gain = rng.uniform(0.5, 1.5, E).astype(np.float32)
+    a0n, sn = oracle.router(xb, Wb, gain, None, eps=eps)
+    a0p, sp = oracle.router_relu_only(xb, Wb, None)
+    np.testing.assert_array_equal(a0n, a0p)
+    rms_ = np.sqrt((sp ** 2).mean(axis=1, keepdims=True) + eps)
+    np.testing.assert_allclose(sn / gain.astype(np.float64) * rms_, sp, rtol=1e-13, atol=1e-15)
+    assert ((sn != 0) == (sp != 0)).all()
+    # positive homogeneity, which the normalised router does not have: doubling x doubles A
+    _, s2 = oracle.router_relu_only(bf(2.0 * wide(xb)), Wb, None)
+    np.testing.assert_allclose(s2, 2.0 * sp, rtol=1e-13)
+
+
+def test_layer_without_rmsnorm_is_the_composition():
+    rng, x, U, D, _ = _small_problem(11)
+    E, d = U.shape[0], x.shape[1]
+    Wb = bf(rng.standard_normal((E, d)) / math.sqrt(d))
+    bias = np.full(E, -0.5, np.float32)
+    res = oracle.layer_forward(x, Wb, None, U, D, bias=bias, union_only=True, rmsnorm=False)
+    a0, sp = oracle.router_relu_only(x, Wb, bias)
+    np.testing.assert_array_equal(res.scores, sp)
+    np.testing.assert_array_equal(res.tok_mask, oracle.token_masks(sp))
+    np.testing.assert_allclose(res.out, oracle.expert_ffn(x, sp, U, D), rtol=1e-12, atol=1e-14)
+    assert 0 < res.n_union <= E
+
+
+def brute_reuse(active_sets):
+    total, pairs = 0.0, 0
+    for a, b in zip(active_sets[:-1], active_sets[1:]):
+        if a:
+            total += len(a & b) / len(a)
+            pairs += 1
+    return total, pairs
+
+
+@pytest.mark.parametrize("L,E,p", [(2, 5, 0.5), (7, 40, 0.3), (32, 33, 0.2), (12, 64, 0.05), (1, 8, 0.5)])
+def test_reuse_ratio_brute_force_with_sets(L, E, p):
+    rng = np.random.default_rng(50 + L)
+    s = sparse_scores(rng, L, E, p)
+    sets = [set(np.nonzero(s[t])[0].tolist()) for t in range(L)]
+    want, pairs = brute_reuse(sets)
+    acc = oracle.reuse_ratio(s)
+    assert acc[1] == pairs
+    assert acc[0] == pytest.approx(want, rel=1e-14, abs=0)
+    # accumulates over calls (one sequence each)
+    acc2 = oracle.reuse_ratio(s, acc.copy())
+    assert acc2[1] == 2 * pairs and acc2[0] == pytest.approx(2 * want, rel=1e-14)
+
+
+def test_reuse_ratio_closed_forms():
+    E = 16
+    row = np.zeros(E); row[[1, 4, 9, 10]] = [0.5, -2.0, 1.0, 3.0]       # sign does not matter
+    same = np.tile(row, (6, 1))
+    acc = oracle.reuse_ratio(same)
+    assert acc.tolist() == [5.0, 5.0]                                   # identical tokens: ratio 1
+    other = np.zeros(E); other[[0, 2, 3]] = 1.0
+    alt = np.stack([row, other, row, other])
+    assert oracle.reuse_ratio(alt).tolist() == [0.0, 3.0]               # disjoint neighbours: ratio 0
+    # nested shrinking sets S_{i+1} within S_i: each ratio is |S_{i+1}| / |S_i|; not symmetric
+    a = np.zeros(E); a[:8] = 1.0
+    b = np.zeros(E); b[:2] = 1.0
+    assert oracle.reuse_ratio(np.stack([a, b]))[0] == 0.25
+    assert oracle.reuse_ratio(np.stack([b, a]))[0] == 1.0
+    # a token with no active expert has no ratio: the pair it starts is left out, the pair it
+    # ends counts with ratio 0
+    z = np.zeros(E)
+    assert oracle.reuse_ratio(np.stack([a, z, a])).tolist() == [0.0, 1.0]
+    assert oracle.reuse_ratio(np.stack([a])).tolist() == [0.0, 0.0]     # L = 1: no pair
+    # -0.0 is inactive, NaN is active (by value, as for the masks)
+    c = np.zeros(E); c[0] = -0.0; c[1] = np.nan
+    n = np.zeros(E); n[1] = 1.0
+    assert oracle.reuse_ratio(np.stack([c, n])).tolist() == [1.0, 1.0]
+
+
+def test_reuse_ratio_agrees_with_the_token_masks():
+    rng = np.random.default_rng(60)
+    L, E = 16, 70
+    s = sparse_scores(rng, L, E, 0.25)
+    tm = oracle.token_masks(s)
+    total = 0.0
+    for i in range(L - 1):
+        n_i = sum(bin(int(w)).count("1") for w in tm[i])
+        both = sum(bin(int(a & b)).count("1") for a, b in zip(tm[i], tm[i + 1]))
+        total += both / n_i
+    assert oracle.reuse_ratio(s)[0] == pytest.approx(total, rel=1e-14)
+
+
 def test_residual_step():
     rng = np.random.default_rng(5)
     res = rng.standard_normal((3, 16))
