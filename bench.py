@@ -746,6 +746,50 @@ def read_ceilings(args, torch, device, B):
     return out
 
 
+def stack_router_on(args, torch, device, peak, layers=None, chunks=16):
+    from paper_2507_08771_b200 import binding as B
+    sh = I.SHAPES[4]
+    layers = layers or I.STACK_LAYERS
+    seed = I.config_seed(4)
+    lay = B.Layer(sh.d, sh.E, sh.d_e, L_max=sh.L, device=device, flags=args.flags)
+    w = I.make_layer(sh, seed, bias_shift=I.ROUTER_BIAS_SHIFT)
+    # residual-branch scale 1/32 (exact in bf16): the running hidden state then stays near unit
+    # scale over the stack, and with it the sparsity the fixed router bias gives
+    w["D"] = I.f32_to_bf16_bits(I.bf16_bits_to_f32(w["D"]) * np.float32(1.0 / 32.0))
+    first = lay.upload_weights(w)
+    dws = [first]
+    for _ in range(layers - 1):
+        t = {k: v.clone() for k, v in first.tensors.items()}
+        dws.append(B.DeviceWeights(B.make_weights(t["W_r"], t["gain"], t["bias"], t["U"], t["D"]), t))
+    # no normalisation of the hidden state sits between the layers (it is not part of this path):
+    # the router sees x ~ N(0,1) at the first layer and the running residual after it
+    xs = np.stack([I.make_correlated_x(sh.d, sh.L, 0.96, seed, chunk=c) for c in range(chunks)])
+    x0 = torch.from_numpy(xs.view(np.int16)).to(device).view(torch.bfloat16)
+    res = torch.zeros(chunks, sh.L, sh.d, dtype=torch.float32, device=device)
+    xpp = torch.zeros(2, sh.L, sh.d, dtype=torch.bfloat16, device=device)
+
+    def enqueue(stream):
+        for c in range(chunks):
+            res[c].copy_(x0[c])
+            xpp[0].copy_(x0[c])
+            for l in range(layers):
+                B.blockffn_layer_forward(lay.h, dws[l].struct, xpp[l % 2], sh.L, res[c], xpp[(l + 1) % 2],
+                                         lay.stats, B.CALL_ACCUMULATE, stream)
+
+    stream = torch.cuda.Stream(device)
+    g = capture(torch, stream, enqueue)
+    ms = time_replays(torch, stream, g, max(3, args.steps // 2), 2)
+    assert lay.last_status() == 0
+    hs = lay.stats_host()
+    mean_u = (1.0 - B.blockffn_cls(hs, sh.E)) * sh.E
+    us_layer = ms * 1e3 / (chunks * layers)
+    return {"layers": layers, "chunks": chunks, "us_per_layer": us_layer, "mean_union": mean_u,
+            "tls": B.blockffn_tls(hs, sh.E), "GBps": mean_u * sh.expert_bytes / us_layer / 1e3,
+            "note": "router on every layer (3 launches per layer: router, up, down); no normalisation between "
+                    "layers, down projections scaled by 1/32 so that the hidden state keeps its scale; the union "
+                    "is whatever the router derives (mean reported)"}
+
+
 def extras(args, torch, device, peak):
     """The other configurations, each as us per call and GB/s of active expert bytes."""
     from paper_2507_08771_b200 import binding as B
@@ -765,8 +809,6 @@ def extras(args, torch, device, peak):
         row = {"L": L}
         for name, variant, form in (("tensor_core", 0, 0), ("tensor_core_pair", 0, B.CFG_TWO_KERNELS),
                                     ("cuda_core", 1, 0)):
-            if name == "tensor_core_pair" and L > 8:
-                continue                    # chunks longer than 8 tokens already run as the pair
             wl = Workload(2, L, chunks, variant, device, args.flags | form)
             us = timed(wl) * 1e3 / wl.calls_per_step
             hs = wl.layer.stats_host()
@@ -799,9 +841,17 @@ def extras(args, torch, device, peak):
         tls, ufrac = wl.sparsity()
         us = ms * 1e3 / chunks
         mean_u = ufrac * sh.E
+        # reuse ratio between successive tokens of a chunk (Sec. 4.1.2), from the scores each of
+        # the first 16 layer calls leaves in the handle; untimed
+        reuse = torch.zeros(2, dtype=torch.float64, device=device)
+        for c in range(min(16, chunks)):
+            B.blockffn_layer_forward(wl.layer.h, wl.dws[0].struct, wl.x[c], sh.L, wl.out[c], None, None, 0)
+            B.blockffn_reuse_ratio(wl.layer.h, None, sh.L, reuse)
+        rr = reuse.cpu().numpy()
         full[name] = {"rho": r, "us_per_call": us, "tls": tls, "mean_union": mean_u,
                       "GBps": mean_u * sh.expert_bytes / us / 1e3,
-                      "launches_per_call": 2}
+                      "launches_per_call": 2,
+                      "reuse_ratio": float(rr[0] / rr[1]) if rr[1] > 0 else None}
         if r is None:                   # stage level: the router entry point from its own graph
             st2 = torch.cuda.Stream(device)
             g2 = capture(torch, st2, wl.enqueue_router_only)
@@ -857,6 +907,11 @@ def extras(args, torch, device, peak):
         del wl
         torch.cuda.empty_cache()
     out["paper_2p8b_shape"] = rows
+
+    # config 4 with the router on: every layer computes its own scores from the running hidden
+    # state (blockffn_layer_forward, Eq. 3 -> Union -> Eq. 1/2), residual and bf16 hand-over as
+    # in the scores-in stack. One layer's weights (router included) at 24 distinct addresses.
+    out["config4_stack_router_on"] = stack_router_on(args, torch, device, peak)
 
     # config 4: 24-layer stack, residual between layers
     wl = Workload(4, None, min(args.chunks, I.STACK_CHUNKS), 0, device, args.flags)

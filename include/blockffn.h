@@ -73,20 +73,26 @@ typedef struct {
   int32_t E;       /* number of experts N_e                                    */
   int32_t d_e;     /* expert width                                             */
   int32_t L_max;   /* largest chunk length a call may pass (<= 32)             */
-  float rms_eps;   /* RMSNorm epsilon, added to the mean square (Eq. 3); 1e-6  */
+  float rms_eps;   /* RMSNorm epsilon, added to the mean square (Eq. 3); 1e-6;
+                      BLOCKFFN_NO_RMSNORM: the router of the Sec. 4.2.3 ablation  */
   int32_t variant; /* BLOCKFFN_VARIANT_*                                       */
   int32_t flags;   /* tuning, 0 = defaults: bits 0-7 ring depth of the up-projection
                       kernel, bits 8-15 of the down-projection kernel (stages of shared
                       memory, 0 = chosen from the shape), BLOCKFFN_CFG_* bits        */
 } blockffn_config;
 
+/* rms_eps value that takes RMSNorm out of the router (the ablation of Sec. 4.2.3, the
+ * ReMoE-style router of Table 1): scores = ReLU(W_router^T x + bias), no normalisation and no
+ * gain (blockffn_weights.gain is not read and may be NULL). Every other rms_eps must be >= 0. */
+#define BLOCKFFN_NO_RMSNORM (-1.0f)
+
 /* The tensor-core kernels are normally launched so that a kernel may start fetching its
  * weights while the kernel enqueued before it on the stream is still finishing
  * (programmatic dependent launch); this bit launches them fully serialised instead. */
 #define BLOCKFFN_CFG_NO_CHAINING 0x10000
-/* Chunks of at most 8 tokens normally run as one kernel per call, several calls in flight per
- * SM; this bit selects the older two-kernel form (up projection, down projection) for them
- * too. Same results within the tolerance; kept for comparison and as the path of longer chunks. */
+/* A call whose x is stable normally runs as one kernel, several calls in flight per SM; this
+ * bit selects the two-kernel form (up projection, down projection), the form every other call
+ * takes, for those calls too. Same results within the tolerance; kept for comparison.        */
 #define BLOCKFFN_CFG_TWO_KERNELS 0x20000000
 /* The one-kernel form runs a call whose x is promised stable (BLOCKFFN_CALL_INDEPENDENT_X) on
  * a third of the SMs, so that three times as many such calls are in flight: every CTA reads all
@@ -223,6 +229,20 @@ BLOCKFFN_API blockffn_status blockffn_last_status(blockffn_handle h, uint32_t* b
  * CLS_L = 1 - n_union / (n_chunks E) with L the chunk length of the calls counted.      */
 BLOCKFFN_API double blockffn_tls(const blockffn_stats* host_stats, int32_t E);
 BLOCKFFN_API double blockffn_cls(const blockffn_stats* host_stats, int32_t E);
+
+/* Reuse ratio between successive tokens (Sec. 4.1.2). With S_i the experts token i of a
+ * sequence activates (nonzero score, by value), adds to reuse[0] the ratios
+ * |S_i n S_{i+1}| / |S_i| of the sequence's L - 1 successive pairs, one after the other in
+ * token order, and to reuse[1] the number of pairs counted; a pair whose first token activates
+ * no expert has no ratio and is left out of both. The sequence's (or, over many calls, the
+ * average) reuse ratio is reuse[0] / reuse[1].
+ * scores: f32 [L][E], device; NULL = the scores the last router-on layer call on this handle
+ * left in its workspace (then L <= L_max). L >= 1 is otherwise not limited by L_max: a
+ * sequence is not a chunk. reuse: f64 [2], device, 8-byte aligned, caller-owned and zeroed
+ * by the caller; calls that share it must be ordered (one stream).
+ * Errors: INVALID_ARG (NULL or misaligned pointer, L < 1, scores NULL with L > L_max).      */
+BLOCKFFN_API blockffn_status blockffn_reuse_ratio(blockffn_handle h, const float* scores,
+                                                  int32_t L, double* reuse, void* stream);
 
 /* Number of kernels the library has launched through this handle (host counter). */
 BLOCKFFN_API uint64_t blockffn_launch_count(blockffn_handle h);

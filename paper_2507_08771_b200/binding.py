@@ -27,6 +27,7 @@ CFG_NO_CHAINING = 0x10000
 CFG_TWO_KERNELS = 0x20000000
 CFG_TEST_EXPIRE_WAIT = 0x10000000
 CFG_NO_SPLIT = 0x40000000
+NO_RMSNORM = -1.0        # rms_eps value: the router without RMSNorm (Sec. 4.2.3)
 
 
 def cfg_expected_union(u: int) -> int:
@@ -38,6 +39,7 @@ EXPORTS = [
     "blockffn_expert_ffn", "blockffn_layer_forward", "blockffn_layer_forward_scores",
     "blockffn_read_routing", "blockffn_last_status", "blockffn_tls", "blockffn_cls",
     "blockffn_launch_count", "blockffn_status_string", "blockffn_expert_ffn_noalloc",
+    "blockffn_reuse_ratio",
 ]
 NOALLOC_SCRATCH_BYTES = 1 << 20
 
@@ -91,6 +93,7 @@ def load():
     lib.blockffn_tls.restype = ctypes.c_double
     lib.blockffn_cls.argtypes = [ctypes.POINTER(Stats), i32]
     lib.blockffn_cls.restype = ctypes.c_double
+    lib.blockffn_reuse_ratio.argtypes = [vp, vp, i32, vp, vp]
     lib.blockffn_launch_count.argtypes = [vp]
     lib.blockffn_launch_count.restype = ctypes.c_uint64
     lib.blockffn_status_string.argtypes = [i32]
@@ -189,6 +192,11 @@ def blockffn_read_routing(h, L, scores=None, tok_mask=None, union_mask=None, uni
     _check(load().blockffn_read_routing(h, L, _ptr(scores), _ptr(tok_mask), _ptr(union_mask),
                                         _ptr(union_ids), _ptr(n_union), _stream(stream)),
            "blockffn_read_routing")
+
+
+def blockffn_reuse_ratio(h, scores, L, reuse, stream=None):
+    _check(load().blockffn_reuse_ratio(h, _ptr(scores), L, _ptr(reuse), _stream(stream)),
+           "blockffn_reuse_ratio")
 
 
 def blockffn_last_status(h, clear=False, stream=None) -> int:

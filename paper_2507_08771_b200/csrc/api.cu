@@ -1,5 +1,6 @@
 // C ABI of the BlockFFN library: argument checks, workspace, dispatch.
 #include <new>
+#include <vector>
 
 #include "common.cuh"
 
@@ -89,7 +90,7 @@ blockffn_status blockffn_create(const blockffn_config* cfg, blockffn_handle* out
   if (cfg->d % 8 || cfg->d_e % 8 || cfg->E > 1024 || cfg->L_max > 32 || cfg->d > (1 << 20) ||
       cfg->d_e > (1 << 16))
     return BLOCKFFN_ERR_UNSUPPORTED;
-  if (!(cfg->rms_eps >= 0.0f)) return BLOCKFFN_ERR_INVALID_ARG;
+  if (!(cfg->rms_eps >= 0.0f) && cfg->rms_eps != BLOCKFFN_NO_RMSNORM) return BLOCKFFN_ERR_INVALID_ARG;
   if (cfg->variant < BLOCKFFN_VARIANT_AUTO || cfg->variant > BLOCKFFN_VARIANT_MMA)
     return BLOCKFFN_ERR_INVALID_ARG;
   if (cfg->flags & ~0x7fffffff) return BLOCKFFN_ERR_INVALID_ARG;
@@ -125,6 +126,7 @@ blockffn_status blockffn_create(const blockffn_config* cfg, blockffn_handle* out
   const size_t lean_bytes = expert_lean_ws_bytes(cfg, c->num_sms);
   const size_t o_lean = take(lean_bytes);
   const size_t o_seq = take(sizeof(unsigned long long) * 96);
+  const size_t o_one = take(sizeof(float) * E);
   const size_t o_tk = take(sizeof(unsigned int) * 8);
   const size_t o_st = take(sizeof(uint32_t));
   void* base = nullptr;
@@ -152,8 +154,17 @@ blockffn_status blockffn_create(const blockffn_config* cfg, blockffn_handle* out
   c->h16 = b + o_h16;
   c->lean_ring = lean_bytes ? b + o_lean : nullptr;
   c->lean_seq = reinterpret_cast<unsigned long long*>(b + o_seq);
+  c->ones = reinterpret_cast<float*>(b + o_one);
   c->ticket = reinterpret_cast<unsigned int*>(b + o_tk);
   c->status = reinterpret_cast<uint32_t*>(b + o_st);
+  {
+    const std::vector<float> ones(E, 1.0f);
+    if (cudaMemcpy(c->ones, ones.data(), sizeof(float) * E, cudaMemcpyHostToDevice) != cudaSuccess) {
+      cudaFree(base);
+      delete c;
+      return BLOCKFFN_ERR_CUDA;
+    }
+  }
   if (expert_mma_setup(c) != cudaSuccess || expert_lean_setup(c) != cudaSuccess) {
     cudaFree(base);
     delete c;
@@ -199,7 +210,7 @@ blockffn_status blockffn_router(blockffn_handle h, const blockffn_weights* w, co
                                 int32_t L, float* scores, uint32_t* tok_mask, void* stream) {
   blockffn_status s = check_call(h, L);
   if (s != BLOCKFFN_OK) return s;
-  if (!w || !w->W_r || !w->gain || !x || !scores) return BLOCKFFN_ERR_INVALID_ARG;
+  if (!w || !w->W_r || (!w->gain && !no_rmsnorm(h)) || !x || !scores) return BLOCKFFN_ERR_INVALID_ARG;
   if (misaligned(w->W_r) || misaligned(x) || misaligned(scores) ||
       (reinterpret_cast<uintptr_t>(w->gain) & 3u) || (reinterpret_cast<uintptr_t>(w->bias) & 3u) ||
       (reinterpret_cast<uintptr_t>(tok_mask) & 3u))
@@ -249,7 +260,8 @@ blockffn_status blockffn_layer_forward(blockffn_handle h, const blockffn_weights
                                        int32_t call_flags, void* stream) {
   blockffn_status s = check_call(h, L);
   if (s != BLOCKFFN_OK) return s;
-  if (!w || !w->W_r || !w->gain || !w->U || !w->D || !x || !out) return BLOCKFFN_ERR_INVALID_ARG;
+  if (!w || !w->W_r || (!w->gain && !no_rmsnorm(h)) || !w->U || !w->D || !x || !out)
+    return BLOCKFFN_ERR_INVALID_ARG;
   if (misaligned(w->W_r) || misaligned(w->U) || misaligned(w->D) || misaligned(x) ||
       misaligned(out) || misaligned(x_next) || (reinterpret_cast<uintptr_t>(w->gain) & 3u) ||
       (reinterpret_cast<uintptr_t>(w->bias) & 3u) || (reinterpret_cast<uintptr_t>(stats) & 7u))
@@ -274,7 +286,7 @@ blockffn_status blockffn_layer_forward(blockffn_handle h, const blockffn_weights
     const bool x_stable = (call_flags & BLOCKFFN_CALL_INDEPENDENT_X) != 0;
     const bool chained = !(h->cfg.flags & BLOCKFFN_CFG_NO_CHAINING);
     const RoutingOut pub{h->union_mask, h->union_ids, h->n_union, stats, h->scores, h->tok_mask};
-    const RouterLogits lg{logits, w->gain, h->cfg.rms_eps};
+    const RouterLogits lg{logits, router_gain(h, w), h->cfg.rms_eps};
     // With x stable the router needs nothing from the caller's stream except that the readers
     // of its logit buffer (the layer call kLogitRing calls back) are done. It then runs on the
     // handle's own stream behind the mark that the call kLogitRing - 1 calls back left at its
@@ -375,6 +387,17 @@ blockffn_status blockffn_read_routing(blockffn_handle h, int32_t L, float* score
   copy(union_mask, h->union_mask, sizeof(uint32_t) * W);
   copy(union_ids, h->union_ids, sizeof(int32_t) * E);
   copy(n_union, h->n_union, sizeof(int32_t));
+  return e == cudaSuccess ? BLOCKFFN_OK : BLOCKFFN_ERR_CUDA;
+}
+
+blockffn_status blockffn_reuse_ratio(blockffn_handle h, const float* scores, int32_t L,
+                                     double* reuse, void* stream) {
+  if (!h || !reuse || L < 1) return BLOCKFFN_ERR_INVALID_ARG;
+  if (!scores && L > h->cfg.L_max) return BLOCKFFN_ERR_INVALID_ARG;
+  if ((reinterpret_cast<uintptr_t>(scores) & 3u) || (reinterpret_cast<uintptr_t>(reuse) & 7u))
+    return BLOCKFFN_ERR_INVALID_ARG;
+  const cudaError_t e = launch_reuse_ratio(h, scores ? scores : h->scores, L, reuse,
+                                           static_cast<cudaStream_t>(stream));
   return e == cudaSuccess ? BLOCKFFN_OK : BLOCKFFN_ERR_CUDA;
 }
 

@@ -42,6 +42,7 @@ struct blockffn_ctx {
   void* lean_ring;      // ring of bf16 intermediates of the one-kernel form (NULL: not used)
   unsigned long long* lean_seq;   // per ring (three of them, 32 words apart): [0] call tickets,
                                   // [1 .. 16] arrival counters of the ring slots
+  float* ones;          // [E] of 1.0f: the gain of the router without RMSNorm
   unsigned int* ticket; // last-block-done counters [8]
   uint32_t* status;     // sticky device status word
 };
@@ -59,6 +60,13 @@ __device__ __forceinline__ uint32_t f32_to_bf16_bits(float f) {
 }
 __device__ __forceinline__ float swish(float z) { return z / (1.0f + __expf(-z)); }
 
+// The router without RMSNorm (rms_eps == BLOCKFFN_NO_RMSNORM) has no gain: the kernels multiply
+// by a vector of ones and skip the normalisation where they see a negative eps.
+inline bool no_rmsnorm(const blockffn_ctx* c) { return c->cfg.rms_eps < 0.0f; }
+inline const float* router_gain(const blockffn_ctx* c, const blockffn_weights* w) {
+  return no_rmsnorm(c) ? c->ones : w->gain;
+}
+
 // ---- launchers (each returns the cudaError_t of its launch) ----------------
 cudaError_t launch_router(blockffn_ctx* c, const blockffn_weights* w, const void* x, int L,
                           float* scores, uint32_t* tok_mask, bool fuse_union,
@@ -69,6 +77,8 @@ cudaError_t launch_router(blockffn_ctx* c, const blockffn_weights* w, const void
 // stream of its own and lets its dependents go only by exiting, behind a fence.
 cudaError_t launch_chunk_union(blockffn_ctx* c, const float* scores, int L, uint32_t* union_mask,
                                int32_t* union_ids, int32_t* n_union, blockffn_stats* stats,
+                               cudaStream_t st);
+cudaError_t launch_reuse_ratio(blockffn_ctx* c, const float* scores, int L, double* reuse,
                                cudaStream_t st);
 cudaError_t launch_expert_simt(blockffn_ctx* c, const blockffn_weights* w, const void* x,
                                const float* scores, int L, const int32_t* union_ids,

@@ -159,7 +159,8 @@ __device__ int derive_union(const float* scores, const RouterLogits& lg, const i
       }
 #pragma unroll
       for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
-      const float r = 1.0f / sqrtf(ss / (float)E + lg.eps);
+      // a negative eps marks the router without RMSNorm (Sec. 4.2.3; lg.gain is then all ones)
+      const float r = lg.eps < 0.0f ? 1.0f : 1.0f / sqrtf(ss / (float)E + lg.eps);
       if (lane == 0) rinv[t] = r;
       if (few) {
 #pragma unroll

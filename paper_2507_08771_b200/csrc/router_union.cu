@@ -180,7 +180,9 @@ router_kernel(const uint16_t* __restrict__ x, const uint16_t* __restrict__ W_r,
     }
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
-    const float r = 1.0f / sqrtf(ss / (float)E + eps);
+    // eps < 0 marks the router without RMSNorm (Sec. 4.2.3): the ReLU values are the scores
+    // (the host passes a gain of ones)
+    const float r = eps < 0.0f ? 1.0f : 1.0f / sqrtf(ss / (float)E + eps);
     for (int w = 0; w < words; ++w) {
       const int e = 32 * w + lane;
       float s = 0.0f;
@@ -217,11 +219,70 @@ cudaError_t launch_router(blockffn_ctx* c, const blockffn_weights* w, const void
   lc.numAttrs = (mode == 2 || (c->cfg.flags & BLOCKFFN_CFG_NO_CHAINING)) ? 0 : 1;
   const cudaError_t e = cudaLaunchKernelEx(
       &lc, router_kernel, static_cast<const uint16_t*>(x), static_cast<const uint16_t*>(w->W_r),
-      w->gain, w->bias, logits, scores, tok_mask, L, c->cfg.d, c->cfg.E, c->cfg.rms_eps, c->ticket,
+      router_gain(c, w), w->bias, logits, scores, tok_mask, L, c->cfg.d, c->cfg.E, c->cfg.rms_eps,
+      c->ticket,
       fuse_union ? 1 : 0, c->union_mask, c->union_ids, c->n_union, stats, raw ? 1 : 0,
       raw ? mode : 0);
   if (e == cudaSuccess) c->launches += 1;
   return e;
+}
+
+namespace {
+
+// Reuse ratio (Sec. 4.1.2). One block. Warp w takes the pairs w, w + 8, ... of a round of eight; thread 0 then adds the
+// round's ratios to the running sum in token order, so the sum has one summation order.
+__global__ void __launch_bounds__(kThreads)
+reuse_ratio_kernel(const float* __restrict__ scores, int L, int E, double* reuse) {
+  __shared__ int n_first[kWarps], n_both[kWarps];
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  double sum = 0.0, pairs = 0.0;
+  if (threadIdx.x == 0) {
+    sum = reuse[0];
+    pairs = reuse[1];
+  }
+  for (int i0 = 0; i0 + 1 < L; i0 += kWarps) {
+    const int i = i0 + warp;
+    int a = 0, b = 0;
+    if (i + 1 < L) {
+      for (int e = lane; e < E; e += 32) {
+        const bool now = scores[(size_t)i * E + e] != 0.0f;
+        const bool next = scores[(size_t)(i + 1) * E + e] != 0.0f;
+        a += now;
+        b += now && next;
+      }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      a += __shfl_xor_sync(0xffffffffu, a, o);
+      b += __shfl_xor_sync(0xffffffffu, b, o);
+    }
+    if (lane == 0) {
+      n_first[warp] = a;
+      n_both[warp] = b;
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+      for (int w = 0; w < kWarps && i0 + w + 1 < L; ++w) {
+        if (n_first[w] == 0) continue;
+        sum += (double)n_both[w] / (double)n_first[w];
+        pairs += 1.0;
+      }
+    }
+    __syncthreads();
+  }
+  if (threadIdx.x == 0) {
+    reuse[0] = sum;
+    reuse[1] = pairs;
+  }
+}
+
+}  // namespace
+
+cudaError_t launch_reuse_ratio(blockffn_ctx* c, const float* scores, int L, double* reuse,
+                               cudaStream_t st) {
+  reuse_ratio_kernel<<<1, kThreads, 0, st>>>(scores, L, c->cfg.E, reuse);
+  c->launches += 1;
+  return cudaGetLastError();
 }
 
 cudaError_t launch_chunk_union(blockffn_ctx* c, const float* scores, int L, uint32_t* union_mask,

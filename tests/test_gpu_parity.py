@@ -770,6 +770,152 @@ def test_bench_launch_configuration_stack():
     assert layer.last_status() == 0
 
 
+def test_stack_router_on_per_layer_in_a_graph():
+    """The stack with the router on: every layer derives its scores from the hidden state the layer
+    before handed over (blockffn_layer_forward with the residual accumulate), all layers in one
+    graph. Per layer, the oracle is fed the exact bf16 input the GPU layer read; a mask flip inside
+    the band is followed through the library's own scores (read back per layer)."""
+    sh, seed = I.SHAPES[4], I.config_seed(4)
+    n_layers, L = 4, sh.L
+    layer = B.Layer(sh.d, sh.E, sh.d_e, L_max=L)
+    ws = [I.make_layer(sh, seed, layer=l, bias_shift=I.ROUTER_BIAS_SHIFT) for l in range(n_layers)]
+    dws = [layer.upload_weights(w) for w in ws]
+    x0 = I.make_correlated_x(sh.d, L, 0.9, seed, chunk=1)
+    x0d = B.to_device_bf16(x0)
+    res = torch.zeros(L, sh.d, device="cuda")
+    xs = torch.zeros(n_layers + 1, L, sh.d, dtype=torch.bfloat16, device="cuda")
+    scores = torch.zeros(n_layers, L, sh.E, device="cuda")
+    ids = torch.zeros(n_layers, sh.E, dtype=torch.int32, device="cuda")
+    nus = torch.zeros(n_layers, dtype=torch.int32, device="cuda")
+
+    def enqueue(stream):
+        res.copy_(x0d)
+        xs[0].copy_(x0d)
+        for l in range(n_layers):
+            B.blockffn_layer_forward(layer.h, dws[l].struct, xs[l], L, res, xs[l + 1], layer.stats,
+                                     B.CALL_ACCUMULATE, stream)
+            B.blockffn_read_routing(layer.h, L, scores[l], None, None, ids[l], nus[l:l + 1], stream)
+
+    graph_of(enqueue)
+    xs_bits = xs.view(torch.int16).cpu().numpy().view(np.uint16)
+    for l in range(n_layers):
+        w = ws[l]
+        ref = oracle.layer_forward(xs_bits[l], w["W_r"], w["gain"], w["U"], w["D"], bias=w["bias"],
+                                   union_only=True)
+        got_s = scores[l].cpu().numpy()
+        flips = (got_s != 0) != (ref.scores != 0)
+        assert np.all(np.abs(ref.a0[flips]) < FLIP_BAND), l
+        n = int(nus[l].item())
+        ffn = ref.out if not flips.any() else oracle.expert_ffn(
+            xs_bits[l], got_s.astype(np.float64), w["U"], w["D"], expert_ids=ids[l].cpu().numpy()[:n])
+        x_in = I.bf16_bits_to_f32(xs_bits[l]).astype(np.float64)
+        x_out = I.bf16_bits_to_f32(xs_bits[l + 1]).astype(np.float64)
+        want = x_in + ffn
+        slack = 2.0 ** -8 * (np.abs(want) + np.abs(x_in))
+        assert np.all(np.abs(x_out - want) <= TOL * rms(ffn) + slack), l
+    assert np.array_equal(xs_bits[n_layers], oracle.round_to_bf16(res.cpu().numpy()))
+    assert layer.last_status() == 0
+
+
+# ----------------------------------------------------------------------------
+# variants the paper describes: router without RMSNorm (Sec. 4.2.3), reuse ratio (Sec. 4.1.2)
+# ----------------------------------------------------------------------------
+@pytest.mark.parametrize("variant", VARIANTS)
+@pytest.mark.parametrize("d,E,d_e,L,bias", [(256, 40, 64, 8, -0.5), (512, 64, 128, 1, None),
+                                             (1024, 128, 64, 5, -0.8), (256, 200, 64, 32, -1.0),
+                                             (104, 33, 24, 3, -0.3)])
+def test_router_without_rmsnorm(variant, d, E, d_e, L, bias):
+    sh = I.Shape("t", d=d, E=E, d_e=d_e, L=L, union_frac=0.3)
+    w = I.make_layer(sh, 700 + d + E, bias_shift=bias)
+    x = I.make_x(d, L, 701 + d, chunk=L)
+    layer = B.Layer(d, E, d_e, L_max=L, rms_eps=B.NO_RMSNORM, variant=variant[0], flags=variant[1])
+    dw = layer.upload_weights({k: v for k, v in w.items() if k != "gain"})   # no gain to read
+    assert dw.struct.gain is None
+    # the router alone: scores are the ReLU of the logits (fp32 sums against the float64 ones)
+    a0, ref_s = oracle.router_relu_only(x, w["W_r"], w["bias"])
+    xd = B.to_device_bf16(x)
+    scores = torch.empty(L, E, device="cuda")
+    tok = torch.zeros(L, layer.words, dtype=torch.int32, device="cuda")
+    B.blockffn_router(layer.h, dw.struct, xd, L, scores, tok)
+    got_s = scores.cpu().numpy()
+    flips = (got_s != 0) != (ref_s != 0)
+    assert np.all(np.abs(a0[flips]) < FLIP_BAND)
+    assert np.abs(got_s - ref_s).max() <= 1e-4 * max(1.0, np.abs(ref_s).max())
+    assert np.array_equal(u32(tok), oracle.token_masks(got_s.astype(np.float64)))
+    # the whole layer, router on
+    ref = oracle.layer_forward(x, w["W_r"], None, w["U"], w["D"], bias=w["bias"], union_only=True,
+                               rmsnorm=False)
+    res = layer.forward(dw, xd)
+    torch.cuda.synchronize()
+    got_s = res.scores.cpu().numpy()
+    flips = (got_s != 0) != (ref.scores != 0)
+    assert np.all(np.abs(ref.a0[flips]) < FLIP_BAND)
+    n = int(res.n_union.item())
+    ids = res.union_ids.cpu().numpy()
+    tm = oracle.token_masks(got_s.astype(np.float64))
+    um2, ids2, n2 = oracle.chunk_union(tm, E)
+    assert n2 == n and np.array_equal(ids2, ids) and np.array_equal(u32(res.tok_mask), tm)
+    want = ref.out if not flips.any() else oracle.expert_ffn(x, got_s.astype(np.float64), w["U"], w["D"],
+                                                             expert_ids=ids[:n])
+    assert_close(res.out.cpu().numpy(), want, "layer out without RMSNorm")
+    assert layer.last_status() == 0
+
+
+def test_rms_eps_values_create_accepts():
+    for eps, ok in [(0.0, True), (1e-6, True), (B.NO_RMSNORM, True), (-0.5, False), (float("nan"), False)]:
+        if ok:
+            B.Layer(64, 8, 16, L_max=4, rms_eps=eps).close()
+        else:
+            with pytest.raises(B.BlockFFNError) as ei:
+                B.blockffn_create(64, 8, 16, 4, eps)
+            assert ei.value.code == B.ERR_INVALID_ARG
+    # with RMSNorm the gain stays mandatory
+    layer = B.Layer(64, 8, 16, L_max=4)
+    w = I.make_layer(I.Shape("t", d=64, E=8, d_e=16, L=4, union_frac=0.5), 5)
+    dw = layer.upload_weights({k: v for k, v in w.items() if k != "gain"})
+    with pytest.raises(B.BlockFFNError) as ei:
+        layer.forward(dw, B.to_device_bf16(I.make_x(64, 4, 5)))
+    assert ei.value.code == B.ERR_INVALID_ARG
+
+
+@pytest.mark.parametrize("L,E,p", [(2, 5, 0.5), (8, 40, 0.3), (9, 64, 0.25), (32, 128, 0.2),
+                                    (17, 1000, 0.02), (300, 96, 0.3), (1, 16, 0.5), (12, 64, 0.0)])
+def test_reuse_ratio_bit_exact(L, E, p):
+    rng = np.random.default_rng(900 + L + E)
+    layer = B.Layer(64, E, 16, L_max=min(L, 32))
+    acc_ref = np.zeros(2)
+    acc = torch.zeros(2, dtype=torch.float64, device="cuda")
+    for call in range(3):                                  # accumulates over sequences, in order
+        s = sparse_scores(rng, L, E, p)
+        if call == 1 and L > 2:
+            s[1] = 0.0                                     # a token with no active expert
+            s[0, 0], s[L - 1, E - 1] = -0.0, np.nan        # inactive / active by value
+        oracle.reuse_ratio(s.astype(np.float64), acc_ref)
+        B.blockffn_reuse_ratio(layer.h, dev(s), L, acc)
+    got = acc.cpu().numpy()
+    assert got.tobytes() == acc_ref.tobytes(), (got, acc_ref)
+
+
+def test_reuse_ratio_of_the_last_layer_call_and_argument_errors():
+    sh, seed = I.SHAPES[0], I.config_seed(0)
+    w = I.make_layer(sh, seed)
+    layer = B.Layer(sh.d, sh.E, sh.d_e, L_max=sh.L)
+    dw = layer.upload_weights(w)
+    x = I.make_correlated_x(sh.d, sh.L, 0.8, seed, chunk=2)
+    res = layer.forward(dw, B.to_device_bf16(x))
+    acc = torch.zeros(2, dtype=torch.float64, device="cuda")
+    B.blockffn_reuse_ratio(layer.h, None, sh.L, acc)       # the scores the layer call left
+    want = oracle.reuse_ratio(res.scores.cpu().numpy().astype(np.float64))
+    assert acc.cpu().numpy().tobytes() == want.tobytes()
+    assert want[1] > 0 and 0.0 <= want[0] / want[1] <= 1.0
+    for args in [(None, sh.L + 1, acc), (res.scores, 0, acc), (res.scores, sh.L, None),
+                 (res.scores, sh.L, acc.view(torch.uint8)[4:12])]:
+        with pytest.raises(B.BlockFFNError) as ei:
+            B.blockffn_reuse_ratio(layer.h, *args)
+        assert ei.value.code == B.ERR_INVALID_ARG
+    assert layer.last_status() == 0
+
+
 def test_bench_read_probe_runs_and_checks_its_arguments():
     """bench.py's read-only ceiling kernel (a library of its own, outside the product ABI)."""
     import bench

@@ -52,7 +52,8 @@ def test_create_rejects_bad_configs_before_touching_the_device(lib):
         (binding.Config(256, 16, 60, 4, 1e-6, 0, 0), binding.ERR_UNSUPPORTED),     # d_e % 8
         (binding.Config(256, 2000, 64, 4, 1e-6, 0, 0), binding.ERR_UNSUPPORTED),   # E too large
         (binding.Config(256, 16, 64, 64, 1e-6, 0, 0), binding.ERR_UNSUPPORTED),    # L_max > 32
-        (binding.Config(256, 16, 64, 4, -1.0, 0, 0), binding.ERR_INVALID_ARG),
+        (binding.Config(256, 16, 64, 4, -0.5, 0, 0), binding.ERR_INVALID_ARG),     # eps < 0, not the
+        (binding.Config(256, 16, 64, 4, float("nan"), 0, 0), binding.ERR_INVALID_ARG),  # no-RMSNorm value
         (binding.Config(256, 16, 64, 4, 1e-6, 9, 0), binding.ERR_INVALID_ARG),
     ]
     for cfg, want in bad:
