@@ -44,8 +44,8 @@
 // its arrival counter is an exact multiple of the call's CTA count when a call starts: the
 // counters only ever grow, nothing is reset, graph replays need no host state. A ticket
 // identifies a call only if every call drawing from the counter has the same number of CTAs, so
-// each kind of call (whole device; a third of it; a third of it in two token slices) has a ring
-// and a counter of its own. The hand-over also needs all CTAs of a call resident at once:
+// each kind of call (whole device; a third of it; a third of it with two teams per CTA) has a
+// ring and a counter of its own. The hand-over also needs all CTAs of a call resident at once:
 // lean_plan refuses grids for which that is not guaranteed.
 // The polling thread issues no asynchronous copies: a fence or an acquire by a thread waits
 // for that thread's own copies in flight.
@@ -588,13 +588,13 @@ __global__ void __launch_bounds__(kThreads, 3) expert_lean_kernel(const LeanPara
 
 // ---- host side ---------------------------------------------------------------------------
 struct LeanPlan {
-  int grid, slices, nc, ntg, cap_bytes, red_rows, max_cols, cols_q, cols_rem, smem, kb, slot_d;
+  int grid, teams, nc, ntg, cap_bytes, red_rows, max_cols, cols_q, cols_rem, smem, kb, slot_d;
   bool ok;
 };
 
 // Shapes: d a multiple of 64 up to 2048 (x fragments of a warp fit its registers); d_e a power
-// of two >= 64; L <= 32 (up to 8 tokens: one token group; 9 .. 16: two; 17 .. 32: four, these
-// only for calls that share the device and do not come with raw router logits).
+// of two >= 64; L <= 32 (up to 8 tokens: one token group; 9 .. 16: two; 17 .. 32: two teams of
+// two; more than 8 only for calls that share the device and do not come with raw router logits).
 //
 // How many CTAs a call gets. Every CTA reads all of x and all of h from L2, whatever its share
 // of the weights: with one CTA per SM that broadcast is half as many bytes again as the weights
@@ -613,8 +613,8 @@ LeanPlan lean_plan(const blockffn_config& cfg, int L, int sms, bool shared) {
   if (d % 64 || d > 512 * kMaxKB || d_e % 64 || (d_e & (d_e - 1)) || d_e > 4096 || E > 1024)
     return pl;
   pl.kb = (d / 64 + kWarps - 1) / kWarps;
-  pl.slices = L > 16 ? 2 : 1;
-  pl.ntg = L <= 8 ? 1 : 2;            // longer chunks: slices of at most 16 tokens, two groups each
+  pl.teams = L > 16 ? 2 : 1;          // more than 16 tokens: two teams of 8 warps in one CTA
+  pl.ntg = L <= 8 ? 1 : 2;            // longer chunks: 16 tokens per team, two groups each
   int u_exp = (cfg.flags >> 17) & 0x7ff;
   if (u_exp == 0) u_exp = (L == 1 ? E + 4 : 3 * E + 5) / (L == 1 ? 8 : 10);
   if (u_exp < 1) u_exp = 1;
@@ -624,7 +624,13 @@ LeanPlan lean_plan(const blockffn_config& cfg, int L, int sms, bool shared) {
   // device and takes all of it
   int split = shared && !(cfg.flags & BLOCKFFN_CFG_NO_SPLIT) ? 3 : 1;
   for (;; --split) {                               // at most three column tiles per CTA
-    pl.grid = (sms + split - 1) / split;
+    // Chunks of more than 8 tokens run one or two CTAs per SM; their grid is rounded down, so
+    // that whole calls fill the SMs (three calls of 49 CTAs on 148 SMs at one CTA per SM, six at
+    // two). With 50 the last call resident is short of two CTAs until an earlier call has ended,
+    // and its hand-over waits for them: measured 12.3 against 8.6 us per call at 32 tokens, 6.0
+    // against 5.2 at 16 (d = 2048, union 19). At three CTAs per SM nine calls are in flight either
+    // way and the slightly smaller share per CTA wins (4.18 against 4.37 us at 8 tokens).
+    pl.grid = pl.ntg == 1 ? (sms + split - 1) / split : sms / split;
     pl.nc = (d + 16 * pl.grid - 1) / (16 * pl.grid);
     if (pl.nc <= 3 || split == 1) break;
   }
@@ -635,18 +641,18 @@ LeanPlan lean_plan(const blockffn_config& cfg, int L, int sms, bool shared) {
   const int rows_exp = (u_exp * d_e + pl.grid - 1) / pl.grid;
   // an expert's slot in the down projection: its slab of D (columns split even / odd around
   // 64 bytes) and, with several token groups, its h tile
-  pl.slot_d = pl.max_cols * 2 * d_e + 64 + (pl.ntg > 1 ? 8 * pl.ntg * 2 * d_e + 64 : 0);
+  pl.slot_d = pl.max_cols * 2 * d_e + 64 + (pl.ntg > 1 ? 8 * pl.ntg * pl.teams * 2 * d_e + 64 : 0);
   const int need = max(min(rows_exp, 32) * 2 * d + 64, min(u_exp, 16) * pl.slot_d);
   // the partial tile (and a stage) is as wide as the expected share, between one row tile per
   // column tile and two row tiles
   int red_rows = rows_exp < 32 ? rows_exp : 32;
   if (red_rows < 16 * pl.nc) red_rows = 16 * pl.nc;
-  const int fixed = lean_layout(E, red_rows * pl.ntg, 0).total;
+  const int fixed = lean_layout(E, red_rows * pl.ntg * pl.teams, 0).total;
   // A call that owns the device gets the most CTAs per SM (three at most) whose shared memory
   // still holds the expected share in one stage; calls that share the device always run three
   // to an SM and stream their larger shares through in stages; chunks of more than 8 tokens
   // take a whole SM (their registers allow no more).
-  for (int n = pl.ntg == 2 ? 2 : 3; n >= 1; --n) {
+  for (int n = pl.teams == 2 ? 1 : pl.ntg == 2 ? 2 : 3; n >= 1; --n) {
     const int budget = (n == 1 ? kSmemMax : (kSmemMax + 1024) / n - 1024) & ~127;
     const int cap = (budget - fixed) & ~127;
     if (cap < need && n > 1 && split == 1) continue;
@@ -654,27 +660,28 @@ LeanPlan lean_plan(const blockffn_config& cfg, int L, int sms, bool shared) {
       if (n > 1) continue;
       if (cap < 2 * 2 * d + 128 || cap < 2 * pl.slot_d) return pl;
     }
-    if (pl.ntg > 1 && cap < 8 * pl.ntg * 16 * pl.nc * kWarps * 4) {            // the final partials
+    if (pl.ntg > 1 && cap < pl.teams * 8 * pl.ntg * 16 * pl.nc * kWarps * 4) {   // the final partials
       if (n > 1) continue;
       return pl;
     }
     // The hand-over inside the kernel needs every CTA of the call resident at once: n CTAs fit
     // an SM (by shared memory here, and the kernels are compiled for at least as many by
     // registers), so the call must not have more than n per SM.
-    if ((long long)pl.grid * pl.slices > (long long)sms * n) return pl;
+    if (pl.grid > sms * n) return pl;
     pl.cap_bytes = cap;
     pl.red_rows = red_rows;
-    pl.smem = lean_layout(E, red_rows * pl.ntg, cap).total;
+    pl.smem = lean_layout(E, red_rows * pl.ntg * pl.teams, cap).total;
     pl.ok = true;
     return pl;
   }
   return pl;
 }
 
-template <int KB, int NC, int NTG, int MODE>
+template <int KB, int NC, int NTG, int MODE, int TEAMS = 1>
 cudaError_t lean_attr() {
   const void* f = NTG == 1 ? reinterpret_cast<const void*>(&expert_lean_kernel<KB, NC, MODE>)
-                           : reinterpret_cast<const void*>(&expert_wide_kernel<KB, NC, NTG == 1 ? 2 : NTG, MODE>);
+                           : reinterpret_cast<const void*>(
+                                 &expert_wide_kernel<KB, NC, NTG == 1 ? 2 : NTG, MODE, TEAMS>);
   cudaError_t e = cudaFuncSetAttribute(f, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemMax);
   if (e != cudaSuccess) return e;
   return cudaFuncSetAttribute(f, cudaFuncAttributePreferredSharedMemoryCarveout,
@@ -687,27 +694,33 @@ cudaError_t lean_attrs_kb() {
   if (e == cudaSuccess) e = lean_attr<KB, NC, 1, 2>();
   if (e == cudaSuccess) e = lean_attr<KB, NC, 2, 0>();
   if (e == cudaSuccess) e = lean_attr<KB, NC, 2, 1>();
+  if (e == cudaSuccess) e = lean_attr<KB, NC, 2, 0, 2>();
+  if (e == cudaSuccess) e = lean_attr<KB, NC, 2, 1, 2>();
   return e;
 }
 
 template <int KB, int NC>
-cudaError_t lean_launch_kb(const cudaLaunchConfig_t& lc, const LeanParams& p, int ntg, int mode) {
+cudaError_t lean_launch_kb(const cudaLaunchConfig_t& lc, const LeanParams& p, int ntg, int teams,
+                           int mode) {
   if (ntg == 1)
     return mode == 2   ? cudaLaunchKernelEx(&lc, expert_lean_kernel<KB, NC, 2>, p)
            : mode == 1 ? cudaLaunchKernelEx(&lc, expert_lean_kernel<KB, NC, 1>, p)
                        : cudaLaunchKernelEx(&lc, expert_lean_kernel<KB, NC, 0>, p);
   if (mode == 2) return cudaErrorNotSupported;
-  return mode == 1 ? cudaLaunchKernelEx(&lc, expert_wide_kernel<KB, NC, 2, 1>, p)
-                   : cudaLaunchKernelEx(&lc, expert_wide_kernel<KB, NC, 2, 0>, p);
+  if (teams == 2)
+    return mode == 1 ? cudaLaunchKernelEx(&lc, expert_wide_kernel<KB, NC, 2, 1, 2>, p)
+                     : cudaLaunchKernelEx(&lc, expert_wide_kernel<KB, NC, 2, 0, 2>, p);
+  return mode == 1 ? cudaLaunchKernelEx(&lc, expert_wide_kernel<KB, NC, 2, 1, 1>, p)
+                   : cudaLaunchKernelEx(&lc, expert_wide_kernel<KB, NC, 2, 0, 1>, p);
 }
 template <int NC>
 cudaError_t lean_launch_nc(int kb, const cudaLaunchConfig_t& lc, const LeanParams& p, int ntg,
-                           int mode) {
+                           int teams, int mode) {
   switch (kb) {
-    case 1: return lean_launch_kb<1, NC>(lc, p, ntg, mode);
-    case 2: return lean_launch_kb<2, NC>(lc, p, ntg, mode);
-    case 3: return lean_launch_kb<3, NC>(lc, p, ntg, mode);
-    default: return lean_launch_kb<4, NC>(lc, p, ntg, mode);
+    case 1: return lean_launch_kb<1, NC>(lc, p, ntg, teams, mode);
+    case 2: return lean_launch_kb<2, NC>(lc, p, ntg, teams, mode);
+    case 3: return lean_launch_kb<3, NC>(lc, p, ntg, teams, mode);
+    default: return lean_launch_kb<4, NC>(lc, p, ntg, teams, mode);
   }
 }
 
@@ -725,8 +738,8 @@ bool expert_lean_supported(const blockffn_ctx* c, int L, bool with_logits) {
   return lean_plan(c->cfg, L, c->num_sms, !with_logits).ok;
 }
 
-// Three rings (calls that own the device, calls that share it, calls that share it in two token
-// slices: their grids differ, so each kind counts its own tickets) of kHRing intermediates of a
+// Three rings (calls that own the device, calls that share it, calls of more than 16 tokens that
+// share it: each kind counts its own tickets) of kHRing intermediates of a
 // chunk of L_max tokens; 0 when the shape never takes this kernel (or the rings would be
 // unreasonably large).
 size_t expert_lean_ws_bytes(const blockffn_config* cfg, int sms) {
@@ -779,7 +792,7 @@ cudaError_t launch_expert_lean(blockffn_ctx* c, const blockffn_weights* w, const
   p.h_slot = lean_h_slot_bytes(c->cfg) / 2;
   // a ring and a ticket counter per kind of call: tickets only identify a call when every call
   // that draws from the counter has the same number of CTAs
-  const int ring = !shared ? 0 : pl.slices == 1 ? 1 : 2;
+  const int ring = !shared ? 0 : pl.teams == 1 ? 1 : 2;
   p.h_ring = static_cast<uint16_t*>(c->lean_ring) + (size_t)ring * kHRing * p.h_slot;
   p.seq = c->lean_seq + 32 * ring;
   p.ready = p.seq + 1;
@@ -818,17 +831,17 @@ cudaError_t launch_expert_lean(blockffn_ctx* c, const blockffn_weights* w, const
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cudaLaunchConfig_t lc{};
-  lc.gridDim = dim3(pl.grid, pl.slices);
-  lc.blockDim = dim3(kThreads);
+  lc.gridDim = dim3(pl.grid);
+  lc.blockDim = dim3(kThreads * pl.teams);
   lc.stream = st;
   lc.attrs = attr;
   lc.numAttrs = chained ? 1 : 0;
   // never less than a quarter of an SM's shared memory: at most three CTAs then fit one SM,
   // whatever the shape, which is what the size of the ring rests on
   lc.dynamicSmemBytes = pl.smem > kMinSmem ? pl.smem : kMinSmem;
-  const cudaError_t e = pl.nc == 3   ? lean_launch_nc<3>(pl.kb, lc, p, pl.ntg, mode)
-                        : pl.nc == 2 ? lean_launch_nc<2>(pl.kb, lc, p, pl.ntg, mode)
-                                     : lean_launch_nc<1>(pl.kb, lc, p, pl.ntg, mode);
+  const cudaError_t e = pl.nc == 3   ? lean_launch_nc<3>(pl.kb, lc, p, pl.ntg, pl.teams, mode)
+                        : pl.nc == 2 ? lean_launch_nc<2>(pl.kb, lc, p, pl.ntg, pl.teams, mode)
+                                     : lean_launch_nc<1>(pl.kb, lc, p, pl.ntg, pl.teams, mode);
   if (e == cudaSuccess) c->launches += 1;
   return e;
 }

@@ -3,34 +3,43 @@
 // shared-memory layout, ring of h buffers and helpers.
 #pragma once
 
-// The same kernel for chunks of 9 .. 32 tokens: NTG groups of 8 tokens (2 or 4) per weight
-// fragment. (A kernel of its own rather than NTG = 1 of this template: written for any NTG the
-// single-group case kept a few more values live and spilled, which cost 15 % at 8 tokens.)
+// The kernel of expert_lean.cu for chunks of 9 .. 32 tokens: NTG = 2 groups of 8 tokens per
+// weight fragment. (A kernel of its own rather than NTG = 1 of this template: written for any
+// NTG the single-group case kept a few more values live and spilled, which cost 15 % at 8 tokens.)
 //
-// Chunks of more than 8 tokens take a whole SM per CTA: the x fragments of all token
-// groups stay in registers (up to 128 of them), every weight fragment read from shared memory is
-// used for all groups at once, and in the down projection the intermediate h of a round's experts
-// is staged in shared memory next to their slabs of D, because its fragments for all groups no
-// longer fit the registers next to NC x NTG accumulator tiles.
-template <int KB, int NC, int NTG, int MODE>
-__global__ void __launch_bounds__(kThreads, NTG == 2 ? 2 : 1) expert_wide_kernel(const LeanParams p) {
+// The x fragments of both token groups stay in registers (up to 64 of them; 128 registers per
+// thread, two CTAs per SM), every weight fragment read from shared memory is used for both
+// groups, and in the down projection the intermediate h of a round's experts is staged in
+// shared memory next to their slabs of D, because its fragments no longer fit the registers
+// next to NC x NTG accumulator tiles.
+//
+// TEAMS = 2 (chunks of 17 .. 32 tokens): a CTA of 512 threads, two teams of 8 warps. Both teams
+// work on the same weights in shared memory (copied once, by all 512 threads) and differ in their
+// tokens: team 0 takes tokens 0 .. 15, team 1 the rest, each with NTG = 2 groups in registers.
+// Within a team everything is as in the one-team kernel: K split over the team's 8 warps,
+// partial tiles and h tiles of its own.
+template <int KB, int NC, int NTG, int MODE, int TEAMS>
+__global__ void __launch_bounds__(kThreads * TEAMS, (NTG == 2 && TEAMS == 1) ? 2 : 1)
+expert_wide_kernel(const LeanParams p) {
   extern __shared__ __align__(128) unsigned char smem[];
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  // A chunk of more than 16 tokens is two slices of at most 16 (blockIdx.y): the slices share
-  // the call's union, its weights (read from DRAM once, the second reader finds them in L2), its
-  // ticket and its h buffer, and differ in their tokens. Lf: tokens of the chunk; tok0, L: the
-  // slice's first token and token count.
+  constexpr int kNT = kThreads * TEAMS;              // threads of the CTA
+  const int tid = threadIdx.x, lane = tid & 31;
+  const int team = TEAMS == 2 ? tid >> 8 : 0;        // which 16 tokens
+  const int ttid = tid & (kThreads - 1);             // thread within the team
+  const int warp = ttid >> 5;                        // warp within the team: its share of K
+  // Lf: tokens of the chunk; tok0, L: the team's first token and token count.
   const int d = p.d, d_e = p.d_e, Lf = p.L;
-  const int tok0 = blockIdx.y * 16, L = min(16, Lf - tok0);
-  const LeanLayout lay = lean_layout(p.E, p.red_rows * NTG, p.cap_bytes);
+  const int tok0 = team * 16, L = min(16, Lf - tok0);
+  const LeanLayout lay = lean_layout(p.E, p.red_rows * NTG * TEAMS, p.cap_bytes);
   const uint32_t sbase = smem_u32(smem);
   const uint32_t wbase = sbase + lay.off_w;
   int* ctl = reinterpret_cast<int*>(smem + kOffCtl);
   int* ids_sm = reinterpret_cast<int*>(smem + kOffIds);
-  float* red = reinterpret_cast<float*>(smem + lay.off_red);
+  float* red0 = reinterpret_cast<float*>(smem + lay.off_red);     // (the union derivation's scratch)
+  float* red = red0 + team * (8 * NTG * p.red_rows * kWarps);     // this team's partial tiles
   const int g = lane >> 2, tg = lane & 3;
-  const int G = gridDim.x, bx = blockIdx.x;   // the weights are shared out over gridDim.x
-  const unsigned Gt = gridDim.x * gridDim.y;  // CTAs of the call
+  const int G = gridDim.x, bx = blockIdx.x;   // the weights are shared out over the CTAs of the call
+  const unsigned Gt = gridDim.x;
 
   if (tid < 8) ctl[tid] = 0;
   unsigned long long ticket = 0;
@@ -47,7 +56,7 @@ __global__ void __launch_bounds__(kThreads, NTG == 2 ? 2 : 1) expert_wide_kernel
     pdl_trigger();
   };
   const int nu = derive_union<MODE>(p.scores, p.lg, p.ids_in, p.n_in, Lf, p.E, ids_sm, ctl,
-                                    reinterpret_cast<uint32_t*>(red), on_ticket);
+                                    reinterpret_cast<uint32_t*>(red0), on_ticket);
 
   // ---- up projection ---------------------------------------------------------------------
   const int R = nu * d_e;
@@ -59,7 +68,7 @@ __global__ void __launch_bounds__(kThreads, NTG == 2 ? 2 : 1) expert_wide_kernel
   // half the region that are refilled as they free
   // (chunks of more than 8 tokens have a whole SM's shared memory: three stages in the ring, so
   // that two are in flight under the math of the third)
-  constexpr int NS = NTG <= 2 ? 2 : 3;
+  constexpr int NS = (NTG <= 2 && TEAMS == 1) ? 2 : 3;
   const int ldr = min(p.red_rows, 32);       // a stage is at most two row tiles
   const bool single = nrows <= min(ldr, cap_rows);
   const int slot_rows = single ? max(nrows, 1) : min(ldr, cap_rows / NS);
@@ -70,8 +79,10 @@ __global__ void __launch_bounds__(kThreads, NTG == 2 ? 2 : 1) expert_wide_kernel
   const int sh = p.de_shift;
   // This thread's part of a row copy: 16-byte chunk my_c of the rows my_sub, my_sub + rpi, ...
   const int cpr = d >> 3;                       // chunks per row (<= 256)
-  const int rpi = cpr > 128 ? 1 : kThreads / cpr;   // rows the CTA copies per step
-  const int my_sub = (tid * p.magic_cpr) >> 16, my_c = tid - my_sub * cpr;
+  const int rpi = cpr > kNT / 2 ? 1 : kNT / cpr;    // rows the CTA copies per step
+  // (the reciprocal multiply is exact for tid < 256 only)
+  const int my_sub = TEAMS == 2 ? tid / cpr : (int)((tid * p.magic_cpr) >> 16);
+  const int my_c = tid - my_sub * cpr;
   const bool copies_u = my_sub < rpi;
   // stage gi: rows [r0 + gi rpg, ...) -> slot gi % NS, row m of the stage at
   // (m >> 1) row_bytes + (m & 1) half_u
@@ -119,7 +130,7 @@ __global__ void __launch_bounds__(kThreads, NTG == 2 ? 2 : 1) expert_wide_kernel
     }
   };
   // score and h element (expert slot, token, neuron) this thread finishes in a stage, per token
-  // group: token 8 n + tid / 32, row tid % 32 of the stage
+  // group: token 8 n + ttid / 32 of the team, row tid % 32 of the stage
   float sc[NTG];
   int hidx[NTG];        // element index into the h buffer, -1: nothing to finish
   auto prepare = [&](int gi) {
@@ -129,7 +140,7 @@ __global__ void __launch_bounds__(kThreads, NTG == 2 ? 2 : 1) expert_wide_kernel
     const int id = m < rows ? ids_sm[hq] : 0;
 #pragma unroll
     for (int n = 0; n < NTG; ++n) {
-      const int t = 8 * n + (tid >> 5);
+      const int t = 8 * n + (ttid >> 5);
       sc[n] = 0.0f;
       hidx[n] = -1;
       if (t < L && m < rows) {
@@ -227,7 +238,7 @@ __global__ void __launch_bounds__(kThreads, NTG == 2 ? 2 : 1) expert_wide_kernel
     for (int n = 0; n < NTG; ++n) {
       if (hidx[n] >= 0) {
         const float4* part =
-            reinterpret_cast<const float4*>(red + ((8 * n + (tid >> 5)) * ldr + (tid & 31)) * kWarps);
+            reinterpret_cast<const float4*>(red + ((8 * n + (ttid >> 5)) * ldr + (tid & 31)) * kWarps);
         const float4 lo = part[0], hi = part[1];
         const float v = ((lo.x + lo.y) + (lo.z + lo.w)) + ((hi.x + hi.y) + (hi.z + hi.w));
         hbuf[hidx[n]] = (uint16_t)f32_to_bf16_bits(sc[n] * swish_fast(v));
@@ -238,7 +249,7 @@ __global__ void __launch_bounds__(kThreads, NTG == 2 ? 2 : 1) expert_wide_kernel
   }
   cp_async_wait_all();
   __syncthreads();                 // every h element of this CTA has been stored
-  if (tid == kSyncThread) {
+  if (tid == kNT - 1) {
     __threadfence();
     asm volatile("red.relaxed.gpu.global.add.u64 [%0], 1;" ::"l"(p.ready + slot) : "memory");
   }
@@ -249,8 +260,8 @@ __global__ void __launch_bounds__(kThreads, NTG == 2 ? 2 : 1) expert_wide_kernel
   // expert's h tile follows its slab: token rows of 2 d_e bytes, split even / odd the same way.
   const int drow = 2 * d_e;
   const int half_d = ((p.max_cols + 1) >> 1) * drow + 64;
-  const int half_h = 4 * NTG * drow + 64;
-  const int slot_d = p.max_cols * drow + 64 + (NTG > 1 ? 8 * NTG * drow + 64 : 0);
+  const int half_h = 4 * NTG * TEAMS * drow + 64;
+  const int slot_d = p.max_cols * drow + 64 + (NTG > 1 ? 8 * NTG * TEAMS * drow + 64 : 0);
   const int h_off = p.max_cols * drow + 64;     // the h tile inside an expert's slot
   const int cap_slabs = p.cap_slabs;
   const bool one_round = nu <= cap_slabs;
@@ -259,13 +270,15 @@ __global__ void __launch_bounds__(kThreads, NTG == 2 ? 2 : 1) expert_wide_kernel
   const int c0 = bx * p.cols_q + min(bx, p.cols_rem);
   const int ncols = p.cols_q + (bx < p.cols_rem ? 1 : 0);
   // A slab is ncols << kshift chunks of 16 bytes; chunk c = column c >> kshift, piece
-  // c & (2^kshift - 1). Thread tid copies chunks tid, tid + kCopyThreads, ... of every expert.
+  // c & (2^kshift - 1). Thread tid copies chunks tid, tid + kDCopy, ... of every expert; the
+  // last warp (the polling thread's) copies none.
   const int kshift = sh - 3;                    // log2(chunks per D row)
   const uint32_t estride16 = (uint32_t)d << kshift;
-  const int nchunks = tid < kCopyThreads ? ncols << kshift : 0;
+  constexpr int kDCopy = kNT - 32;
+  const int nchunks = tid < kDCopy ? ncols << kshift : 0;
   auto issue_d = [&](int r) {
     const int q0 = r * rsz, n = min(rsz, nu - q0);
-    for (int c = tid; c < nchunks; c += kCopyThreads) {
+    for (int c = tid; c < nchunks; c += kDCopy) {
       const int cc = c >> kshift, k = c & ((1 << kshift) - 1);
       const uint32_t src0 = ((uint32_t)(c0 + cc) << kshift) + k;          // + id * d << kshift
       uint32_t dst = wbase + (r & 1) * rsz * slot_d + (cc >> 1) * drow + (cc & 1) * half_d + k * 16;
@@ -275,13 +288,15 @@ __global__ void __launch_bounds__(kThreads, NTG == 2 ? 2 : 1) expert_wide_kernel
     }
   };
   // (several token groups) the h tiles of a round's experts: L rows of 2 d_e bytes per expert,
-  // contiguous in the h buffer; chunk c = token c >> kshift, piece c & (2^kshift - 1)
+  // contiguous in the h buffer; chunk c = token c >> kshift, piece c & (2^kshift - 1). Each team
+  // fetches its own tokens into its own rows of the tile (team 1: rows 16 ..).
   auto issue_h = [&](int r) {
     const int q0 = r * rsz, n = min(rsz, nu - q0);
     const uint32_t hstep16 = (uint32_t)(Lf * d_e) >> 3;
-    for (int c = tid; c < (L << kshift); c += kThreads) {
+    for (int c = ttid; c < (L << kshift); c += kThreads) {
       const int t = c >> kshift, k = c & ((1 << kshift) - 1);
-      uint32_t dst = wbase + (r & 1) * rsz * slot_d + h_off + (t >> 1) * drow + (t & 1) * half_h + k * 16;
+      uint32_t dst = wbase + (r & 1) * rsz * slot_d + h_off + (8 * team + (t >> 1)) * drow +
+                     (t & 1) * half_h + k * 16;
       uint32_t src = (uint32_t)q0 * hstep16 + ((uint32_t)tok0 << kshift) + c;
       for (int i = 0; i < n; ++i, dst += slot_d, src += hstep16) cp_async16(dst, at16(hbuf, src));
     }
@@ -290,9 +305,9 @@ __global__ void __launch_bounds__(kThreads, NTG == 2 ? 2 : 1) expert_wide_kernel
   cp_async_commit();
   if (nrounds > 1) issue_d(1);
   cp_async_commit();
-  const int ot = tid >> 5, om = tid & 31;   // this thread's outputs: tokens ot (+ 8), columns om (+ 32)
+  const int ot = ttid >> 5, om = tid & 31;  // this thread's outputs: tokens ot (+ 8), columns om (+ 32)
   // hand-over: all CTAs of this call have stored their part of h
-  if (tid == kSyncThread) {
+  if (tid == kNT - 1) {
     const unsigned long long target = *reinterpret_cast<const unsigned long long*>(ctl + 138);
     const unsigned long long t0 = global_ns();
     // once a wait has run out on this handle the later ones give up quickly, until the caller
@@ -346,7 +361,7 @@ __global__ void __launch_bounds__(kThreads, NTG == 2 ? 2 : 1) expert_wide_kernel
   const uint32_t hstep16 = (uint32_t)(Lf * d_e) >> 3;        // one expert further, in 16 bytes
   // (several token groups) token rows 8 n + g of an h tile in shared memory (rows beyond the
   // chunk hold whatever the buffer held: their columns of the result are dropped)
-  const uint32_t hs_off = h_off + (g >> 1) * drow + (g & 1) * half_h + 16 * tg;
+  const uint32_t hs_off = h_off + (8 * team + (g >> 1)) * drow + (g & 1) * half_h + 16 * tg;
   for (int r = 0; r < nrounds && !dead; ++r) {
     const int q0 = r * rsz, n = min(rsz, nu - q0);
     const int nblk = n << pshift;
@@ -423,7 +438,9 @@ __global__ void __launch_bounds__(kThreads, NTG == 2 ? 2 : 1) expert_wide_kernel
     if (nu > 0) {
       // partial tiles -> part[t][m][warp] (m < 16 NC), then one thread per output element; with
       // several token groups the partials take the weight region, which is free by now
-      float* part0 = NTG == 1 ? red : reinterpret_cast<float*>(smem + lay.off_w);
+      float* part0 = NTG == 1 ? red
+                              : reinterpret_cast<float*>(smem + lay.off_w) +
+                                    team * (8 * NTG * (16 * NC) * kWarps);
       float* mine = part0 + (2 * tg * (16 * NC) + g) * kWarps + warp;
 #pragma unroll
       for (int n = 0; n < NTG; ++n) {
@@ -468,11 +485,11 @@ __global__ void __launch_bounds__(kThreads, NTG == 2 ? 2 : 1) expert_wide_kernel
     }
   }
   // CTA 0 publishes the routing it derived (after the wait: earlier readers are done)
-  if (blockIdx.x == 0 && blockIdx.y == 0) {
+  if (blockIdx.x == 0) {
     if (p.lg.a0 != nullptr && p.pub_scores != nullptr) {
       const int words = (p.E + 31) >> 5;
       const float* rinv = reinterpret_cast<const float*>(ctl + 104);
-      for (int t = warp; t < Lf; t += kWarps) {
+      for (int t = tid >> 5; t < Lf; t += kNT / 32) {
         for (int w = 0; w < words; ++w) {
           const int e = 32 * w + lane;
           float sv = 0.0f;
@@ -490,7 +507,7 @@ __global__ void __launch_bounds__(kThreads, NTG == 2 ? 2 : 1) expert_wide_kernel
     if (p.ids_in == nullptr) {
       const int words = (p.E + 31) >> 5;
       const uint32_t* um = reinterpret_cast<const uint32_t*>(ctl + 8);
-      for (int e = tid; e < p.E; e += kThreads) {
+      for (int e = tid; e < p.E; e += kNT) {
         if (p.pub_ids) p.pub_ids[e] = e < nu ? ids_sm[e] : -1;
         if (p.pub_mask && e < words) p.pub_mask[e] = um[e];
       }
