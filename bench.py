@@ -888,7 +888,7 @@ def extras(args, torch, device, peak):
     rows = {}
     for name, L, u in (("tree_32_tokens", 32, sh5.u), ("dense_32_tokens", 32, sh5.E),
                        ("one_token", 1, u1), ("dense_one_token", 1, sh5.E)):
-        wl = Workload(5, L, min(chunks, 16), 0, device, args.flags | B.cfg_expected_union(u), u=u)
+        wl = Workload(5, L, min(chunks, 64), 0, device, args.flags | B.cfg_expected_union(u), u=u)
         us = timed(wl) * 1e3 / wl.calls_per_step
         rows[name] = {"L": L, "u": u, "E": sh5.E, "us_per_call": us,
                       "GBps": wl.active_bytes / us / 1e3}

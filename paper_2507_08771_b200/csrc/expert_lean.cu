@@ -640,8 +640,8 @@ LeanPlan lean_plan(const blockffn_config& cfg, int L, int sms, bool shared) {
   pl.max_cols = pl.cols_q + (pl.cols_rem ? 1 : 0);
   const int rows_exp = (u_exp * d_e + pl.grid - 1) / pl.grid;
   // an expert's slot in the down projection: its slab of D (columns split even / odd around
-  // 64 bytes) and, with several token groups, its h tile
-  pl.slot_d = pl.max_cols * 2 * d_e + 64 + (pl.ntg > 1 ? 8 * pl.ntg * pl.teams * 2 * d_e + 64 : 0);
+  // 64 bytes) and, with two teams, its h tile
+  pl.slot_d = pl.max_cols * 2 * d_e + 64 + (pl.teams == 2 ? 8 * pl.ntg * pl.teams * 2 * d_e + 64 : 0);
   const int need = max(min(rows_exp, 32) * 2 * d + 64, min(u_exp, 16) * pl.slot_d);
   // the partial tile (and a stage) is as wide as the expected share, between one row tile per
   // column tile and two row tiles

@@ -8,16 +8,19 @@
 // NTG the single-group case kept a few more values live and spilled, which cost 15 % at 8 tokens.)
 //
 // The x fragments of both token groups stay in registers (up to 64 of them; 128 registers per
-// thread, two CTAs per SM), every weight fragment read from shared memory is used for both
-// groups, and in the down projection the intermediate h of a round's experts is staged in
-// shared memory next to their slabs of D, because its fragments no longer fit the registers
-// next to NC x NTG accumulator tiles.
+// thread, two CTAs per SM) and every weight fragment read from shared memory is used for both
+// groups. In the down projection the fragments of the intermediate h come from L2 straight into
+// registers, a few k blocks ahead of their use, in the registers the x fragments have left
+// (measured at 16 tokens, d = 2048, union 19: 5.04 us per call against 5.25 with h staged in
+// shared memory).
 //
 // TEAMS = 2 (chunks of 17 .. 32 tokens): a CTA of 512 threads, two teams of 8 warps. Both teams
 // work on the same weights in shared memory (copied once, by all 512 threads) and differ in their
 // tokens: team 0 takes tokens 0 .. 15, team 1 the rest, each with NTG = 2 groups in registers.
-// Within a team everything is as in the one-team kernel: K split over the team's 8 warps,
-// partial tiles and h tiles of its own.
+// Within a team everything is as in the one-team kernel: K split over the team's 8 warps and
+// partial tiles of its own, except that the intermediate h of a round's experts is staged in
+// shared memory next to their slabs of D: with one CTA per SM nothing else runs under the round
+// trips of direct fragment loads (measured at 32 tokens: 9.4 us per call direct, 8.6 staged).
 template <int KB, int NC, int NTG, int MODE, int TEAMS>
 __global__ void __launch_bounds__(kThreads * TEAMS, (NTG == 2 && TEAMS == 1) ? 2 : 1)
 expert_wide_kernel(const LeanParams p) {
@@ -256,12 +259,12 @@ expert_wide_kernel(const LeanParams p) {
 
   // ---- down projection -------------------------------------------------------------------
   // Slab of one expert: the CTA's columns (at most 16 NC, NC mma row tiles) as rows of 2 d_e
-  // bytes, even columns first, 64 bytes of padding, odd columns. With several token groups the
-  // expert's h tile follows its slab: token rows of 2 d_e bytes, split even / odd the same way.
+  // bytes, even columns first, 64 bytes of padding, odd columns. With two teams the expert's
+  // h tile follows its slab: token rows of 2 d_e bytes, split even / odd the same way.
   const int drow = 2 * d_e;
   const int half_d = ((p.max_cols + 1) >> 1) * drow + 64;
   const int half_h = 4 * NTG * TEAMS * drow + 64;
-  const int slot_d = p.max_cols * drow + 64 + (NTG > 1 ? 8 * NTG * TEAMS * drow + 64 : 0);
+  const int slot_d = p.max_cols * drow + 64 + (TEAMS == 2 ? 8 * NTG * TEAMS * drow + 64 : 0);
   const int h_off = p.max_cols * drow + 64;     // the h tile inside an expert's slot
   const int cap_slabs = p.cap_slabs;
   const bool one_round = nu <= cap_slabs;
@@ -287,7 +290,7 @@ expert_wide_kernel(const LeanParams p) {
         cp_async16(dst, at16(p.D, src0 + (uint32_t)ids_sm[q0 + i] * estride16));
     }
   };
-  // (several token groups) the h tiles of a round's experts: L rows of 2 d_e bytes per expert,
+  // (two teams) the h tiles of a round's experts: L rows of 2 d_e bytes per expert,
   // contiguous in the h buffer; chunk c = token c >> kshift, piece c & (2^kshift - 1). Each team
   // fetches its own tokens into its own rows of the tile (team 1: rows 16 ..).
   auto issue_h = [&](int r) {
@@ -328,7 +331,7 @@ expert_wide_kernel(const LeanParams p) {
   }
   __syncthreads();
   const bool dead = ctl[5] != 0;    // the wait ran out: out is left untouched
-  if constexpr (NTG > 1) {
+  if constexpr (TEAMS == 2) {
     if (!dead) {
       if (nrounds > 0) issue_h(0);
       cp_async_commit();
@@ -357,30 +360,37 @@ expert_wide_kernel(const LeanParams p) {
     offs[c][0] = col_off(g + 16 * c);
     offs[c][1] = col_off(g + 16 * c + 8);
   }
-  const uint4* hrow = reinterpret_cast<const uint4*>(hbuf + (tok0 + min(g, L - 1)) * d_e) + tg;
+  // token rows 8 n + g of this team in the h buffer (rows beyond the chunk repeat its last one:
+  // their columns of the result are dropped)
+  const uint4* hrow[NTG];
+#pragma unroll
+  for (int n = 0; n < NTG; ++n)
+    hrow[n] = reinterpret_cast<const uint4*>(hbuf + (tok0 + min(8 * n + g, L - 1)) * d_e) + tg;
   const uint32_t hstep16 = (uint32_t)(Lf * d_e) >> 3;        // one expert further, in 16 bytes
-  // (several token groups) token rows 8 n + g of an h tile in shared memory (rows beyond the
-  // chunk hold whatever the buffer held: their columns of the result are dropped)
+  // (two teams) token rows 8 n + g of an h tile in shared memory (rows beyond the chunk hold
+  // whatever the buffer held: their columns of the result are dropped)
   const uint32_t hs_off = h_off + (8 * team + (g >> 1)) * drow + (g & 1) * half_h + 16 * tg;
   for (int r = 0; r < nrounds && !dead; ++r) {
     const int q0 = r * rsz, n = min(rsz, nu - q0);
     const int nblk = n << pshift;
     const uint32_t d_base = wbase + (r & 1) * rsz * slot_d;
-    if constexpr (NTG == 1) {
+    if constexpr (TEAMS == 1) {
       // this warp's k blocks b = warp + 8 i of the round, in batches whose h fragments are all
       // requested before the first is used; block b = expert b >> pshift, k block b & (npairs - 1)
-      // (fewer per batch with more column tiles: their accumulators need the registers, and a
-      // round then holds fewer experts anyway)
-      constexpr int kHB = NC == 1 ? 5 : NC == 2 ? 3 : 2;
-      Frag64 fh[kHB];
+      // (fewer per batch with more column tiles: their accumulators need the registers)
+      constexpr int kHB = NC == 1 ? 4 : NC == 2 ? 3 : 2;
+      Frag64 fh[kHB][NTG];
       auto load_h = [&](int b0) {
 #pragma unroll
         for (int i = 0; i < kHB; ++i) {
           const int b = b0 + kWarps * i;
           if (b < nblk) {
-            const uint4* hp = hrow + (uint32_t)(q0 + (b >> pshift)) * hstep16 + 8 * (b & (npairs - 1));
-            fh[i].lo = ld_cg_v4(hp);
-            fh[i].hi = ld_cg_v4(hp + 4);
+            const uint32_t ho = (uint32_t)(q0 + (b >> pshift)) * hstep16 + 8 * (b & (npairs - 1));
+#pragma unroll
+            for (int n2 = 0; n2 < NTG; ++n2) {
+              fh[i][n2].lo = ld_cg_v4(hrow[n2] + ho);
+              fh[i][n2].hi = ld_cg_v4(hrow[n2] + ho + 4);
+            }
           }
         }
       };
@@ -398,7 +408,9 @@ expert_wide_kernel(const LeanParams p) {
             for (int c = 0; c < NC; ++c) {
               const uint4 alo = lds128(da + offs[c][0]), ahi = lds128(da + offs[c][0] + 64);
               const uint4 blo = lds128(da + offs[c][1]), bhi = lds128(da + offs[c][1] + 64);
-              mma64(acc[c][0][0], acc[c][0][1], alo, ahi, blo, bhi, fh[i]);
+#pragma unroll
+              for (int n2 = 0; n2 < NTG; ++n2)
+                mma64(acc[c][n2][0], acc[c][n2][1], alo, ahi, blo, bhi, fh[i][n2]);
             }
           }
         }
@@ -428,7 +440,7 @@ expert_wide_kernel(const LeanParams p) {
     __syncthreads();               // every warp is done with this round's slabs
     if (r + 2 < nrounds) {
       issue_d(r + 2);
-      if constexpr (NTG > 1) issue_h(r + 2);
+      if constexpr (TEAMS == 2) issue_h(r + 2);
     }
     cp_async_commit();
   }
