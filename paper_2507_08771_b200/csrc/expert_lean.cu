@@ -62,15 +62,28 @@ constexpr int kMaxKB = 4;            // 64-wide k blocks of x per warp: d <= 8 *
 struct LeanLayout {
   int off_red, off_w, total;
 };
-// red: cross-warp partials [8 tokens][rows][8 warps] f32, rows = red_rows (up) or 16 per column
-// tile (down); red_rows is at least 16 (32 with two column tiles)
-__host__ __device__ inline LeanLayout lean_layout(int E, int red_rows, int cap_bytes) {
+// red: cross-warp partial tiles, f32. The long-chunk kernel keeps them [token][warp][row]: a
+// warp's rows are ws = rows rounded up to even apart, a token is ts = 8 ws + 4 words further. The 32 lanes of a partial store
+// (tokens 2 tg (+ 1), rows g (+ 8)) then fall into 32 different banks, and the eight partials
+// of an element are read by consecutive lanes from consecutive words. (With the warp index
+// innermost every such store was an 8-way bank conflict: a third of the shared-memory
+// wavefronts of a stage.) The 8-token kernel keeps [token][row][warp] inside the same region
+// (see there). rows = red_rows in the up projection, 16 per column tile in the down projection;
+// red_rows is at least 16 (16 per column tile); groups: token groups of 8.
+__host__ __device__ inline int red_ws(int rows) { return (rows + 1) & ~1; }
+__host__ __device__ inline int red_ts(int rows) { return kWarps * red_ws(rows) + 4; }
+__host__ __device__ inline LeanLayout lean_layout(int E, int red_rows, int groups, int cap_bytes) {
   LeanLayout s;
   s.off_red = kOffIds + align128(E * 4);
-  const int red = kWarps * 8 * 4 * red_rows;
+  const int red = groups == 1 ? kWarps * 8 * 4 * red_rows              // [token][row][warp]
+                              : groups * 8 * red_ts(red_rows) * 4;     // [token][warp][row]
   s.off_w = s.off_red + align128(red);
   s.total = s.off_w + cap_bytes;
   return s;
+}
+// sum of an element's eight partials, e: the first one, ws apart (fixed order)
+__device__ __forceinline__ float red_sum(const float* e, int ws) {
+  return ((e[0] + e[ws]) + (e[2 * ws] + e[3 * ws])) + ((e[4 * ws] + e[5 * ws]) + (e[6 * ws] + e[7 * ws]));
 }
 
 struct LeanParams {
@@ -168,7 +181,7 @@ __global__ void __launch_bounds__(kThreads, 3) expert_lean_kernel(const LeanPara
   extern __shared__ __align__(128) unsigned char smem[];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int d = p.d, d_e = p.d_e, L = p.L;
-  const LeanLayout lay = lean_layout(p.E, p.red_rows, p.cap_bytes);
+  const LeanLayout lay = lean_layout(p.E, p.red_rows, 1, p.cap_bytes);
   const uint32_t sbase = smem_u32(smem);
   const uint32_t wbase = sbase + lay.off_w;
   int* ctl = reinterpret_cast<int*>(smem + kOffCtl);
@@ -321,6 +334,9 @@ __global__ void __launch_bounds__(kThreads, 3) expert_lean_kernel(const LeanPara
     cp_async_wait_group<1>();      // all but the newest group: this stage has landed
     __syncthreads();
     // partial tiles -> red[t][m][warp]: the eight partials of an element are 32 contiguous bytes
+    // (two 128-bit loads; the stores conflict on banks, but this kernel is bound by its
+    // instruction count: the conflict-free layout of the long-chunk kernel costs six more
+    // loads per element and measured 3 % slower here)
     float* mine = red + (2 * tg * ldr + g) * kWarps + warp;
     const int nt = ldr * kWarps;           // one token further
     {
@@ -647,7 +663,7 @@ LeanPlan lean_plan(const blockffn_config& cfg, int L, int sms, bool shared) {
   // column tile and two row tiles
   int red_rows = rows_exp < 32 ? rows_exp : 32;
   if (red_rows < 16 * pl.nc) red_rows = 16 * pl.nc;
-  const int fixed = lean_layout(E, red_rows * pl.ntg * pl.teams, 0).total;
+  const int fixed = lean_layout(E, red_rows, pl.ntg * pl.teams, 0).total;
   // A call that owns the device gets the most CTAs per SM (three at most) whose shared memory
   // still holds the expected share in one stage; calls that share the device always run three
   // to an SM and stream their larger shares through in stages; chunks of more than 8 tokens
@@ -660,7 +676,7 @@ LeanPlan lean_plan(const blockffn_config& cfg, int L, int sms, bool shared) {
       if (n > 1) continue;
       if (cap < 2 * 2 * d + 128 || cap < 2 * pl.slot_d) return pl;
     }
-    if (pl.ntg > 1 && cap < pl.teams * 8 * pl.ntg * 16 * pl.nc * kWarps * 4) {   // the final partials
+    if (pl.ntg > 1 && cap < pl.teams * 8 * pl.ntg * red_ts(16 * pl.nc) * 4) {    // the final partials
       if (n > 1) continue;
       return pl;
     }
@@ -670,7 +686,7 @@ LeanPlan lean_plan(const blockffn_config& cfg, int L, int sms, bool shared) {
     if (pl.grid > sms * n) return pl;
     pl.cap_bytes = cap;
     pl.red_rows = red_rows;
-    pl.smem = lean_layout(E, red_rows * pl.ntg * pl.teams, cap).total;
+    pl.smem = lean_layout(E, red_rows, pl.ntg * pl.teams, cap).total;
     pl.ok = true;
     return pl;
   }

@@ -33,13 +33,13 @@ expert_wide_kernel(const LeanParams p) {
   // Lf: tokens of the chunk; tok0, L: the team's first token and token count.
   const int d = p.d, d_e = p.d_e, Lf = p.L;
   const int tok0 = team * 16, L = min(16, Lf - tok0);
-  const LeanLayout lay = lean_layout(p.E, p.red_rows * NTG * TEAMS, p.cap_bytes);
+  const LeanLayout lay = lean_layout(p.E, p.red_rows, NTG * TEAMS, p.cap_bytes);
   const uint32_t sbase = smem_u32(smem);
   const uint32_t wbase = sbase + lay.off_w;
   int* ctl = reinterpret_cast<int*>(smem + kOffCtl);
   int* ids_sm = reinterpret_cast<int*>(smem + kOffIds);
   float* red0 = reinterpret_cast<float*>(smem + lay.off_red);     // (the union derivation's scratch)
-  float* red = red0 + team * (8 * NTG * p.red_rows * kWarps);     // this team's partial tiles
+  float* red = red0 + team * (8 * NTG * red_ts(p.red_rows));      // this team's partial tiles
   const int g = lane >> 2, tg = lane & 3;
   const int G = gridDim.x, bx = blockIdx.x;   // the weights are shared out over the CTAs of the call
   const unsigned Gt = gridDim.x;
@@ -199,9 +199,9 @@ expert_wide_kernel(const LeanParams p) {
     };
     cp_async_wait_group<NS - 1>(); // all but the NS - 1 newest groups: this stage has landed
     __syncthreads();
-    // partial tiles -> red[t][m][warp]: the eight partials of an element are 32 contiguous bytes
-    float* mine = red + (2 * tg * ldr + g) * kWarps + warp;
-    const int nt = ldr * kWarps;           // one token further
+    // partial tiles -> red[t][warp][m]
+    const int ws = red_ws(ldr), nt = red_ts(ldr);      // one warp, one token further
+    float* mine = red + 2 * tg * nt + warp * ws + g;
     auto do_tile = [&](const int tile) {
       const uint32_t a0 = row_addr(g + 16 * tile), b0 = row_addr(g + 16 * tile + 8);
       float c0[NTG][4], c1[NTG][4];
@@ -221,14 +221,14 @@ expert_wide_kernel(const LeanParams p) {
       const int m0 = g + 16 * tile;
 #pragma unroll
       for (int n = 0; n < NTG; ++n) {
-        float* o = mine + (8 * n * ldr + 16 * tile) * kWarps;
+        float* o = mine + 8 * n * nt + 16 * tile;
         if (m0 < ldr) {
           o[0] = c0[n][0] + c1[n][0];
           o[nt] = c0[n][1] + c1[n][1];
         }
         if (m0 + 8 < ldr) {
-          o[8 * kWarps] = c0[n][2] + c1[n][2];
-          o[nt + 8 * kWarps] = c0[n][3] + c1[n][3];
+          o[8] = c0[n][2] + c1[n][2];
+          o[nt + 8] = c0[n][3] + c1[n][3];
         }
       }
     };
@@ -240,10 +240,7 @@ expert_wide_kernel(const LeanParams p) {
 #pragma unroll
     for (int n = 0; n < NTG; ++n) {
       if (hidx[n] >= 0) {
-        const float4* part =
-            reinterpret_cast<const float4*>(red + ((8 * n + (ttid >> 5)) * ldr + (tid & 31)) * kWarps);
-        const float4 lo = part[0], hi = part[1];
-        const float v = ((lo.x + lo.y) + (lo.z + lo.w)) + ((hi.x + hi.y) + (hi.z + hi.w));
+        const float v = red_sum(red + (8 * n + (ttid >> 5)) * red_ts(ldr) + (tid & 31), red_ws(ldr));
         hbuf[hidx[n]] = (uint16_t)f32_to_bf16_bits(sc[n] * swish_fast(v));
       }
     }
@@ -448,21 +445,20 @@ expert_wide_kernel(const LeanParams p) {
   pdl_wait();                      // out (and x_next) may still be in use by the call before
   if (!dead) {
     if (nu > 0) {
-      // partial tiles -> part[t][m][warp] (m < 16 NC), then one thread per output element; with
-      // several token groups the partials take the weight region, which is free by now
-      float* part0 = NTG == 1 ? red
-                              : reinterpret_cast<float*>(smem + lay.off_w) +
-                                    team * (8 * NTG * (16 * NC) * kWarps);
-      float* mine = part0 + (2 * tg * (16 * NC) + g) * kWarps + warp;
+      // partial tiles -> part[t][warp][m] (m < 16 NC), then one thread per output element; the
+      // partials take the weight region, which is free by now
+      constexpr int ws2 = 16 * NC, ts2 = kWarps * ws2 + 4;
+      float* part0 = reinterpret_cast<float*>(smem + lay.off_w) + team * (8 * NTG * ts2);
+      float* mine = part0 + 2 * tg * ts2 + warp * ws2 + g;
 #pragma unroll
       for (int n = 0; n < NTG; ++n) {
 #pragma unroll
         for (int c = 0; c < NC; ++c) {
-          float* o = mine + (8 * n * (16 * NC) + 16 * c) * kWarps;
+          float* o = mine + 8 * n * ts2 + 16 * c;
           o[0] = acc[c][n][0][0] + acc[c][n][1][0];
-          o[(16 * NC) * kWarps] = acc[c][n][0][1] + acc[c][n][1][1];
-          o[8 * kWarps] = acc[c][n][0][2] + acc[c][n][1][2];
-          o[(16 * NC + 8) * kWarps] = acc[c][n][0][3] + acc[c][n][1][3];
+          o[ts2] = acc[c][n][0][1] + acc[c][n][1][1];
+          o[8] = acc[c][n][0][2] + acc[c][n][1][2];
+          o[ts2 + 8] = acc[c][n][0][3] + acc[c][n][1][3];
         }
       }
       __syncthreads();
@@ -474,9 +470,7 @@ expert_wide_kernel(const LeanParams p) {
           for (int k = 0; k < (NC + 1) / 2; ++k) {
             const int m = om + 32 * k;
             if (m < ncols) {
-              const float4* part = reinterpret_cast<const float4*>(part0 + (t * (16 * NC) + m) * kWarps);
-              const float4 lo = part[0], hi = part[1];
-              float v = ((lo.x + lo.y) + (lo.z + lo.w)) + ((hi.x + hi.y) + (hi.z + hi.w));
+              float v = red_sum(part0 + t * ts2 + m, ws2);
               const int o = (tok0 + t) * d + c0 + m;
               if (p.accumulate) v += __ldcg(p.out + o);
               p.out[o] = v;
