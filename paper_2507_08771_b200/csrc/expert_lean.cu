@@ -188,6 +188,7 @@ __global__ void __launch_bounds__(kThreads, 3) expert_lean_kernel(const LeanPara
   int* ids_sm = reinterpret_cast<int*>(smem + kOffIds);
   float* red = reinterpret_cast<float*>(smem + lay.off_red);
   const int g = lane >> 2, tg = lane & 3;
+  const int wpos = (warp + 2 * tg + (g >> 2)) & 7;   // where this warp's partial of an element sits
   const int G = gridDim.x, bx = blockIdx.x;
 
   if (tid < 8) ctl[tid] = 0;
@@ -333,11 +334,13 @@ __global__ void __launch_bounds__(kThreads, 3) expert_lean_kernel(const LeanPara
     const uint32_t a0 = row_addr(g), b0 = row_addr(g + 8);
     cp_async_wait_group<1>();      // all but the newest group: this stage has landed
     __syncthreads();
-    // partial tiles -> red[t][m][warp]: the eight partials of an element are 32 contiguous bytes
-    // (two 128-bit loads; the stores conflict on banks, but this kernel is bound by its
-    // instruction count: the conflict-free layout of the long-chunk kernel costs six more
-    // loads per element and measured 3 % slower here)
-    float* mine = red + (2 * tg * ldr + g) * kWarps + warp;
+    // partial tiles -> red[t][m][.]: the eight partials of an element are 32 contiguous bytes
+    // (two 128-bit loads: this kernel is bound by its instruction count, and the layout of the
+    // long-chunk kernel costs six more loads per element). Warp w's partial sits at position
+    // (w + 2 tg + g / 4) mod 8 of those eight words: the 32 lanes of a store then fall into 32
+    // different banks (with w itself as the position they fell into four), and the reader adds
+    // all eight words anyway.
+    float* mine = red + (2 * tg * ldr + g) * kWarps + wpos;
     const int nt = ldr * kWarps;           // one token further
     {
       float c0[4] = {0.f, 0.f, 0.f, 0.f}, c1[4] = {0.f, 0.f, 0.f, 0.f};
@@ -522,7 +525,7 @@ __global__ void __launch_bounds__(kThreads, 3) expert_lean_kernel(const LeanPara
   if (!dead) {
     if (nu > 0) {
       // partial tiles -> red[t][m][warp] (m < 16 NC), then one thread per output element
-      float* mine = red + (2 * tg * (16 * NC) + g) * kWarps + warp;
+      float* mine = red + (2 * tg * (16 * NC) + g) * kWarps + wpos;
 #pragma unroll
       for (int c = 0; c < NC; ++c) {
         mine[(16 * c) * kWarps] = acc[c][0][0] + acc[c][1][0];
