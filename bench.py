@@ -603,7 +603,8 @@ def run_ours(args):
         "gpu_launches_per_step": launches_per_step,
         "roofline": {
             "bound": "hbm",
-            "kernel": ("expert_lean_kernel (one launch per call: up projection, hand-over, down projection)"
+            "kernel": (("expert_lean_kernel" if wl.L <= 8 else "expert_wide_kernel") +
+                       " (one launch per call: up projection, hand-over, down projection)"
                        if launches_per_call == 1 else
                        "expert_up_mma + expert_down_mma (the chained pair of one call)"
                        if launches_per_call == 2 and args.variant != 1 else "expert_up_simt + expert_down_simt"),
