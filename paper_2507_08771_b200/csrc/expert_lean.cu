@@ -128,6 +128,15 @@ __device__ __forceinline__ unsigned long long ld_acquire_u64(const unsigned long
   asm volatile("ld.acquire.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(p) : "memory");
   return v;
 }
+// Asks L2 for the 128-byte lines that hold [p, p + bytes) (whole lines that contain a valid byte:
+// never beyond the page of the range), shared out over the CTA's threads.
+__device__ __forceinline__ void prefetch_l2(const void* p, int bytes) {
+  const unsigned long long a = reinterpret_cast<unsigned long long>(p);
+  const unsigned long long a0 = a & ~127ull;
+  const int lines = (int)((a + (unsigned long long)bytes - a0 + 127ull) >> 7);
+  for (int i = threadIdx.x; i < lines; i += blockDim.x)
+    asm volatile("prefetch.global.L2 [%0];" ::"l"(a0 + 128ull * (unsigned)i));
+}
 // A 64-wide k block of a small operand row straight from global memory (L2): this lane's 8
 // consecutive k of each 32-wide half, the same k permutation load_frag64 applies to the
 // shared-memory operand.
@@ -205,6 +214,9 @@ __global__ void __launch_bounds__(kThreads, 3) expert_lean_kernel(const LeanPara
         p.hold ? ~0ull : (n / kHRing + 1ull) * (unsigned)G;
     pdl_trigger();
   };
+  // With the caller's union list the scores are first read when the first stage is finished:
+  // their lines are requested now, or that read waits for DRAM in the middle of the up projection.
+  if constexpr (MODE == 1) prefetch_l2(p.scores, L * p.E * 4);
   const int nu = derive_union<MODE>(p.scores, p.lg, p.ids_in, p.n_in, L, p.E, ids_sm, ctl,
                                     reinterpret_cast<uint32_t*>(red), on_ticket);
 

@@ -58,6 +58,8 @@ expert_wide_kernel(const LeanParams p) {
         p.hold ? ~0ull : (n / kHRing + 1ull) * Gt;
     pdl_trigger();
   };
+  // (the caller's union list: the scores are first read at the end of the first stage)
+  if constexpr (MODE == 1) prefetch_l2(p.scores, Lf * p.E * 4);
   const int nu = derive_union<MODE>(p.scores, p.lg, p.ids_in, p.n_in, Lf, p.E, ids_sm, ctl,
                                     reinterpret_cast<uint32_t*>(red0), on_ticket);
 
