@@ -29,11 +29,14 @@ cudaError_t launch_tensor_core(blockffn_ctx* c, const blockffn_weights* w, const
                                const RoutingOut* pub, const RouterLogits* logits, bool logits_final,
                                cudaStream_t st) {
   // The one-kernel form pays off where calls overlap freely, i.e. where x is stable (for a
-  // router-on call: the router has finished before the expert stage starts). A call in a
-  // dependent chain (x comes from the call before) runs as the pair, whose two hand-overs are
-  // shorter than a grid-wide exchange inside one kernel.
+  // router-on call: the router has finished before the expert stage starts). A call of up to 8
+  // tokens in a dependent chain (x comes from the call before) runs as the pair, whose two
+  // hand-overs are shorter than a grid-wide exchange inside one kernel; a longer chunk in such a
+  // chain (weights and scores promised stable) takes the one-kernel form on the whole device,
+  // which keeps its weights in shared memory for all tokens at once.
   const bool x_stable = logits ? logits_final : (call_flags & BLOCKFFN_CALL_INDEPENDENT_X) != 0;
-  if (x_stable && expert_lean_supported(c, L, logits != nullptr))
+  const bool dep_long = !x_stable && !logits && (call_flags & BLOCKFFN_CALL_INDEPENDENT) && L > 8;
+  if ((x_stable || dep_long) && expert_lean_supported(c, L, logits != nullptr, x_stable && !logits))
     return launch_expert_lean(c, w, x, scores, L, union_ids, n_union, out, x_next, call_flags, pub,
                               logits, logits_final, st);
   return launch_expert_mma(c, w, x, scores, L, union_ids, n_union, out, x_next, call_flags, pub,

@@ -107,6 +107,7 @@ struct LeanParams {
   uint32_t magic_cpr;          // ceil(2^16 / (d / 8)): tid / (d / 8) = tid * magic_cpr >> 16
   int max_cols, cols_q, cols_rem;
   int accumulate;
+  int dep;                     // x comes from the call before on the stream: wait before reading it
   int hold;                    // test aid: wait for an arrival that never comes
   unsigned long long wait_ns;  // bound of the hand-over wait
   uint32_t* status;
@@ -640,7 +641,6 @@ LeanPlan lean_plan(const blockffn_config& cfg, int L, int sms, bool shared) {
   pl.ok = false;
   const int d = cfg.d, d_e = cfg.d_e, E = cfg.E;
   if (L < 1 || L > 32 || sms < 1) return pl;
-  if (L > 8 && !shared) return pl;
   if (d % 64 || d > 512 * kMaxKB || d_e % 64 || (d_e & (d_e - 1)) || d_e > 4096 || E > 1024)
     return pl;
   pl.kb = (d / 64 + kWarps - 1) / kWarps;
@@ -782,10 +782,10 @@ size_t lean_h_slot_bytes(const blockffn_config& cfg) {
 
 // Whether a call of L tokens whose x is stable takes the one-kernel form (with_logits: it comes
 // with raw router logits, i.e. it is the expert stage of a router-on layer call).
-bool expert_lean_supported(const blockffn_ctx* c, int L, bool with_logits) {
+bool expert_lean_supported(const blockffn_ctx* c, int L, bool with_logits, bool shared) {
   if (c->lean_ring == nullptr || (c->cfg.flags & BLOCKFFN_CFG_TWO_KERNELS)) return false;
   if (with_logits && L > 8) return false;
-  return lean_plan(c->cfg, L, c->num_sms, !with_logits).ok;
+  return lean_plan(c->cfg, L, c->num_sms, shared).ok;
 }
 
 // Three rings (calls that own the device, calls that share it, calls of more than 16 tokens that
@@ -822,13 +822,17 @@ cudaError_t launch_expert_lean(blockffn_ctx* c, const blockffn_weights* w, const
                                const int32_t* n_union, float* out, void* x_next, int call_flags,
                                const RoutingOut* pub, const RouterLogits* logits, bool logits_final,
                                cudaStream_t st) {
-  // Only for calls whose x is stable (for a router-on call: whose router has finished).
-  if (logits ? !logits_final : !(call_flags & BLOCKFFN_CALL_INDEPENDENT_X)) return cudaErrorNotSupported;
-  if (!expert_lean_supported(c, L, logits != nullptr)) return cudaErrorNotSupported;
-  // No router in front: the call consumes nothing of its predecessors and shares the device
+  // For calls whose x is stable (for a router-on call: whose router has finished), and for
+  // chunks of more than 8 tokens in a dependent chain (weights and scores stable, x from the
+  // call before): those wait for their predecessor before they read x.
+  const bool x_stable = logits ? logits_final : (call_flags & BLOCKFFN_CALL_INDEPENDENT_X) != 0;
+  const bool dep = !x_stable && !logits && (call_flags & BLOCKFFN_CALL_INDEPENDENT) && L > 8;
+  if (!x_stable && !dep) return cudaErrorNotSupported;
+  // No router in front and nothing consumed from its predecessors: the call shares the device
   // with them (a router-on call is ordered behind its router by events, which keeps too few of
-  // them in flight for a third of the device each).
-  const bool shared = !logits;
+  // them in flight for a third of the device each; a dependent call runs alone anyway).
+  const bool shared = x_stable && !logits;
+  if (!expert_lean_supported(c, L, logits != nullptr, shared)) return cudaErrorNotSupported;
   const LeanPlan pl = lean_plan(c->cfg, L, c->num_sms, shared);
   if (!pl.ok) return cudaErrorNotSupported;
   LeanParams p{};
@@ -864,6 +868,7 @@ cudaError_t launch_expert_lean(blockffn_ctx* c, const blockffn_weights* w, const
   p.cols_q = pl.cols_q;
   p.cols_rem = pl.cols_rem;
   p.accumulate = (call_flags & BLOCKFFN_CALL_ACCUMULATE) ? 1 : 0;
+  p.dep = dep ? 1 : 0;
   p.hold = (c->cfg.flags & BLOCKFFN_CFG_TEST_EXPIRE_WAIT) ? 1 : 0;
   p.wait_ns = 1000000000ull;      // one second
   p.status = c->status;

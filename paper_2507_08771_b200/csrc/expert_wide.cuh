@@ -179,12 +179,17 @@ expert_wide_kernel(const LeanParams p) {
     }
   };
   // x goes first: its short round trip then runs under the long issue of the weights instead
-  // of behind it
-  load_x();
+  // of behind it. In a dependent chain x is what the call before leaves: the weights (stable)
+  // are requested under that call, then the kernel waits for it and reads x.
+  if (!p.dep) load_x();
 #pragma unroll
   for (int gi = 0; gi < NS; ++gi) {          // one commit group per stage, empty ones included
     if (gi < ngroups) issue_u(gi);
     cp_async_commit();
+  }
+  if (p.dep) {
+    pdl_wait();
+    load_x();
   }
   if (ngroups > 0) prepare(0);
   const int slot = ctl[6];       // (written before the barriers inside derive_union)

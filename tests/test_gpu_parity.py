@@ -183,10 +183,12 @@ def test_expert_ffn(variant, d, E, d_e, L, p):
     (2048, 128, 128, 31, 0.3), (512, 24, 64, 32, 0.5), (2048, 64, 128, 12, 1.0)])
 def test_expert_ffn_under_call_promises(kind, d, E, d_e, L, p):
     """The expert stage under the two per-call promises. With x promised stable the one-kernel form
-    runs a call on a third of the SMs (up to four column tiles of out and several stages per CTA);
-    with only the weights promised stable it owns the device. Shapes cover one to three column
-    tiles, one and several stages, unions from a few experts to all of them, and chunks of 9 to
-    32 tokens (two and four token groups per weight fragment in the one-kernel form)."""
+    runs a call on about a third of the SMs (up to three column tiles of out and several stages per
+    CTA); with only the weights promised stable it owns the device (up to 8 tokens: the up/down
+    pair; longer chunks: the one-kernel form, which then waits for its predecessor before it reads
+    x). Shapes cover one to three column tiles, one and several stages, unions from a few experts
+    to all of them, and chunks of 9 to 32 tokens (two token groups per weight fragment; from 17
+    tokens on two teams of them in one CTA)."""
     seed = 3000 + d + E + L
     sh, w = small_layer(d, E, d_e, seed)
     rng = np.random.default_rng(seed)
@@ -215,10 +217,9 @@ def test_expert_ffn_under_call_promises(kind, d, E, d_e, L, p):
 
 @pytest.mark.parametrize("L", [8, 16, 32])
 def test_stable_x_calls_that_keep_the_whole_device(L):
-    """BLOCKFFN_CFG_NO_SPLIT: calls with stable x get all SMs each. A chunk of more than 16 tokens
-    would then need two CTAs per SM resident at once for its hand-over; where the shared memory
-    of the shape does not allow that the library must take the two-kernel form instead of
-    waiting for CTAs that cannot start."""
+    """BLOCKFFN_CFG_NO_SPLIT: calls with stable x get all SMs each (one 512-thread CTA per SM
+    for more than 16 tokens). The hand-over inside the kernel needs every CTA of a call resident
+    at once; the plan must never pick a grid for which that is not guaranteed."""
     sh, seed = I.SHAPES[2], I.config_seed(2)
     w = I.make_layer(sh, seed, with_router=False)
     layer = B.Layer(sh.d, sh.E, sh.d_e, L_max=32, flags=B.CFG_NO_SPLIT)
@@ -718,11 +719,14 @@ def test_bench_launch_configuration_scores_in(cfg, flag, L):
     assert layer.last_status() == 0
 
 
-def test_bench_launch_configuration_stack():
+@pytest.mark.parametrize("L", [None, 12, 16, 32])
+def test_bench_launch_configuration_stack(L):
     """Config 4 as the benchmark runs it: residual accumulate, bf16 hand-over between layers,
-    CALL_INDEPENDENT on every layer call, one graph; compared with the oracle's stack."""
+    CALL_INDEPENDENT on every layer call, one graph; compared with the oracle's stack. Chunks of
+    more than 8 tokens take the one-kernel form in its dependent-chain mode (it waits for the
+    layer before, then reads x), shorter ones the up/down pair."""
     sh, seed = I.SHAPES[4], I.config_seed(4)
-    n_layers, L = 5, sh.L
+    n_layers, L = (5, sh.L) if L is None else (4, L)
     layer = B.Layer(sh.d, sh.E, sh.d_e, L_max=L)
     ws = [I.make_layer(sh, seed, layer=l, with_router=False) for l in range(n_layers)]
     dws = [layer.upload_weights(w) for w in ws]
