@@ -95,7 +95,7 @@ typedef struct {
  * takes, for those calls too. Same results within the tolerance; kept for comparison.        */
 #define BLOCKFFN_CFG_TWO_KERNELS 0x20000000
 /* The one-kernel form runs a call whose x is promised stable (BLOCKFFN_CALL_INDEPENDENT_X) on
- * a third of the SMs, so that three times as many such calls are in flight: every CTA reads all
+ * about a third of the SMs, so that about three times as many such calls are in flight: every CTA reads all
  * of x and of the intermediate from L2, and fewer, larger CTAs per call keep that broadcast
  * small next to the weight stream. This bit gives those calls the whole device each, like the
  * calls of a dependent chain.                                                              */
@@ -141,7 +141,9 @@ typedef struct {
                                        stable: nothing enqueued on `stream` since the last call made
                                        without this flag (or since the last host synchronisation)
                                        writes them. x and out may still come from the work just
-                                       before. The weight fetch then overlaps the previous kernel.  */
+                                       before. The weight fetch then overlaps the previous kernel
+                                       (a chunk of more than 8 tokens then runs as one kernel that
+                                       waits for that work before it reads x).                      */
 #define BLOCKFFN_CALL_INDEPENDENT_X 4 /* in addition x is stable in the same sense (the chunk does
                                        not consume the previous call's output); implies
                                        BLOCKFFN_CALL_INDEPENDENT. The up projection then runs in full
