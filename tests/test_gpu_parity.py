@@ -380,12 +380,16 @@ def test_bad_union_entries_are_flagged_not_followed():
         assert layer.last_status(clear=True) == B.DEV_BAD_UNION_COUNT
 
 
-def test_bounded_wait_expires_cleanly():
-    """The hand-over inside the one-kernel form (calls whose x is promised stable) is a bounded
-    wait. With the test bit set it waits
+@pytest.mark.parametrize("L,kind", [(8, B.CALL_INDEPENDENT_X), (16, B.CALL_INDEPENDENT_X),
+                                    (32, B.CALL_INDEPENDENT_X), (32, B.CALL_INDEPENDENT)])
+def test_bounded_wait_expires_cleanly(L, kind):
+    """The hand-over inside the one-kernel form (calls whose x is promised stable, and chunks of
+    more than 8 tokens in a dependent chain) is a bounded wait. With the test bit set it waits
     for an arrival that never comes: the call must come back with BLOCKFFN_DEV_WAIT_EXPIRED set,
-    out untouched and the device usable; the next handle (without the bit) works as usual."""
+    out untouched and the device usable; the next handle (without the bit) works as usual.
+    All three kernels of that form are covered: 8 tokens, 16 tokens, 32 tokens (two teams)."""
     sh, seed = I.SHAPES[1], I.config_seed(1)
+    sh = I.Shape(sh.name, d=sh.d, E=sh.E, d_e=sh.d_e, L=L, union_frac=sh.u / sh.E)
     w = I.make_layer(sh, seed, with_router=False)
     x = I.make_x(sh.d, sh.L, seed)
     s = I.make_scores(sh.E, sh.L, sh.u, seed)
@@ -393,13 +397,13 @@ def test_bounded_wait_expires_cleanly():
     dw = held.upload_weights(w)
     out = torch.full((sh.L, sh.d), 7.0, device="cuda")
     for _ in range(2):                                     # the counters stay consistent
-        held.forward_scores(dw, B.to_device_bf16(x), dev(s), out=out, call_flags=B.CALL_INDEPENDENT_X)
+        held.forward_scores(dw, B.to_device_bf16(x), dev(s), out=out, call_flags=kind)
         assert held.last_status(clear=True) == B.DEV_WAIT_EXPIRED
         assert bool((out == 7.0).all())
     assert held.last_status() == 0
     layer = B.Layer(sh.d, sh.E, sh.d_e, L_max=sh.L)
     dw2 = layer.upload_weights(w)
-    res = layer.forward_scores(dw2, B.to_device_bf16(x), dev(s), call_flags=B.CALL_INDEPENDENT_X)
+    res = layer.forward_scores(dw2, B.to_device_bf16(x), dev(s), call_flags=kind)
     ref = oracle.layer_forward_scores(x, s, w["U"], w["D"], union_only=True)
     assert_close(res.out.cpu().numpy(), ref.out, "after an expired wait")
     assert layer.last_status() == 0

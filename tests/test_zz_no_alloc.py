@@ -53,8 +53,12 @@ def test_noalloc_matches_handle_based_entry_point_twice_in_a_row():
         B.blockffn_expert_ffn(layer.h, dw.struct, xd, sd, L, idd, nd, want)
         got = torch.full((L, d), float("nan"), device="cuda")
         nxt = torch.zeros(L, d, dtype=torch.bfloat16, device="cuda")
+        torch.cuda.synchronize()
+        free_before = torch.cuda.mem_get_info()[0]
         B.blockffn_expert_ffn_noalloc(cfg, dw.struct, xd, sd, L, idd, nd, got, x_next=nxt)
         torch.cuda.synchronize()
+        if call > 0:      # (the first call on a device may make the driver load the library's image)
+            assert torch.cuda.mem_get_info()[0] >= free_before, "the call took device memory"
         g, wnt = got.cpu().numpy(), want.cpu().numpy()
         rms = float(np.sqrt(np.mean(ref ** 2)))
         assert np.isfinite(g).all()
