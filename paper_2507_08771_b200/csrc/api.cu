@@ -36,7 +36,7 @@ cudaError_t launch_tensor_core(blockffn_ctx* c, const blockffn_weights* w, const
   // which keeps its weights in shared memory for all tokens at once.
   const bool x_stable = logits ? logits_final : (call_flags & BLOCKFFN_CALL_INDEPENDENT_X) != 0;
   const bool dep_long = !x_stable && !logits && (call_flags & BLOCKFFN_CALL_INDEPENDENT) && L > 8;
-  if ((x_stable || dep_long) && expert_lean_supported(c, L, logits != nullptr, x_stable && !logits))
+  if ((x_stable || dep_long) && expert_lean_supported(c, L, logits != nullptr, x_stable))
     return launch_expert_lean(c, w, x, scores, L, union_ids, n_union, out, x_next, call_flags, pub,
                               logits, logits_final, st);
   return launch_expert_mma(c, w, x, scores, L, union_ids, n_union, out, x_next, call_flags, pub,
@@ -300,6 +300,7 @@ blockffn_status blockffn_layer_forward(blockffn_handle h, const blockffn_weights
     bool capturing = false;
     unsigned long long cap_id = 0;
     const bool marks = x_stable && chained && h->side && capture_state(st, &capturing, &cap_id);
+    cudaStream_t side = h->side;
     const auto& prev = h->call_mark[oldest];
     const bool aside = marks && prev.set && prev.stream == st && prev.capturing == capturing &&
                        prev.id == cap_id;
@@ -311,10 +312,10 @@ blockffn_status blockffn_layer_forward(blockffn_handle h, const blockffn_weights
       h->call_mark[b].id = cap_id;
     }
     if (aside) {
-      if (cudaStreamWaitEvent(h->side, h->ev_call[oldest], 0) != cudaSuccess ||
+      if (cudaStreamWaitEvent(side, h->ev_call[oldest], 0) != cudaSuccess ||
           launch_router(h, w, x, L, h->scores, h->tok_mask, false, nullptr, true, logits, 2,
-                        h->side) != cudaSuccess ||
-          cudaEventRecord(h->ev_router[b], h->side) != cudaSuccess ||
+                        side) != cudaSuccess ||
+          cudaEventRecord(h->ev_router[b], side) != cudaSuccess ||
           cudaStreamWaitEvent(st, h->ev_router[b], 0) != cudaSuccess)
         return BLOCKFFN_ERR_CUDA;
       h->last_layer_waited_first = false;

@@ -845,10 +845,10 @@ cudaError_t launch_expert_lean(blockffn_ctx* c, const blockffn_weights* w, const
   const bool x_stable = logits ? logits_final : (call_flags & BLOCKFFN_CALL_INDEPENDENT_X) != 0;
   const bool dep = !x_stable && !logits && (call_flags & BLOCKFFN_CALL_INDEPENDENT) && L > 8;
   if (!x_stable && !dep) return cudaErrorNotSupported;
-  // No router in front and nothing consumed from its predecessors: the call shares the device
-  // with them (a router-on call is ordered behind its router by events, which keeps too few of
-  // them in flight for a third of the device each; a dependent call runs alone anyway).
-  const bool shared = x_stable && !logits;
+  // Nothing consumed from its predecessors: the call shares the device with them (a router-on
+  // call is ordered behind its own router by an event, and the routers run far enough ahead on
+  // streams of the handle's own); a dependent call runs alone anyway.
+  const bool shared = x_stable;
   if (!expert_lean_supported(c, L, logits != nullptr, shared)) return cudaErrorNotSupported;
   const LeanPlan pl = lean_plan(c->cfg, L, c->num_sms, shared);
   if (!pl.ok) return cudaErrorNotSupported;

@@ -39,8 +39,13 @@ def assert_close(got, ref, what=""):
 
 
 def same_up_to_summation_order(a, b):
-    """Two results of the same call from launch configurations that sum in different orders."""
-    return bool(np.isfinite(a).all() and np.abs(a.astype(np.float64) - b).max() <= 1e-4 * rms(b))
+    """Two results of the same call from launch configurations that sum in different orders. The
+    fp32 sums differ by about 1e-6 of the RMS; where the sum behind an element of the bf16
+    intermediate lands on the other side of a rounding boundary that element moves by one bf16
+    step (2^-8 relative), which shows as a few 1e-4 of the RMS in the outputs it feeds. 1e-3
+    covers a handful of such elements and is still twenty times tighter than the tolerance
+    against the oracle."""
+    return bool(np.isfinite(a).all() and np.abs(a.astype(np.float64) - b).max() <= 1e-3 * rms(b))
 
 
 def dev(a, dtype=None):
