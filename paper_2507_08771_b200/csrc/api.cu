@@ -128,7 +128,7 @@ blockffn_status blockffn_create(const blockffn_config* cfg, blockffn_handle* out
   const size_t o_h16 = take(expert_mma_h_bytes(cfg));
   const size_t lean_bytes = expert_lean_ws_bytes(cfg, c->num_sms);
   const size_t o_lean = take(lean_bytes);
-  const size_t o_seq = take(sizeof(unsigned long long) * 96);
+  const size_t o_seq = take(sizeof(unsigned long long) * 256);   // four rings, 64 words each
   const size_t o_one = take(sizeof(float) * E);
   const size_t o_tk = take(sizeof(unsigned int) * 8);
   const size_t o_st = take(sizeof(uint32_t));
@@ -282,6 +282,19 @@ blockffn_status blockffn_layer_forward(blockffn_handle h, const blockffn_weights
     // publishes scores, masks, union and counters.
     // Successive calls cycle through kLogitRing logit buffers: a router that runs under earlier
     // calls never writes what their kernels still read.
+    const bool x_stable_call = (call_flags & BLOCKFFN_CALL_INDEPENDENT_X) != 0;
+    if (x_stable_call && expert_lean_supported(h, L, true, true)) {
+      // x is stable and the shape takes the one-kernel form: the router runs inside that kernel
+      // (its CTAs share the experts' logits out between them and exchange them through L2), so
+      // the call is one launch that overlaps its neighbours like a scores-in call.
+      const RoutingOut pub_in{h->union_mask, h->union_ids, h->n_union, stats, h->scores, h->tok_mask};
+      const RouterLogits lg_in{nullptr, router_gain(h, w), h->cfg.rms_eps};
+      h->last_layer_waited_first = false;
+      return launch_tensor_core(h, w, x, h->scores, L, nullptr, nullptr, out, x_next, flags, &pub_in,
+                                &lg_in, true, st) == cudaSuccess
+                 ? BLOCKFFN_OK
+                 : BLOCKFFN_ERR_CUDA;
+    }
     const int b = h->a0_phase;
     const int oldest = (b + 1) % kLogitRing;   // the call kLogitRing - 1 calls back
     h->a0_phase = oldest;

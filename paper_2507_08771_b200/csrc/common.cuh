@@ -43,9 +43,11 @@ struct blockffn_ctx {
   int32_t* n_union;     // [1]
   float* h32;           // [E][L_max][d_e] fp32 intermediate (SIMT variant)
   void* h16;            // bf16 intermediate (MMA variant), slot-major padded rows
-  void* lean_ring;      // ring of bf16 intermediates of the one-kernel form (NULL: not used)
-  unsigned long long* lean_seq;   // per ring (three of them, 32 words apart): [0] call tickets,
-                                  // [1 .. 16] arrival counters of the ring slots
+  void* lean_ring;      // rings of bf16 intermediates of the one-kernel form, then its rings of
+                        // router logits (NULL: not used)
+  unsigned long long* lean_seq;   // per ring (four of them, 64 words apart): [0] call tickets,
+                                  // [1 .. 16] arrival counters of the ring slots, [17 .. 32] those
+                                  // of the logit hand-over when the router runs inside the kernel
   float* ones;          // [E] of 1.0f: the gain of the router without RMSNorm
   unsigned int* ticket; // last-block-done counters [8]
   uint32_t* status;     // sticky device status word

@@ -44,7 +44,7 @@
 // its arrival counter is an exact multiple of the call's CTA count when a call starts: the
 // counters only ever grow, nothing is reset, graph replays need no host state. A ticket
 // identifies a call only if every call drawing from the counter has the same number of CTAs, so
-// each kind of call (whole device; a third of it; a third of it with two teams per CTA) has a
+// each kind of call (whole device; part of it with up to 8, up to 16, up to 32 tokens) has a
 // ring and a counter of its own. The hand-over also needs all CTAs of a call resident at once:
 // lean_plan refuses grids for which that is not guaranteed.
 // The polling thread issues no asynchronous copies: a fence or an acquire by a thread waits
@@ -54,6 +54,7 @@
 namespace {
 
 constexpr int kHRing = 16;           // h buffers and arrival counters per ring (see the bound above)
+constexpr int kRings = 4;            // kinds of calls that count their own tickets (see below)
 constexpr int kMinSmem = 60 * 1024;  // four such CTAs do not fit one SM (228 KB, 1 KB reserved each)
 constexpr int kSyncThread = kThreads - 1;
 constexpr int kCopyThreads = kThreads - 32;   // the last warp (the polling thread's) issues no D copies
@@ -94,10 +95,15 @@ struct LeanParams {
   RouterLogits lg;
   const int32_t* ids_in;
   const int32_t* n_in;
+  const uint16_t* W_r;     // MODE 3: router weight bf16 [E][d], bias f32 [E] or NULL (Eq. 3)
+  const float* bias;
+  float* logit_ring;       // MODE 3: kHRing buffers of logit_slot floats, each f32 [L][E]
+  size_t logit_slot;
   uint16_t* h_ring;        // kHRing buffers of h_slot elements, each bf16 [q][L][d_e]
   size_t h_slot;
   unsigned long long* seq;     // tickets: one per CTA per call
   unsigned long long* ready;   // [kHRing] arrivals, never reset
+  unsigned long long* ready2;  // MODE 3: [kHRing] arrivals of the logit hand-over, likewise
   float* out;
   uint16_t* x_next;
   int L, d, E, d_e, de_shift;
@@ -184,8 +190,14 @@ __device__ __forceinline__ void mma64(float (&c0)[4], float (&c1)[4], const uint
 }
 
 // KB: 64-wide k blocks of x per warp (ceil(d / 512)); NC: 16-column tiles of out per CTA
-// (1 .. 4); MODE as derive_union. Everything the call reads is stable (x included): nothing
-// waits for the kernel before it until out is touched.
+// (1 .. 4); MODE as derive_union, or 3: the router runs inside the kernel (Eq. 3). CTA b then
+// computes the logits of experts b, b + grid, ... for all tokens (the arithmetic of the router
+// kernel: one 16-byte piece of the rows per thread, fp32 FMAs, warp shuffles, the eight warp sums
+// added in order), stores them in the call's slot of a ring of logit buffers, arrives on that
+// slot's counter and waits (bounded) until all CTAs of the call have: a first hand-over of the
+// same kind as the one for h. Then every CTA finishes Eq. 3 as in MODE 2.
+// Everything the call reads is stable (x included): nothing waits for the kernel before it
+// until out is touched.
 template <int KB, int NC, int MODE>
 __global__ void __launch_bounds__(kThreads, 3) expert_lean_kernel(const LeanParams p) {
   extern __shared__ __align__(128) unsigned char smem[];
@@ -218,8 +230,77 @@ __global__ void __launch_bounds__(kThreads, 3) expert_lean_kernel(const LeanPara
   // With the caller's union list the scores are first read when the first stage is finished:
   // their lines are requested now, or that read waits for DRAM in the middle of the up projection.
   if constexpr (MODE == 1) prefetch_l2(p.scores, L * p.E * 4);
-  const int nu = derive_union<MODE>(p.scores, p.lg, p.ids_in, p.n_in, L, p.E, ids_sm, ctl,
-                                    reinterpret_cast<uint32_t*>(red), on_ticket);
+  RouterLogits lg = p.lg;
+  if constexpr (MODE == 3) {
+    if (tid == 0) on_ticket();
+    __syncthreads();
+    const int rslot = ctl[6];
+    float* a0 = p.logit_ring + (size_t)rslot * p.logit_slot;
+    lg.a0 = a0;
+    const int chunks = d >> 3;                 // 16-byte pieces of a row (<= 256: one per thread)
+    float* wsum = red;                         // [8 warps][8 tokens]
+    for (int e = bx; e < p.E; e += G) {
+      float acc[8];
+#pragma unroll
+      for (int t = 0; t < 8; ++t) acc[t] = 0.0f;
+      if (tid < chunks) {
+        const uint4 wv = __ldg(reinterpret_cast<const uint4*>(p.W_r + (size_t)e * d) + tid);
+        const uint32_t wp[4] = {wv.x, wv.y, wv.z, wv.w};
+        uint4 xv[8];
+#pragma unroll
+        for (int t = 0; t < 8; ++t)
+          xv[t] = t < L ? __ldcg(reinterpret_cast<const uint4*>(p.x + (size_t)t * d) + tid)
+                        : make_uint4(0u, 0u, 0u, 0u);
+#pragma unroll
+        for (int t = 0; t < 8; ++t) {
+          const uint32_t xp[4] = {xv[t].x, xv[t].y, xv[t].z, xv[t].w};
+#pragma unroll
+          for (int q = 0; q < 4; ++q) {
+            acc[t] = fmaf(bf16_lo(wp[q]), bf16_lo(xp[q]), acc[t]);
+            acc[t] = fmaf(bf16_hi(wp[q]), bf16_hi(xp[q]), acc[t]);
+          }
+        }
+      }
+#pragma unroll
+      for (int t = 0; t < 8; ++t) {
+        float v = acc[t];
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+        if (lane == 0) wsum[warp * 8 + t] = v;
+      }
+      __syncthreads();
+      if (tid < L) {
+        float v = p.bias ? p.bias[e] : 0.0f;
+#pragma unroll
+        for (int w8 = 0; w8 < kWarps; ++w8) v += wsum[w8 * 8 + tid];
+        a0[(size_t)tid * p.E + e] = v;
+      }
+      __syncthreads();
+    }
+    if (tid == kSyncThread) {
+      __threadfence();
+      asm volatile("red.relaxed.gpu.global.add.u64 [%0], 1;" ::"l"(p.ready2 + rslot) : "memory");
+      const unsigned long long target = *reinterpret_cast<const unsigned long long*>(ctl + 138);
+      const unsigned long long t0 = global_ns();
+      const unsigned long long limit = p.hold ? 2000000ull : p.wait_ns;
+      while (ld_acquire_u64(p.ready2 + rslot) < target) {
+        if (global_ns() - t0 > limit) {
+          ctl[5] = 1;
+          atomicOr(p.status, BLOCKFFN_DEV_WAIT_EXPIRED);
+          break;
+        }
+      }
+    }
+    __syncthreads();
+  }
+  int nu_;
+  if constexpr (MODE == 3)       // (the dependents were released above)
+    nu_ = derive_union<2>(p.scores, lg, p.ids_in, p.n_in, L, p.E, ids_sm, ctl,
+                          reinterpret_cast<uint32_t*>(red));
+  else
+    nu_ = derive_union<MODE>(p.scores, lg, p.ids_in, p.n_in, L, p.E, ids_sm, ctl,
+                             reinterpret_cast<uint32_t*>(red), on_ticket);
+  const int nu = nu_;
 
   // ---- up projection ---------------------------------------------------------------------
   const int R = nu * d_e;
@@ -300,10 +381,10 @@ __global__ void __launch_bounds__(kThreads, 3) expert_lean_kernel(const LeanPara
       const int hq = (ra + m) >> sh;
       hidx = (hq * L + t) * d_e + (ra + m - (hq << sh));
       const int id = ids_sm[hq];
-      if constexpr (MODE == 2) {
-        float v = __ldcg(p.lg.a0 + t * p.E + id);
+      if constexpr (MODE >= 2) {
+        float v = __ldcg(lg.a0 + t * p.E + id);
         v = v > 0.0f ? v : 0.0f;
-        sc = __ldg(p.lg.gain + id) * v * reinterpret_cast<const float*>(ctl + 104)[t];
+        sc = __ldg(lg.gain + id) * v * reinterpret_cast<const float*>(ctl + 104)[t];
       } else {
         sc = __ldcg(p.scores + t * p.E + id);
       }
@@ -411,6 +492,10 @@ __global__ void __launch_bounds__(kThreads, 3) expert_lean_kernel(const LeanPara
   if (tid == kSyncThread) {
     __threadfence();
     asm volatile("red.relaxed.gpu.global.add.u64 [%0], 1;" ::"l"(p.ready + slot) : "memory");
+    // the counters of the logit hand-over advance in step with these, whether or not the call
+    // has one: a slot's two counters then always agree on how often the slot has been used
+    if constexpr (MODE != 3)
+      asm volatile("red.relaxed.gpu.global.add.u64 [%0], 1;" ::"l"(p.ready2 + slot) : "memory");
   }
 
   // ---- down projection -------------------------------------------------------------------
@@ -573,7 +658,7 @@ __global__ void __launch_bounds__(kThreads, 3) expert_lean_kernel(const LeanPara
   }
   // CTA 0 publishes the routing it derived (after the wait: earlier readers are done)
   if (blockIdx.x == 0) {
-    if (p.lg.a0 != nullptr && p.pub_scores != nullptr) {
+    if (lg.a0 != nullptr && p.pub_scores != nullptr) {
       const int words = (p.E + 31) >> 5;
       const float* rinv = reinterpret_cast<const float*>(ctl + 104);
       for (int t = warp; t < L; t += kWarps) {
@@ -581,9 +666,9 @@ __global__ void __launch_bounds__(kThreads, 3) expert_lean_kernel(const LeanPara
           const int e = 32 * w + lane;
           float sv = 0.0f;
           if (e < p.E) {
-            float v = __ldcg(p.lg.a0 + (size_t)t * p.E + e);
+            float v = __ldcg(lg.a0 + (size_t)t * p.E + e);
             v = v > 0.0f ? v : 0.0f;
-            sv = __ldg(p.lg.gain + e) * v * rinv[t];
+            sv = __ldg(lg.gain + e) * v * rinv[t];
             p.pub_scores[(size_t)t * p.E + e] = sv;
           }
           const uint32_t m = __ballot_sync(0xffffffffu, sv != 0.0f);
@@ -746,9 +831,11 @@ LeanPlan lean_plan(const blockffn_config& cfg, int L, int sms, bool shared) {
 
 template <int KB, int NC, int NTG, int MODE, int TEAMS = 1>
 cudaError_t lean_attr() {
-  const void* f = NTG == 1 ? reinterpret_cast<const void*>(&expert_lean_kernel<KB, NC, MODE>)
-                           : reinterpret_cast<const void*>(
-                                 &expert_wide_kernel<KB, NC, NTG == 1 ? 2 : NTG, MODE, TEAMS>);
+  const void* f;
+  if constexpr (NTG == 1)
+    f = reinterpret_cast<const void*>(&expert_lean_kernel<KB, NC, MODE>);
+  else
+    f = reinterpret_cast<const void*>(&expert_wide_kernel<KB, NC, NTG, MODE, TEAMS>);
   cudaError_t e = cudaFuncSetAttribute(f, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemMax);
   if (e != cudaSuccess) return e;
   return cudaFuncSetAttribute(f, cudaFuncAttributePreferredSharedMemoryCarveout,
@@ -759,6 +846,7 @@ cudaError_t lean_attrs_kb() {
   cudaError_t e = lean_attr<KB, NC, 1, 0>();
   if (e == cudaSuccess) e = lean_attr<KB, NC, 1, 1>();
   if (e == cudaSuccess) e = lean_attr<KB, NC, 1, 2>();
+  if (e == cudaSuccess) e = lean_attr<KB, NC, 1, 3>();
   if (e == cudaSuccess) e = lean_attr<KB, NC, 2, 0>();
   if (e == cudaSuccess) e = lean_attr<KB, NC, 2, 1>();
   if (e == cudaSuccess) e = lean_attr<KB, NC, 2, 0, 2>();
@@ -770,10 +858,11 @@ template <int KB, int NC>
 cudaError_t lean_launch_kb(const cudaLaunchConfig_t& lc, const LeanParams& p, int ntg, int teams,
                            int mode) {
   if (ntg == 1)
-    return mode == 2   ? cudaLaunchKernelEx(&lc, expert_lean_kernel<KB, NC, 2>, p)
+    return mode == 3   ? cudaLaunchKernelEx(&lc, expert_lean_kernel<KB, NC, 3>, p)
+           : mode == 2 ? cudaLaunchKernelEx(&lc, expert_lean_kernel<KB, NC, 2>, p)
            : mode == 1 ? cudaLaunchKernelEx(&lc, expert_lean_kernel<KB, NC, 1>, p)
                        : cudaLaunchKernelEx(&lc, expert_lean_kernel<KB, NC, 0>, p);
-  if (mode == 2) return cudaErrorNotSupported;
+  if (mode >= 2) return cudaErrorNotSupported;
   if (teams == 2)
     return mode == 1 ? cudaLaunchKernelEx(&lc, expert_wide_kernel<KB, NC, 2, 1, 2>, p)
                      : cudaLaunchKernelEx(&lc, expert_wide_kernel<KB, NC, 2, 0, 2>, p);
@@ -791,6 +880,11 @@ cudaError_t lean_launch_nc(int kb, const cudaLaunchConfig_t& lc, const LeanParam
   }
 }
 
+// (router inside the kernel) the logits of a chunk: f32 [L_max][E]; the logit rings follow the
+// h rings in the workspace
+size_t lean_logit_slot_bytes(const blockffn_config& cfg) {
+  return ((size_t)cfg.L_max * cfg.E * sizeof(float) + 255) & ~(size_t)255;
+}
 size_t lean_h_slot_bytes(const blockffn_config& cfg) {
   return ((size_t)cfg.E * cfg.L_max * cfg.d_e * sizeof(uint16_t) + 255) & ~(size_t)255;
 }
@@ -805,16 +899,16 @@ bool expert_lean_supported(const blockffn_ctx* c, int L, bool with_logits, bool 
   return lean_plan(c->cfg, L, c->num_sms, shared).ok;
 }
 
-// Three rings (calls that own the device, calls that share it, calls of more than 16 tokens that
-// share it: each kind counts its own tickets) of kHRing intermediates of a
+// Four rings (calls that own the device; calls that share it with up to 8, up to 16, up to 32
+// tokens: their grids differ, so each kind counts its own tickets) of kHRing intermediates of a
 // chunk of L_max tokens; 0 when the shape never takes this kernel (or the rings would be
 // unreasonably large).
 size_t expert_lean_ws_bytes(const blockffn_config* cfg, int sms) {
   const int L = cfg->L_max < 8 ? cfg->L_max : 8;
   if (!lean_plan(*cfg, L, sms, false).ok || !lean_plan(*cfg, L, sms, true).ok) return 0;
-  const size_t slot = lean_h_slot_bytes(*cfg);
-  if (3 * kHRing * slot > ((size_t)256 << 20)) return 0;
-  return 3 * kHRing * slot;
+  const size_t slot = lean_h_slot_bytes(*cfg) + lean_logit_slot_bytes(*cfg);
+  if (kRings * kHRing * slot > ((size_t)256 << 20)) return 0;
+  return kRings * kHRing * slot;
 }
 
 cudaError_t expert_lean_setup(blockffn_ctx* c) {
@@ -858,15 +952,24 @@ cudaError_t launch_expert_lean(blockffn_ctx* c, const blockffn_weights* w, const
   p.D = static_cast<const uint16_t*>(w->D);
   p.scores = scores;
   if (logits) p.lg = *logits;
+  const bool router_inside = logits && logits->a0 == nullptr;
+  if (router_inside && (L > 8 || !w->W_r)) return cudaErrorNotSupported;
+  p.W_r = static_cast<const uint16_t*>(w->W_r);
+  p.bias = w->bias;
   p.ids_in = union_ids;
   p.n_in = n_union;
   p.h_slot = lean_h_slot_bytes(c->cfg) / 2;
   // a ring and a ticket counter per kind of call: tickets only identify a call when every call
   // that draws from the counter has the same number of CTAs
-  const int ring = !shared ? 0 : pl.teams == 1 ? 1 : 2;
+  const int ring = !shared ? 0 : L <= 8 ? 1 : L <= 16 ? 2 : 3;
   p.h_ring = static_cast<uint16_t*>(c->lean_ring) + (size_t)ring * kHRing * p.h_slot;
-  p.seq = c->lean_seq + 32 * ring;
+  p.seq = c->lean_seq + 64 * ring;
   p.ready = p.seq + 1;
+  p.ready2 = p.seq + 1 + kHRing;
+  p.logit_slot = lean_logit_slot_bytes(c->cfg) / sizeof(float);
+  p.logit_ring = reinterpret_cast<float*>(static_cast<char*>(c->lean_ring) +
+                                          kRings * kHRing * lean_h_slot_bytes(c->cfg)) +
+                 (size_t)ring * kHRing * p.logit_slot;
   p.out = out;
   p.x_next = static_cast<uint16_t*>(x_next);
   p.L = L;
@@ -898,7 +1001,7 @@ cudaError_t launch_expert_lean(blockffn_ctx* c, const blockffn_weights* w, const
     p.pub_tok = pub->tok_mask;
   }
   const bool chained = !(c->cfg.flags & BLOCKFFN_CFG_NO_CHAINING);
-  const int mode = logits ? 2 : union_ids ? 1 : 0;
+  const int mode = router_inside ? 3 : logits ? 2 : union_ids ? 1 : 0;
   cudaLaunchAttribute attr[1];
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[0].val.programmaticStreamSerializationAllowed = 1;

@@ -259,6 +259,8 @@ expert_wide_kernel(const LeanParams p) {
   if (tid == kNT - 1) {
     __threadfence();
     asm volatile("red.relaxed.gpu.global.add.u64 [%0], 1;" ::"l"(p.ready + slot) : "memory");
+    // (the slot's counter of the logit hand-over advances in step, see expert_lean_kernel)
+    asm volatile("red.relaxed.gpu.global.add.u64 [%0], 1;" ::"l"(p.ready2 + slot) : "memory");
   }
 
   // ---- down projection -------------------------------------------------------------------

@@ -728,6 +728,32 @@ def test_bench_launch_configuration_scores_in(cfg, flag, L):
     assert layer.last_status() == 0
 
 
+def test_mixed_chunk_lengths_on_one_handle_in_a_graph():
+    """Calls of different chunk lengths, all with stable x, interleaved on one handle and one
+    stream: short, medium and long chunks run on grids of different sizes and must not share a
+    ticket counter or a ring of intermediates. Every call is checked against the oracle."""
+    sh, seed = I.SHAPES[2], I.config_seed(2)
+    w = I.make_layer(sh, seed, with_router=False)
+    layer = B.Layer(sh.d, sh.E, sh.d_e, L_max=32)
+    dw = layer.upload_weights(w)
+    Ls = [8, 12, 32, 4, 16, 8, 17, 1, 32, 12, 8, 8, 24, 9, 2, 16, 8, 32, 5, 12]
+    xs = [I.make_x(sh.d, L, seed, chunk=200 + c) for c, L in enumerate(Ls)]
+    ss = [I.make_scores(sh.E, L, sh.u, seed, chunk=200 + c) for c, L in enumerate(Ls)]
+    xd, sd = [B.to_device_bf16(x) for x in xs], [dev(s_) for s_ in ss]
+    outs = [torch.full((L, sh.d), float("nan"), device="cuda") for L in Ls]
+
+    def enqueue(stream):
+        for c, L in enumerate(Ls):
+            B.blockffn_layer_forward_scores(layer.h, dw.struct, xd[c], sd[c], L, outs[c], None,
+                                            layer.stats, B.CALL_INDEPENDENT_X, stream)
+
+    graph_of(enqueue)
+    assert layer.last_status() == 0
+    for c, L in enumerate(Ls):
+        ref = oracle.layer_forward_scores(xs[c], ss[c], w["U"], w["D"], union_only=True)
+        assert_close(outs[c].cpu().numpy(), ref.out, f"call {c}, L = {L}")
+
+
 @pytest.mark.parametrize("L", [None, 12, 16, 32])
 def test_bench_launch_configuration_stack(L):
     """Config 4 as the benchmark runs it: residual accumulate, bf16 hand-over between layers,
