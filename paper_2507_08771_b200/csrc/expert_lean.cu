@@ -230,13 +230,13 @@ __global__ void __launch_bounds__(kThreads, 3) expert_lean_kernel(const LeanPara
   // With the caller's union list the scores are first read when the first stage is finished:
   // their lines are requested now, or that read waits for DRAM in the middle of the up projection.
   if constexpr (MODE == 1) prefetch_l2(p.scores, L * p.E * 4);
-  RouterLogits lg = p.lg;
+  RouterLogits lg3 = p.lg;       // MODE 3 only: the logits are this call's slot of the logit ring
   if constexpr (MODE == 3) {
     if (tid == 0) on_ticket();
     __syncthreads();
     const int rslot = ctl[6];
     float* a0 = p.logit_ring + (size_t)rslot * p.logit_slot;
-    lg.a0 = a0;
+    lg3.a0 = a0;
     const int chunks = d >> 3;                 // 16-byte pieces of a row (<= 256: one per thread)
     float* wsum = red;                         // [8 warps][8 tokens]
     for (int e = bx; e < p.E; e += G) {
@@ -293,6 +293,8 @@ __global__ void __launch_bounds__(kThreads, 3) expert_lean_kernel(const LeanPara
     }
     __syncthreads();
   }
+  // (the other modes read the kernel parameter where they need it: nothing to keep in registers)
+  const RouterLogits& lg = MODE == 3 ? lg3 : p.lg;
   int nu_;
   if constexpr (MODE == 3)       // (the dependents were released above)
     nu_ = derive_union<2>(p.scores, lg, p.ids_in, p.n_in, L, p.E, ids_sm, ctl,
@@ -494,8 +496,9 @@ __global__ void __launch_bounds__(kThreads, 3) expert_lean_kernel(const LeanPara
     asm volatile("red.relaxed.gpu.global.add.u64 [%0], 1;" ::"l"(p.ready + slot) : "memory");
     // the counters of the logit hand-over advance in step with these, whether or not the call
     // has one: a slot's two counters then always agree on how often the slot has been used
-    if constexpr (MODE != 3)
-      asm volatile("red.relaxed.gpu.global.add.u64 [%0], 1;" ::"l"(p.ready2 + slot) : "memory");
+    static_assert(kHRing * sizeof(unsigned long long) == 128, "offset of ready2 below");
+    if constexpr (MODE != 3)     // (ready2 = ready + kHRing)
+      asm volatile("red.relaxed.gpu.global.add.u64 [%0 + 128], 1;" ::"l"(p.ready + slot) : "memory");
   }
 
   // ---- down projection -------------------------------------------------------------------
