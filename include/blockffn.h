@@ -148,9 +148,9 @@ typedef struct {
                                        not consume the previous call's output); implies
                                        BLOCKFFN_CALL_INDEPENDENT. The up projection then runs in full
                                        under the previous call and only its store waits. In
-                                       blockffn_layer_forward (whose router writes the scores the
-                                       expert stage consumes) the router alone runs ahead: it
-                                       computes the logits under the previous call.                 */
+                                       blockffn_layer_forward the router then runs inside the expert
+                                       kernel (one launch per call) where the shape allows it, else
+                                       ahead of it on a stream of the handle.                       */
 
 typedef struct blockffn_ctx* blockffn_handle;
 
