@@ -778,7 +778,9 @@ def stack_router_on(args, torch, device, peak, layers=None, chunks=16):
                                          lay.stats, B.CALL_ACCUMULATE, stream)
 
     stream = torch.cuda.Stream(device)
+    n0 = lay.launch_count()
     g = capture(torch, stream, enqueue)
+    launches_per_layer = (lay.launch_count() - n0) / (2 * chunks * layers)   # capture() enqueues twice
     ms = time_replays(torch, stream, g, max(3, args.steps // 2), 2)
     assert lay.last_status() == 0
     hs = lay.stats_host()
@@ -786,7 +788,9 @@ def stack_router_on(args, torch, device, peak, layers=None, chunks=16):
     us_layer = ms * 1e3 / (chunks * layers)
     return {"layers": layers, "chunks": chunks, "us_per_layer": us_layer, "mean_union": mean_u,
             "tls": B.blockffn_tls(hs, sh.E), "GBps": mean_u * sh.expert_bytes / us_layer / 1e3,
-            "note": "router on every layer (3 launches per layer: router, up, down); no normalisation between "
+            "launches_per_layer": launches_per_layer,
+            "note": "router on every layer (one kernel per layer with the router inside, or router, up, down where "
+                    "the shape does not take that form); no normalisation between "
                     "layers, down projections scaled by 1/32 so that the hidden state keeps its scale; the union "
                     "is whatever the router derives (mean reported)"}
 

@@ -36,7 +36,9 @@ cudaError_t launch_tensor_core(blockffn_ctx* c, const blockffn_weights* w, const
   // which keeps its weights in shared memory for all tokens at once.
   const bool x_stable = logits ? logits_final : (call_flags & BLOCKFFN_CALL_INDEPENDENT_X) != 0;
   const bool dep_long = !x_stable && !logits && (call_flags & BLOCKFFN_CALL_INDEPENDENT) && L > 8;
-  if ((x_stable || dep_long) && expert_lean_supported(c, L, logits != nullptr, x_stable))
+  const bool dep_inside = !x_stable && logits && logits->a0 == nullptr;   // router inside the kernel
+  if ((x_stable || dep_long || dep_inside) &&
+      expert_lean_supported(c, L, logits != nullptr, x_stable))
     return launch_expert_lean(c, w, x, scores, L, union_ids, n_union, out, x_next, call_flags, pub,
                               logits, logits_final, st);
   return launch_expert_mma(c, w, x, scores, L, union_ids, n_union, out, x_next, call_flags, pub,
@@ -283,15 +285,16 @@ blockffn_status blockffn_layer_forward(blockffn_handle h, const blockffn_weights
     // Successive calls cycle through kLogitRing logit buffers: a router that runs under earlier
     // calls never writes what their kernels still read.
     const bool x_stable_call = (call_flags & BLOCKFFN_CALL_INDEPENDENT_X) != 0;
-    if (x_stable_call && expert_lean_supported(h, L, true, true)) {
-      // x is stable and the shape takes the one-kernel form: the router runs inside that kernel
-      // (its CTAs share the experts' logits out between them and exchange them through L2), so
-      // the call is one launch that overlaps its neighbours like a scores-in call.
+    if (expert_lean_supported(h, L, true, x_stable_call)) {
+      // The shape takes the one-kernel form: the router runs inside that kernel (its CTAs share
+      // the experts' logits out between them and exchange them through L2), so the call is one
+      // launch. With x stable it overlaps its neighbours like a scores-in call; otherwise it
+      // owns the device and waits for the work before it ahead of its first read.
       const RoutingOut pub_in{h->union_mask, h->union_ids, h->n_union, stats, h->scores, h->tok_mask};
       const RouterLogits lg_in{nullptr, router_gain(h, w), h->cfg.rms_eps};
       h->last_layer_waited_first = false;
       return launch_tensor_core(h, w, x, h->scores, L, nullptr, nullptr, out, x_next, flags, &pub_in,
-                                &lg_in, true, st) == cudaSuccess
+                                &lg_in, x_stable_call, st) == cudaSuccess
                  ? BLOCKFFN_OK
                  : BLOCKFFN_ERR_CUDA;
     }

@@ -234,6 +234,9 @@ __global__ void __launch_bounds__(kThreads, 3) expert_lean_kernel(const LeanPara
   if constexpr (MODE == 3) {
     if (tid == 0) on_ticket();
     __syncthreads();
+    // In a dependent chain x (and, without any promise, everything else) is what the call
+    // before leaves: nothing has been read so far, and nothing is before that call is done.
+    if (p.dep) pdl_wait();
     const int rslot = ctl[6];
     float* a0 = p.logit_ring + (size_t)rslot * p.logit_slot;
     lg3.a0 = a0;
@@ -939,8 +942,12 @@ cudaError_t launch_expert_lean(blockffn_ctx* c, const blockffn_weights* w, const
   // For calls whose x is stable (for a router-on call: whose router has finished), and for
   // chunks of more than 8 tokens in a dependent chain (weights and scores stable, x from the
   // call before): those wait for their predecessor before they read x.
+  // A router-on call of up to 8 tokens whose router runs inside the kernel (logits->a0 == NULL)
+  // may be dependent as well, with or without promises: it waits before it reads anything.
+  const bool inside = logits && logits->a0 == nullptr;
   const bool x_stable = logits ? logits_final : (call_flags & BLOCKFFN_CALL_INDEPENDENT_X) != 0;
-  const bool dep = !x_stable && !logits && (call_flags & BLOCKFFN_CALL_INDEPENDENT) && L > 8;
+  const bool dep = !x_stable &&
+                   (inside || (!logits && (call_flags & BLOCKFFN_CALL_INDEPENDENT) && L > 8));
   if (!x_stable && !dep) return cudaErrorNotSupported;
   // Nothing consumed from its predecessors: the call shares the device with them (a router-on
   // call is ordered behind its own router by an event, and the routers run far enough ahead on
@@ -955,7 +962,7 @@ cudaError_t launch_expert_lean(blockffn_ctx* c, const blockffn_weights* w, const
   p.D = static_cast<const uint16_t*>(w->D);
   p.scores = scores;
   if (logits) p.lg = *logits;
-  const bool router_inside = logits && logits->a0 == nullptr;
+  const bool router_inside = inside;
   if (router_inside && (L > 8 || !w->W_r)) return cudaErrorNotSupported;
   p.W_r = static_cast<const uint16_t*>(w->W_r);
   p.bias = w->bias;
