@@ -441,14 +441,18 @@ def test_host_side_argument_errors():
     B.Layer(264, 9, 72, L_max=8, variant=B.VARIANT_AUTO)                # AUTO picks the other family
 
 
+@pytest.mark.parametrize("form", [0, B.CFG_TWO_KERNELS])
 @pytest.mark.parametrize("flag", [0, B.CALL_INDEPENDENT_X])
-def test_bench_launch_configuration_router_on(flag):
-    """Back-to-back blockffn_layer_forward calls in a graph; with the promise set the router of a
-    call runs under the expert kernels of the call before it (alternating logit buffers)."""
+def test_bench_launch_configuration_router_on(flag, form):
+    """Back-to-back blockffn_layer_forward calls in a graph. One-kernel form: the router runs
+    inside the expert kernel (with the promise the calls overlap, without it each waits for the
+    one before). Two-kernel form: with the promise the router of a call runs on a stream of the
+    handle, several calls ahead of its expert kernels (a ring of logit buffers, marks and events
+    that become graph edges); without it the router stays on the caller's stream."""
     sh, seed = I.SHAPES[3], I.config_seed(3)
     n_chunks, n_copies = 13, 3                             # odd: replays meet on the same buffer
     w = I.make_layer(sh, seed, bias_shift=I.ROUTER_BIAS_SHIFT)
-    layer = B.Layer(sh.d, sh.E, sh.d_e, L_max=sh.L)
+    layer = B.Layer(sh.d, sh.E, sh.d_e, L_max=sh.L, flags=form)
     dws = [layer.upload_weights(w) for _ in range(n_copies)]
     xs = [I.make_x(sh.d, sh.L, seed, chunk=c) for c in range(n_chunks)]
     xd = [B.to_device_bf16(x) for x in xs]
@@ -468,7 +472,7 @@ def test_bench_launch_configuration_router_on(flag):
     # chunk; it is checked against the oracle (flips only inside the band, else the oracle FFN
     # driven by the library's scores), and the overlapped run must reproduce it up to the order
     # of the fp32 sums (a call that shares the device splits its columns and experts differently
-    # from one that owns it; the bf16 intermediate is the same bits either way).
+    # from one that owns it).
     for c in range(n_chunks):
         alone = check_layer_router_on(layer, dws[c % n_copies], w, xs[c], sh.L, bias=w.get("bias"),
                                       want_out=True)
