@@ -38,7 +38,7 @@ cudaError_t launch_tensor_core(blockffn_ctx* c, const blockffn_weights* w, const
   const bool dep_long = !x_stable && !logits && (call_flags & BLOCKFFN_CALL_INDEPENDENT) && L > 8;
   const bool dep_inside = !x_stable && logits && logits->a0 == nullptr;   // router inside the kernel
   if ((x_stable || dep_long || dep_inside) &&
-      expert_lean_supported(c, L, logits != nullptr, x_stable))
+      expert_lean_supported(c, L, logits != nullptr, x_stable, logits && logits->a0 == nullptr))
     return launch_expert_lean(c, w, x, scores, L, union_ids, n_union, out, x_next, call_flags, pub,
                               logits, logits_final, st);
   return launch_expert_mma(c, w, x, scores, L, union_ids, n_union, out, x_next, call_flags, pub,
@@ -285,7 +285,7 @@ blockffn_status blockffn_layer_forward(blockffn_handle h, const blockffn_weights
     // Successive calls cycle through kLogitRing logit buffers: a router that runs under earlier
     // calls never writes what their kernels still read.
     const bool x_stable_call = (call_flags & BLOCKFFN_CALL_INDEPENDENT_X) != 0;
-    if (expert_lean_supported(h, L, true, x_stable_call)) {
+    if (expert_lean_supported(h, L, true, x_stable_call, true)) {
       // The shape takes the one-kernel form: the router runs inside that kernel (its CTAs share
       // the experts' logits out between them and exchange them through L2), so the call is one
       // launch. With x stable it overlaps its neighbours like a scores-in call; otherwise it

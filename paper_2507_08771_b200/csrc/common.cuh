@@ -109,7 +109,8 @@ struct RouterLogits {
 
 // One-kernel form of the tensor-core expert stage for chunks of at most 8 tokens (same
 // arguments as launch_expert_mma below).
-bool expert_lean_supported(const blockffn_ctx* c, int L, bool with_logits, bool shared);
+bool expert_lean_supported(const blockffn_ctx* c, int L, bool with_logits, bool shared,
+                           bool inside = false);
 size_t expert_lean_ws_bytes(const blockffn_config* cfg, int grid);
 cudaError_t expert_lean_setup(blockffn_ctx* c);
 cudaError_t launch_expert_lean(blockffn_ctx* c, const blockffn_weights* w, const void* x,

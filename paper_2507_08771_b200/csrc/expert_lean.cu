@@ -857,6 +857,8 @@ cudaError_t lean_attrs_kb() {
   if (e == cudaSuccess) e = lean_attr<KB, NC, 2, 1>();
   if (e == cudaSuccess) e = lean_attr<KB, NC, 2, 0, 2>();
   if (e == cudaSuccess) e = lean_attr<KB, NC, 2, 1, 2>();
+  if (e == cudaSuccess) e = lean_attr<KB, NC, 2, 3>();
+  if (e == cudaSuccess) e = lean_attr<KB, NC, 2, 3, 2>();
   return e;
 }
 
@@ -868,12 +870,14 @@ cudaError_t lean_launch_kb(const cudaLaunchConfig_t& lc, const LeanParams& p, in
            : mode == 2 ? cudaLaunchKernelEx(&lc, expert_lean_kernel<KB, NC, 2>, p)
            : mode == 1 ? cudaLaunchKernelEx(&lc, expert_lean_kernel<KB, NC, 1>, p)
                        : cudaLaunchKernelEx(&lc, expert_lean_kernel<KB, NC, 0>, p);
-  if (mode >= 2) return cudaErrorNotSupported;
+  if (mode == 2) return cudaErrorNotSupported;
   if (teams == 2)
-    return mode == 1 ? cudaLaunchKernelEx(&lc, expert_wide_kernel<KB, NC, 2, 1, 2>, p)
-                     : cudaLaunchKernelEx(&lc, expert_wide_kernel<KB, NC, 2, 0, 2>, p);
-  return mode == 1 ? cudaLaunchKernelEx(&lc, expert_wide_kernel<KB, NC, 2, 1, 1>, p)
-                   : cudaLaunchKernelEx(&lc, expert_wide_kernel<KB, NC, 2, 0, 1>, p);
+    return mode == 3   ? cudaLaunchKernelEx(&lc, expert_wide_kernel<KB, NC, 2, 3, 2>, p)
+           : mode == 1 ? cudaLaunchKernelEx(&lc, expert_wide_kernel<KB, NC, 2, 1, 2>, p)
+                       : cudaLaunchKernelEx(&lc, expert_wide_kernel<KB, NC, 2, 0, 2>, p);
+  return mode == 3   ? cudaLaunchKernelEx(&lc, expert_wide_kernel<KB, NC, 2, 3, 1>, p)
+         : mode == 1 ? cudaLaunchKernelEx(&lc, expert_wide_kernel<KB, NC, 2, 1, 1>, p)
+                     : cudaLaunchKernelEx(&lc, expert_wide_kernel<KB, NC, 2, 0, 1>, p);
 }
 template <int NC>
 cudaError_t lean_launch_nc(int kb, const cudaLaunchConfig_t& lc, const LeanParams& p, int ntg,
@@ -899,9 +903,11 @@ size_t lean_h_slot_bytes(const blockffn_config& cfg) {
 
 // Whether a call of L tokens whose x is stable takes the one-kernel form (with_logits: it comes
 // with raw router logits, i.e. it is the expert stage of a router-on layer call).
-bool expert_lean_supported(const blockffn_ctx* c, int L, bool with_logits, bool shared) {
+// (inside: the logits are computed in the kernel, which every chunk length can; logits from a
+// router kernel are taken by the 8-token kernel only)
+bool expert_lean_supported(const blockffn_ctx* c, int L, bool with_logits, bool shared, bool inside) {
   if (c->lean_ring == nullptr || (c->cfg.flags & BLOCKFFN_CFG_TWO_KERNELS)) return false;
-  if (with_logits && L > 8) return false;
+  if (with_logits && !inside && L > 8) return false;
   return lean_plan(c->cfg, L, c->num_sms, shared).ok;
 }
 
@@ -953,7 +959,7 @@ cudaError_t launch_expert_lean(blockffn_ctx* c, const blockffn_weights* w, const
   // call is ordered behind its own router by an event, and the routers run far enough ahead on
   // streams of the handle's own); a dependent call runs alone anyway.
   const bool shared = x_stable;
-  if (!expert_lean_supported(c, L, logits != nullptr, shared)) return cudaErrorNotSupported;
+  if (!expert_lean_supported(c, L, logits != nullptr, shared, inside)) return cudaErrorNotSupported;
   const LeanPlan pl = lean_plan(c->cfg, L, c->num_sms, shared);
   if (!pl.ok) return cudaErrorNotSupported;
   LeanParams p{};
@@ -963,7 +969,7 @@ cudaError_t launch_expert_lean(blockffn_ctx* c, const blockffn_weights* w, const
   p.scores = scores;
   if (logits) p.lg = *logits;
   const bool router_inside = inside;
-  if (router_inside && (L > 8 || !w->W_r)) return cudaErrorNotSupported;
+  if (router_inside && !w->W_r) return cudaErrorNotSupported;
   p.W_r = static_cast<const uint16_t*>(w->W_r);
   p.bias = w->bias;
   p.ids_in = union_ids;

@@ -60,8 +60,87 @@ expert_wide_kernel(const LeanParams p) {
   };
   // (the caller's union list: the scores are first read at the end of the first stage)
   if constexpr (MODE == 1) prefetch_l2(p.scores, Lf * p.E * 4);
-  const int nu = derive_union<MODE>(p.scores, p.lg, p.ids_in, p.n_in, Lf, p.E, ids_sm, ctl,
-                                    reinterpret_cast<uint32_t*>(red0), on_ticket);
+  // MODE 3: the router inside the kernel, as in expert_lean_kernel, 8 tokens per pass. The
+  // first 8 warps of the CTA do it (a row has at most 256 pieces of 16 bytes).
+  RouterLogits lg3 = p.lg;
+  if constexpr (MODE == 3) {
+    if (tid == 0) on_ticket();
+    __syncthreads();
+    if (p.dep) pdl_wait();
+    const int rslot = ctl[6];
+    float* a0 = p.logit_ring + (size_t)rslot * p.logit_slot;
+    lg3.a0 = a0;
+    const int chunks = d >> 3;
+    float* wsum = red0;                        // [8 warps][8 tokens]
+    const int w8 = tid >> 5;                   // warp of the CTA
+    for (int e = bx; e < p.E; e += G) {
+      uint4 wv = make_uint4(0u, 0u, 0u, 0u);
+      if (tid < chunks) wv = __ldg(reinterpret_cast<const uint4*>(p.W_r + (size_t)e * d) + tid);
+      const uint32_t wp[4] = {wv.x, wv.y, wv.z, wv.w};
+      for (int t0 = 0; t0 < Lf; t0 += 8) {
+        float acc[8];
+#pragma unroll
+        for (int t = 0; t < 8; ++t) acc[t] = 0.0f;
+        if (tid < chunks) {
+          uint4 xv[8];
+#pragma unroll
+          for (int t = 0; t < 8; ++t)
+            xv[t] = t0 + t < Lf ? __ldcg(reinterpret_cast<const uint4*>(p.x + (size_t)(t0 + t) * d) + tid)
+                                : make_uint4(0u, 0u, 0u, 0u);
+#pragma unroll
+          for (int t = 0; t < 8; ++t) {
+            const uint32_t xp[4] = {xv[t].x, xv[t].y, xv[t].z, xv[t].w};
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+              acc[t] = fmaf(bf16_lo(wp[q]), bf16_lo(xp[q]), acc[t]);
+              acc[t] = fmaf(bf16_hi(wp[q]), bf16_hi(xp[q]), acc[t]);
+            }
+          }
+        }
+        if (w8 < kWarps) {
+#pragma unroll
+          for (int t = 0; t < 8; ++t) {
+            float v = acc[t];
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+            if (lane == 0) wsum[w8 * 8 + t] = v;
+          }
+        }
+        __syncthreads();
+        if (tid < 8 && t0 + tid < Lf) {
+          float v = p.bias ? p.bias[e] : 0.0f;
+#pragma unroll
+          for (int q = 0; q < kWarps; ++q) v += wsum[q * 8 + tid];
+          a0[(size_t)(t0 + tid) * p.E + e] = v;
+        }
+        __syncthreads();
+      }
+    }
+    if (tid == kNT - 1) {
+      __threadfence();
+      asm volatile("red.relaxed.gpu.global.add.u64 [%0], 1;" ::"l"(p.ready2 + rslot) : "memory");
+      const unsigned long long target = *reinterpret_cast<const unsigned long long*>(ctl + 138);
+      const unsigned long long t0 = global_ns();
+      const unsigned long long limit = p.hold ? 2000000ull : p.wait_ns;
+      while (ld_acquire_u64(p.ready2 + rslot) < target) {
+        if (global_ns() - t0 > limit) {
+          ctl[5] = 1;
+          atomicOr(p.status, BLOCKFFN_DEV_WAIT_EXPIRED);
+          break;
+        }
+      }
+    }
+    __syncthreads();
+  }
+  const RouterLogits& lg = MODE == 3 ? lg3 : p.lg;
+  int nu_;
+  if constexpr (MODE == 3)
+    nu_ = derive_union<2>(p.scores, lg, p.ids_in, p.n_in, Lf, p.E, ids_sm, ctl,
+                          reinterpret_cast<uint32_t*>(red0));
+  else
+    nu_ = derive_union<MODE>(p.scores, lg, p.ids_in, p.n_in, Lf, p.E, ids_sm, ctl,
+                             reinterpret_cast<uint32_t*>(red0), on_ticket);
+  const int nu = nu_;
 
   // ---- up projection ---------------------------------------------------------------------
   const int R = nu * d_e;
@@ -150,10 +229,10 @@ expert_wide_kernel(const LeanParams p) {
       hidx[n] = -1;
       if (t < L && m < rows) {
         hidx[n] = (hq * Lf + tok0 + t) * d_e + (ra + m - (hq << sh));
-        if constexpr (MODE == 2) {
-          float v = __ldcg(p.lg.a0 + (tok0 + t) * p.E + id);
+        if constexpr (MODE >= 2) {
+          float v = __ldcg(lg.a0 + (tok0 + t) * p.E + id);
           v = v > 0.0f ? v : 0.0f;
-          sc[n] = __ldg(p.lg.gain + id) * v * reinterpret_cast<const float*>(ctl + 104)[tok0 + t];
+          sc[n] = __ldg(lg.gain + id) * v * reinterpret_cast<const float*>(ctl + 104)[tok0 + t];
         } else {
           sc[n] = __ldcg(p.scores + (tok0 + t) * p.E + id);
         }
@@ -260,7 +339,8 @@ expert_wide_kernel(const LeanParams p) {
     __threadfence();
     asm volatile("red.relaxed.gpu.global.add.u64 [%0], 1;" ::"l"(p.ready + slot) : "memory");
     // (the slot's counter of the logit hand-over advances in step, see expert_lean_kernel)
-    asm volatile("red.relaxed.gpu.global.add.u64 [%0], 1;" ::"l"(p.ready2 + slot) : "memory");
+    if constexpr (MODE != 3)
+      asm volatile("red.relaxed.gpu.global.add.u64 [%0], 1;" ::"l"(p.ready2 + slot) : "memory");
   }
 
   // ---- down projection -------------------------------------------------------------------
@@ -501,7 +581,7 @@ expert_wide_kernel(const LeanParams p) {
   }
   // CTA 0 publishes the routing it derived (after the wait: earlier readers are done)
   if (blockIdx.x == 0) {
-    if (p.lg.a0 != nullptr && p.pub_scores != nullptr) {
+    if (lg.a0 != nullptr && p.pub_scores != nullptr) {
       const int words = (p.E + 31) >> 5;
       const float* rinv = reinterpret_cast<const float*>(ctl + 104);
       for (int t = tid >> 5; t < Lf; t += kNT / 32) {
@@ -509,9 +589,9 @@ expert_wide_kernel(const LeanParams p) {
           const int e = 32 * w + lane;
           float sv = 0.0f;
           if (e < p.E) {
-            float v = __ldcg(p.lg.a0 + (size_t)t * p.E + e);
+            float v = __ldcg(lg.a0 + (size_t)t * p.E + e);
             v = v > 0.0f ? v : 0.0f;
-            sv = __ldg(p.lg.gain + e) * v * rinv[t];
+            sv = __ldg(lg.gain + e) * v * rinv[t];
             p.pub_scores[(size_t)t * p.E + e] = sv;
           }
           const uint32_t m = __ballot_sync(0xffffffffu, sv != 0.0f);

@@ -520,12 +520,12 @@ def test_router_ahead_mixed_sequence():
 # ----------------------------------------------------------------------------
 # whole layer: the benchmark configurations
 # ----------------------------------------------------------------------------
-def check_layer_router_on(layer, dw, w, x, L, bias=None, want_out=False):
+def check_layer_router_on(layer, dw, w, x, L, bias=None, want_out=False, call_flags=0):
     """One blockffn_layer_forward call against the oracle. No chunk is ever skipped: where a
     mask bit differs from the oracle's (allowed only inside the band around a zero logit), the
     output is compared with the oracle FFN driven by the library's own scores and union."""
     ref = oracle.layer_forward(x, w["W_r"], w["gain"], w["U"], w["D"], bias=bias, union_only=True)
-    res = layer.forward(dw, B.to_device_bf16(x))
+    res = layer.forward(dw, B.to_device_bf16(x), call_flags=call_flags)
     torch.cuda.synchronize()
     E = layer.E
     got_s = res.scores.cpu().numpy()
@@ -552,6 +552,23 @@ def check_layer_router_on(layer, dw, w, x, L, bias=None, want_out=False):
     if want_out:
         return res.out.cpu().numpy()
     return ref, n
+
+
+@pytest.mark.parametrize("flag", [0, B.CALL_INDEPENDENT_X])
+@pytest.mark.parametrize("L", [9, 16, 17, 32])
+def test_router_on_long_chunks(L, flag):
+    """blockffn_layer_forward on chunks of more than 8 tokens: the router runs inside the
+    long-chunk kernel (8 tokens per pass), with and without the x-stable promise; several calls
+    in a row on one handle."""
+    sh, seed = I.SHAPES[3], I.config_seed(3)
+    w = I.make_layer(sh, seed, bias_shift=I.ROUTER_BIAS_SHIFT)
+    layer = B.Layer(sh.d, sh.E, sh.d_e, L_max=32)
+    dw = layer.upload_weights(w)
+    for chunk in range(3):
+        x = I.make_correlated_x(sh.d, L, 0.9, seed, chunk=40 + chunk)
+        check_layer_router_on(layer, dw, w, x, L, bias=w["bias"], call_flags=flag)
+    hs = layer.stats_host()
+    assert hs.n_chunks == 3 and hs.n_tokens == 3 * L
 
 
 @pytest.mark.parametrize("variant", VARIANTS)
