@@ -841,7 +841,9 @@ def extras(args, torch, device, peak):
         del probe
     for name, r in (("iid_tokens", None), ("correlated_tokens", rho)):
         wl = RouterWorkload(chunks, device, r, n_copies)
+        n0 = wl.layer.launch_count()
         ms = timed(wl)
+        launches = (wl.layer.launch_count() - n0) / (2 * chunks)     # capture() enqueues the step twice
         hs = wl.layer.stats_host()
         tls, ufrac = wl.sparsity()
         us = ms * 1e3 / chunks
@@ -855,7 +857,7 @@ def extras(args, torch, device, peak):
         rr = reuse.cpu().numpy()
         full[name] = {"rho": r, "us_per_call": us, "tls": tls, "mean_union": mean_u,
                       "GBps": mean_u * sh.expert_bytes / us / 1e3,
-                      "launches_per_call": 2,
+                      "launches_per_call": launches,
                       "reuse_ratio": float(rr[0] / rr[1]) if rr[1] > 0 else None}
         if r is None:                   # stage level: the router entry point from its own graph
             st2 = torch.cuda.Stream(device)
