@@ -60,8 +60,8 @@ expert_wide_kernel(const LeanParams p) {
   };
   // (the caller's union list: the scores are first read at the end of the first stage)
   if constexpr (MODE == 1) prefetch_l2(p.scores, Lf * p.E * 4);
-  // MODE 3: the router inside the kernel, as in expert_lean_kernel, 8 tokens per pass. The
-  // first 8 warps of the CTA do it (a row has at most 256 pieces of 16 bytes).
+  // MODE 3: the router inside the kernel, as in expert_lean_kernel, 8 tokens per pass and team
+  // (a row has at most 256 pieces of 16 bytes: one per thread of a team).
   RouterLogits lg3 = p.lg;
   if constexpr (MODE == 3) {
     if (tid == 0) on_ticket();
@@ -71,50 +71,53 @@ expert_wide_kernel(const LeanParams p) {
     float* a0 = p.logit_ring + (size_t)rslot * p.logit_slot;
     lg3.a0 = a0;
     const int chunks = d >> 3;
-    float* wsum = red0;                        // [8 warps][8 tokens]
-    const int w8 = tid >> 5;                   // warp of the CTA
-    for (int e = bx; e < p.E; e += G) {
-      uint4 wv = make_uint4(0u, 0u, 0u, 0u);
-      if (tid < chunks) wv = __ldg(reinterpret_cast<const uint4*>(p.W_r + (size_t)e * d) + tid);
-      const uint32_t wp[4] = {wv.x, wv.y, wv.z, wv.w};
-      for (int t0 = 0; t0 < Lf; t0 += 8) {
-        float acc[8];
+    // Work units: (expert, pass of 8 tokens), dealt out over the teams of all CTAs, so that the
+    // router part of a 32-token chunk is as many short steps per team as it takes (with whole
+    // experts per CTA the CTAs that get two of them held everyone up at the hand-over).
+    float* wsum = red0 + team * 64;            // [8 warps][8 tokens] per team
+    const int npass = (Lf + 7) >> 3;
+    const int units = p.E * npass, stride = G * TEAMS;
+    const int rounds = (units + stride - 1) / stride;      // the same for every thread: barriers inside
+    for (int k = 0; k < rounds; ++k) {
+      const int u = k * stride + bx * TEAMS + team;
+      const bool live = u < units;
+      const int e = live ? u / npass : 0, t0 = live ? 8 * (u - e * npass) : 0;
+      float acc[8];
 #pragma unroll
-        for (int t = 0; t < 8; ++t) acc[t] = 0.0f;
-        if (tid < chunks) {
-          uint4 xv[8];
+      for (int t = 0; t < 8; ++t) acc[t] = 0.0f;
+      if (live && ttid < chunks) {
+        const uint4 wv = __ldg(reinterpret_cast<const uint4*>(p.W_r + (size_t)e * d) + ttid);
+        const uint32_t wp[4] = {wv.x, wv.y, wv.z, wv.w};
+        uint4 xv[8];
 #pragma unroll
-          for (int t = 0; t < 8; ++t)
-            xv[t] = t0 + t < Lf ? __ldcg(reinterpret_cast<const uint4*>(p.x + (size_t)(t0 + t) * d) + tid)
-                                : make_uint4(0u, 0u, 0u, 0u);
+        for (int t = 0; t < 8; ++t)
+          xv[t] = t0 + t < Lf ? __ldcg(reinterpret_cast<const uint4*>(p.x + (size_t)(t0 + t) * d) + ttid)
+                              : make_uint4(0u, 0u, 0u, 0u);
 #pragma unroll
-          for (int t = 0; t < 8; ++t) {
-            const uint32_t xp[4] = {xv[t].x, xv[t].y, xv[t].z, xv[t].w};
+        for (int t = 0; t < 8; ++t) {
+          const uint32_t xp[4] = {xv[t].x, xv[t].y, xv[t].z, xv[t].w};
 #pragma unroll
-            for (int q = 0; q < 4; ++q) {
-              acc[t] = fmaf(bf16_lo(wp[q]), bf16_lo(xp[q]), acc[t]);
-              acc[t] = fmaf(bf16_hi(wp[q]), bf16_hi(xp[q]), acc[t]);
-            }
+          for (int q = 0; q < 4; ++q) {
+            acc[t] = fmaf(bf16_lo(wp[q]), bf16_lo(xp[q]), acc[t]);
+            acc[t] = fmaf(bf16_hi(wp[q]), bf16_hi(xp[q]), acc[t]);
           }
         }
-        if (w8 < kWarps) {
-#pragma unroll
-          for (int t = 0; t < 8; ++t) {
-            float v = acc[t];
-#pragma unroll
-            for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-            if (lane == 0) wsum[w8 * 8 + t] = v;
-          }
-        }
-        __syncthreads();
-        if (tid < 8 && t0 + tid < Lf) {
-          float v = p.bias ? p.bias[e] : 0.0f;
-#pragma unroll
-          for (int q = 0; q < kWarps; ++q) v += wsum[q * 8 + tid];
-          a0[(size_t)(t0 + tid) * p.E + e] = v;
-        }
-        __syncthreads();
       }
+#pragma unroll
+      for (int t = 0; t < 8; ++t) {
+        float v = acc[t];
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+        if (lane == 0) wsum[warp * 8 + t] = v;
+      }
+      __syncthreads();
+      if (live && ttid < 8 && t0 + ttid < Lf) {
+        float v = p.bias ? p.bias[e] : 0.0f;
+#pragma unroll
+        for (int q = 0; q < kWarps; ++q) v += wsum[q * 8 + ttid];
+        a0[(size_t)(t0 + ttid) * p.E + e] = v;
+      }
+      __syncthreads();
     }
     if (tid == kNT - 1) {
       __threadfence();
