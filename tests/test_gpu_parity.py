@@ -414,6 +414,27 @@ def test_bounded_wait_expires_cleanly(L, kind):
     assert layer.last_status() == 0
 
 
+@pytest.mark.parametrize("L", [8, 32])
+def test_bounded_wait_expires_cleanly_with_the_router_inside(L):
+    """The same for a layer call whose router runs inside the kernel: its first hand-over (the
+    logits) is a bounded wait of the same kind. The call comes back with the status bit set and
+    out untouched; a handle without the test bit then gives the right result."""
+    sh, seed = I.SHAPES[3], I.config_seed(3)
+    w = I.make_layer(sh, seed, bias_shift=I.ROUTER_BIAS_SHIFT)
+    x = I.make_correlated_x(sh.d, L, 0.9, seed, chunk=77)
+    held = B.Layer(sh.d, sh.E, sh.d_e, L_max=L, flags=B.CFG_TEST_EXPIRE_WAIT)
+    dw = held.upload_weights(w)
+    out = torch.full((L, sh.d), 7.0, device="cuda")
+    for _ in range(2):
+        held.forward(dw, B.to_device_bf16(x), out=out, call_flags=B.CALL_INDEPENDENT_X)
+        assert held.last_status(clear=True) == B.DEV_WAIT_EXPIRED
+        assert bool((out == 7.0).all())
+    layer = B.Layer(sh.d, sh.E, sh.d_e, L_max=L)
+    dw2 = layer.upload_weights(w)
+    check_layer_router_on(layer, dw2, w, x, L, bias=w["bias"], call_flags=B.CALL_INDEPENDENT_X)
+    assert layer.last_status() == 0
+
+
 def test_host_side_argument_errors():
     layer = B.Layer(256, 16, 64, L_max=4)
     w = B.make_weights()
