@@ -646,11 +646,14 @@ def run_ours(args):
 class RouterWorkload:
     """Config 3 with the router on: blockffn_layer_forward over correlated or iid chunks."""
 
-    def __init__(self, chunks, device, rho, n_copies):
+    def __init__(self, chunks, device, rho, n_copies, L=None):
         import torch
         from paper_2507_08771_b200 import binding as B
         self.torch, self.B, self.chunks = torch, B, chunks
-        self.sh = sh = I.SHAPES[3]
+        sh = I.SHAPES[3]
+        if L is not None:
+            sh = I.Shape(sh.name, d=sh.d, E=sh.E, d_e=sh.d_e, L=L, union_frac=sh.union_frac)
+        self.sh = sh
         seed = I.config_seed(3)
         self.layer = B.Layer(sh.d, sh.E, sh.d_e, L_max=sh.L, device=device)
         w = I.make_layer(sh, seed, bias_shift=I.ROUTER_BIAS_SHIFT)
@@ -859,6 +862,17 @@ def extras(args, torch, device, peak):
                       "GBps": mean_u * sh.expert_bytes / us / 1e3,
                       "launches_per_call": launches,
                       "reuse_ratio": float(rr[0] / rr[1]) if rr[1] > 0 else None}
+        if r is not None:               # longer chunks of the same correlated tokens, router on
+            for Ll in (16, 32):
+                wll = RouterWorkload(chunks, device, r, n_copies, L=Ll)
+                msl = timed(wll)
+                tl, ul = wll.sparsity()
+                usl = msl * 1e3 / chunks
+                full[f"{name}_L{Ll}"] = {"rho": r, "L": Ll, "us_per_call": usl, "tls": tl,
+                                         "mean_union": ul * sh.E,
+                                         "GBps": ul * sh.E * sh.expert_bytes / usl / 1e3}
+                del wll
+                torch.cuda.empty_cache()
         if r is None:                   # stage level: the router entry point from its own graph
             st2 = torch.cuda.Stream(device)
             g2 = capture(torch, st2, wl.enqueue_router_only)
